@@ -1,0 +1,195 @@
+"""Pins for the oracle's FFN / combine half and for every gradient.
+
+Forward: library SwiGLU (torch float64) for one expert and for the dense reduction
+(expert choice with C = T selects every pair, so Y[t] = sum_i delta_ti E_i(x_t)), the
+dispatch/CSR identity, permutation equivariance.  Backward: central finite differences
+of the double-precision oracle with the selection frozen, torch.autograd of the dense
+reduction, and the orthogonality identities that scale invariance of the cosine forces.
+"""
+import numpy as np
+import pytest
+import torch
+import torch.nn.functional as F
+
+from gen import workloads as gw
+from oracle import binding as ob
+
+
+@pytest.fixture(scope="module")
+def o32():
+    return ob.Oracle("f32")
+
+
+@pytest.fixture(scope="module")
+def o64():
+    return ob.Oracle("f64")
+
+
+def problem(seed, T=12, d=8, D=2, E=3, h=6):
+    rng = np.random.default_rng(seed)
+    q, _ = np.linalg.qr(rng.standard_normal((d // D, E)))
+    return dict(X=rng.standard_normal((T, d)), R=q.T.copy(),
+                W1g=rng.standard_normal((E, h, d)) / np.sqrt(d),
+                W1u=rng.standard_normal((E, h, d)) / np.sqrt(d),
+                W2=rng.standard_normal((E, d, h)) / np.sqrt(d),
+                dY=rng.standard_normal((T, d)))
+
+
+def torch_swiglu(x, W1g, W1u, W2):
+    return (F.silu(x @ W1g.T) * (x @ W1u.T)) @ W2.T
+
+
+def torch_affinity(X, R, D):
+    """cos(x_t, w_i) with w_i the dense d-vector of the GrAP router (library ops only)."""
+    W = R.repeat_interleave(D, dim=1) / D
+    return F.cosine_similarity(X[:, None, :], W[None, :, :], dim=-1, eps=0.0)
+
+
+def test_single_expert_is_library_swiglu(o64):
+    p = problem(1, E=1, D=2)
+    fw = o64.forward(p["X"], p["R"], p["W1g"], p["W1u"], p["W2"], D=2, k=1, capacity=12,
+                     mode=ob.MODE_TCR)
+    t = {k: torch.from_numpy(v) for k, v in p.items()}
+    ref = torch_affinity(t["X"], t["R"], 2) * torch_swiglu(t["X"], t["W1g"][0], t["W1u"][0], t["W2"][0])
+    assert np.allclose(fw.Y, ref.numpy(), rtol=1e-12, atol=1e-13)
+    assert fw.route.counts.tolist() == [12]
+
+
+def dense_moe_torch(t, D):
+    delta = torch_affinity(t["X"], t["R"], D)
+    Y = 0
+    for i in range(t["R"].shape[0]):
+        Y = Y + delta[:, i:i + 1] * torch_swiglu(t["X"], t["W1g"][i], t["W1u"][i], t["W2"][i])
+    return Y
+
+
+def test_expert_choice_full_capacity_is_dense_moe_fwd_bwd(o64):
+    """C = T in expert choice: the general MoE form with every gate active.  Forward and
+    all five gradients against torch.autograd in float64."""
+    p = problem(2)
+    fw = o64.forward(p["X"], p["R"], p["W1g"], p["W1u"], p["W2"], D=2, k=2, capacity=12,
+                     mode=ob.MODE_ECR)
+    bw = o64.backward(fw, p["X"], p["R"], p["W1g"], p["W1u"], p["W2"], p["dY"])
+    t = {k: torch.from_numpy(v).requires_grad_(k != "dY") for k, v in p.items()}
+    Y = dense_moe_torch(t, 2)
+    (Y * t["dY"]).sum().backward()
+    assert np.allclose(fw.Y, Y.detach().numpy(), rtol=1e-12, atol=1e-13)
+    for name, got in [("X", bw.dX), ("R", bw.dR), ("W1g", bw.dW1g), ("W1u", bw.dW1u), ("W2", bw.dW2)]:
+        want = t[name].grad.numpy()
+        assert np.allclose(got, want, rtol=1e-10, atol=1e-12), name
+
+
+def test_dispatch_then_inverse_is_identity(o32):
+    w = gw.WORKLOADS["tiny"]
+    R = gw.expert_embeddings(w)
+    X = gw.tokens(w, R)
+    delta, *_ = o32.affinity(X, R, D=w.D)
+    rt = o32.select(delta, w.k, ob.MODE_TCR, w.capacity, w.C_stride)
+    Xp = o32.dispatch(X, rt)
+    valid = rt.slot_token >= 0
+    assert np.array_equal(Xp[valid], X[rt.slot_token[valid]]) and np.all(Xp[~valid] == 0)
+    back = o32.dispatch_bwd(Xp, rt)           # sums the rows of each token
+    nrows = np.diff(rt.tok_ptr)[:, None]
+    assert np.allclose(back, nrows * X, rtol=1e-6, atol=1e-6)
+
+
+def test_combine_weights_are_selected_affinities(o32):
+    w = gw.WORKLOADS["tiny"]
+    R = gw.expert_embeddings(w)
+    X = gw.tokens(w, R)
+    delta, *_ = o32.affinity(X, R, D=w.D)
+    rt = o32.select(delta, w.k, ob.MODE_TCR, 100, w.C_stride)
+    O = np.ones((w.E * w.C_stride, 4), np.float32)      # combine then returns sum of gates
+    Y = o32.combine(O, rt)
+    want = np.zeros(w.T)
+    for r in np.nonzero(rt.slot_token >= 0)[0]:
+        want[rt.slot_token[r]] += float(delta[rt.slot_token[r], r // w.C_stride])
+    assert np.allclose(Y[:, 0], want, atol=1e-6)
+    unrouted = np.diff(rt.tok_ptr) == 0
+    assert unrouted.any() and np.all(Y[unrouted] == 0)
+
+
+@pytest.mark.parametrize("mode", [ob.MODE_TCR, ob.MODE_ECR])
+def test_permutation_equivariance(o64, mode):
+    p = problem(3, T=16)
+    kw = dict(D=2, k=2, capacity=7, mode=mode)
+    base = o64.forward(p["X"], p["R"], p["W1g"], p["W1u"], p["W2"], **kw).Y
+    perm = np.random.default_rng(0).permutation(16)
+    Yp = o64.forward(p["X"][perm], p["R"], p["W1g"], p["W1u"], p["W2"], **kw).Y
+    assert np.allclose(Yp, base[perm], atol=1e-13)
+    ep = np.array([2, 0, 1])
+    Ye = o64.forward(p["X"], p["R"][ep], p["W1g"][ep], p["W1u"][ep], p["W2"][ep], **kw).Y
+    assert np.allclose(Ye, base, atol=1e-13)
+
+
+@pytest.mark.parametrize("mode,cap", [(ob.MODE_TCR, 5), (ob.MODE_ECR, 5), (ob.MODE_TCR, 3)])
+def test_gradients_by_finite_differences(o64, mode, cap):
+    p = problem(4)
+    kw = dict(D=2, k=2, capacity=cap, mode=mode)
+    fw = o64.forward(p["X"], p["R"], p["W1g"], p["W1u"], p["W2"], **kw)
+    assert fw.route.dropped > 0                       # the capacity bound is active
+    bw = o64.backward(fw, p["X"], p["R"], p["W1g"], p["W1u"], p["W2"], p["dY"])
+
+    def loss(q):
+        y = o64.forward(q["X"], q["R"], q["W1g"], q["W1u"], q["W2"], route=fw.route, **kw).Y
+        return float((y * p["dY"]).sum())
+
+    eps = 1e-6
+    grads = dict(X=bw.dX, R=bw.dR, W1g=bw.dW1g, W1u=bw.dW1u, W2=bw.dW2)
+    rng = np.random.default_rng(5)
+    for name, g in grads.items():
+        flat_n = p[name].size
+        picks = range(flat_n) if flat_n <= 128 else rng.choice(flat_n, 96, replace=False)
+        scale = np.abs(g).max()
+        for idx in picks:
+            q = {k: v.copy() for k, v in p.items()}
+            q[name].reshape(-1)[idx] += eps
+            up = loss(q)
+            q[name].reshape(-1)[idx] -= 2 * eps
+            fd = (up - loss(q)) / (2 * eps)
+            assert abs(fd - g.reshape(-1)[idx]) <= 2e-7 * scale + 1e-9, (name, idx, fd, g.reshape(-1)[idx])
+
+
+def test_router_gradient_orthogonality(o64):
+    """The cosine ignores the scale of x_t and of R_i, so the router path's gradient
+    satisfies <dX_router[t], x_t> = 0 and <dR_i, R_i> = 0."""
+    p = problem(6)
+    fw = o64.forward(p["X"], p["R"], p["W1g"], p["W1u"], p["W2"], D=2, k=2, capacity=6, mode=ob.MODE_TCR)
+    bw = o64.backward(fw, p["X"], p["R"], p["W1g"], p["W1u"], p["W2"], p["dY"])
+    dX_router = bw.dX - bw.dX_ffn
+    assert np.abs(dX_router).max() > 1e-3
+    assert np.allclose((dX_router * p["X"]).sum(1), 0, atol=1e-12)
+    assert np.allclose((bw.dR * p["R"]).sum(1), 0, atol=1e-12)
+
+
+def test_f32_layer_close_to_f64(o32, o64):
+    w = gw.scaled(gw.WORKLOADS["tiny"], T=128, h=64)
+    inp = gw.make_inputs(w)
+    kw = dict(D=w.D, k=w.k, capacity=w.capacity, mode=ob.MODE_TCR)
+    a = o32.forward(inp["X"], inp["R"], inp["W1g"], inp["W1u"], inp["W2"], **kw)
+    b = o64.forward(inp["X"], inp["R"], inp["W1g"], inp["W1u"], inp["W2"], route=a.route, **kw)
+    assert np.max(np.abs(a.Y - b.Y)) <= 1e-5 * np.sqrt((b.Y ** 2).mean())
+    ga = o32.backward(a, inp["X"], inp["R"], inp["W1g"], inp["W1u"], inp["W2"], inp["dY"])
+    gb = o64.backward(b, inp["X"], inp["R"], inp["W1g"], inp["W1u"], inp["W2"], inp["dY"])
+    for f in ("dX", "dR", "dW1g", "dW1u", "dW2"):
+        x, y = getattr(ga, f), getattr(gb, f)
+        assert np.max(np.abs(x - y)) <= 2e-5 * np.sqrt((y ** 2).mean()), f
+
+
+def test_oracle_is_thread_count_independent(o32):
+    w = gw.scaled(gw.WORKLOADS["tiny"], T=96, h=32)
+    inp = gw.make_inputs(w)
+    kw = dict(D=w.D, k=w.k, capacity=w.capacity, mode=ob.MODE_TCR)
+    n = ob.set_threads(0)
+    try:
+        ob.set_threads(1)
+        a = o32.forward(inp["X"], inp["R"], inp["W1g"], inp["W1u"], inp["W2"], **kw)
+        ga = o32.backward(a, inp["X"], inp["R"], inp["W1g"], inp["W1u"], inp["W2"], inp["dY"])
+        ob.set_threads(4)
+        b = o32.forward(inp["X"], inp["R"], inp["W1g"], inp["W1u"], inp["W2"], **kw)
+        gb = o32.backward(b, inp["X"], inp["R"], inp["W1g"], inp["W1u"], inp["W2"], inp["dY"])
+    finally:
+        ob.set_threads(n)
+    assert np.array_equal(a.Y, b.Y)
+    for f in ("dX", "dR", "dW1g", "dW1u", "dW2"):
+        assert np.array_equal(getattr(ga, f), getattr(gb, f))
