@@ -1,0 +1,241 @@
+/*
+ * libetr — forward and backward pass of an Expert-Token Resonance (ETR) MoE layer
+ * (arXiv 2406.00023) on one NVIDIA B200 (sm_100a).
+ *
+ * Plain C ABI.  Unless a parameter says "host", every data pointer is DEVICE memory
+ * owned by the caller; the library allocates no device memory.  `stream` is a
+ * cudaStream_t passed as void* (NULL = default stream); every call only enqueues work
+ * on it and returns without synchronising, except etr_read_stats and
+ * etr_layer_step_host.
+ *
+ * Notation (the paper's in brackets): T tokens [s], d hidden size, D GrAP group size,
+ * m = d/D pooled width, E experts [n], k experts per token [l], C per-expert capacity,
+ * h FFN hidden size.
+ *
+ * Layouts: row-major, innermost index contiguous.
+ *   X, Y, dY, dX [T,d]      R, dR [E,m] fp32        delta [T,E] fp32      Z [T,m] fp32
+ *   W1g, W1u [E,h,d]        W2 [E,d,h]              (gradients: same shape and dtype)
+ *   Xp, O, dO, dXp [E*C_stride, d]                  G, U, H, dG, dU [E*C_stride, h]
+ * C_stride = capacity rounded up to a multiple of 128.  Expert i owns rows
+ * [i*C_stride, (i+1)*C_stride); the first counts[i] of them are in use.  Rows from
+ * counts[i] up to the next multiple of 128 are kept zero by the library ("pad rows");
+ * rows beyond that are never read or written.
+ * Activations and expert weights are `dtype` (fp32 or bf16); routing tensors are fp32,
+ * maps are int32.  All accumulation is fp32.
+ *
+ * Requirements checked on the host before anything is launched (ETR_ERR_* otherwise):
+ *   d % D == 0, d % 8 == 0, h % 8 == 0, 1 <= k <= E <= 256, E <= m, 1 <= capacity,
+ *   T >= 1, T*E < 2^31, data pointers 16-byte aligned and non-NULL.
+ *   bf16 tensor-core path: d % 64 == 0 and h % 64 == 0 (else ETR_ERR_UNSUPPORTED).
+ *
+ * Errors: every function returns an etr_status.  Argument errors are reported before
+ * any launch.  A launch failure maps to ETR_ERR_CUDA.  Device-side problems (a bounded
+ * wait in the GEMM pipeline that ran out) never trap: the kernel records a code in
+ * etr_stats.error_word, stops issuing work and returns; etr_read_stats reports it as
+ * ETR_ERR_TIMEOUT.
+ */
+#ifndef ETR_H_
+#define ETR_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  ETR_OK = 0,
+  ETR_ERR_ARG = 1,          /* NULL pointer, non-positive size, bad enum */
+  ETR_ERR_SHAPE = 2,        /* sizes violate the divisibility / range rules above */
+  ETR_ERR_ALIGN = 3,        /* a data pointer is not 16-byte aligned */
+  ETR_ERR_WORKSPACE = 4,    /* caller-provided buffer too small */
+  ETR_ERR_CUDA = 5,         /* CUDA runtime / driver call failed */
+  ETR_ERR_TIMEOUT = 6,      /* a bounded device-side wait expired (see etr_stats) */
+  ETR_ERR_UNSUPPORTED = 7   /* valid request the library has no kernel for */
+} etr_status;
+
+typedef enum { ETR_F32 = 0, ETR_BF16 = 1 } etr_dtype;
+typedef enum { ETR_MODE_AUTO = 0, ETR_MODE_TCR = 1, ETR_MODE_ECR = 2 } etr_mode;
+typedef enum { ETR_GEMM_AUTO = 0, ETR_GEMM_SIMT = 1, ETR_GEMM_TCGEN05 = 2 } etr_gemm_impl;
+
+/* Immutable description of one layer call (host struct, passed by pointer). */
+typedef struct etr_config {
+  int32_t T, d, D, E, k, h;
+  int32_t capacity;           /* upper bound on rows per expert, ceil(cf*T*k/E) */
+  int32_t c_floor;            /* lower clamp of the adaptive bound (>= 1) */
+  int32_t adaptive;           /* 0: C = capacity.  1: C = clamp(ceil(C_min), c_floor, capacity) */
+  float delta_max_override;   /* < 0: use this batch's max affinity; >= 0: use this value */
+  int64_t step, switch_step;  /* ETR_MODE_AUTO: token choice while step < switch_step */
+  int32_t mode;               /* etr_mode */
+  int32_t dtype;              /* etr_dtype of activations and expert weights */
+  int32_t gemm_impl;          /* etr_gemm_impl; AUTO = tcgen05 for bf16, SIMT for fp32 */
+  int32_t reserved;
+} etr_config;
+
+/* Per-call scalars produced and consumed on the device (device struct, 64 bytes). */
+typedef struct etr_stats {
+  int32_t mode;               /* etr_mode actually used */
+  int32_t C;                  /* capacity actually used */
+  int32_t dropped;            /* candidate (token,expert) pairs cut by the capacity */
+  int32_t unrouted;           /* tokens that ended up in no expert */
+  float delta_max;            /* max affinity of this batch */
+  uint32_t delta_max_key;     /* order-preserving integer image of delta_max */
+  int32_t error_word;         /* 0, or a code left by a kernel that gave up a wait */
+  int32_t rows_total;         /* sum of counts */
+  int32_t reserved[8];
+} etr_stats;
+
+/* Routing maps (host struct of device pointers). */
+typedef struct etr_route {
+  int32_t* topk_idx;          /* [T,k]  token choice: experts by descending affinity; -1 in expert choice */
+  int32_t* counts;            /* [E]    rows in use per expert */
+  int32_t* slot_token;        /* [E*C_stride] token id held by each row, -1 if unused */
+  float* gate;                /* [E*C_stride] affinity of that (token, expert) pair, 0 if unused */
+  int32_t* tok_ptr;           /* [T+1]  CSR: rows of token t are tok_row[tok_ptr[t] .. tok_ptr[t+1]) */
+  int32_t* tok_row;           /* [E*C_stride] row ids, ascending expert order inside a token */
+} etr_route;
+
+/* Every device buffer a forward+backward needs besides inputs, parameters and outputs
+ * (host struct of device pointers).  etr_buffers_bind carves them out of one block. */
+typedef struct etr_buffers {
+  etr_stats* stats;
+  etr_route route;
+  float* delta;               /* [T,E] */
+  float* Z;                   /* [T,m] pooled tokens, saved for the router gradient */
+  float* xnorm;               /* [T] */
+  float* rnorm;               /* [E] */
+  void* Xp; void* G; void* U; void* H; void* O;          /* forward activations */
+  void* dO; void* dG; void* dU; void* dXp; float* dgate; /* backward activations */
+  void* ws;                   /* scratch, ws_bytes long */
+  size_t ws_bytes;
+  /* staging used only by etr_layer_step_host */
+  void* X_dev; void* dY_dev; void* Y_dev; void* dX_dev;
+} etr_buffers;
+
+const char* etr_status_string(etr_status s);
+
+/* Checks a config against the rules in the header comment. */
+etr_status etr_validate(const etr_config* cfg);
+
+/* C_stride for a config (capacity rounded up to 128). */
+int32_t etr_c_stride(const etr_config* cfg);
+
+/* Scratch bytes the calls below need in `ws` (max over all of them). */
+etr_status etr_workspace_bytes(const etr_config* cfg, size_t* bytes);
+
+/* Size of one block holding every etr_buffers member, and the carving of such a block
+ * (base must be 256-byte aligned).  with_host_staging != 0 also reserves X_dev, dY_dev,
+ * Y_dev, dX_dev. */
+etr_status etr_buffers_bytes(const etr_config* cfg, int with_host_staging, size_t* bytes);
+etr_status etr_buffers_bind(const etr_config* cfg, int with_host_staging, void* base, size_t bytes,
+                            etr_buffers* out);
+
+/* ---- forward stages ---------------------------------------------------------------- */
+
+/* GrAP pooling and cosine affinity ("Cost-Efficient Sparse Expert-Token Affinity": the
+ * W_aff equations and delta_ti = cos(x_t, w_i)), generalised to learned embeddings:
+ *   z_t = avgpool_D(x_t);  delta_ti = sqrt(D) <z_t, R_i> / (||x_t|| ||R_i||), 0 if a norm is 0.
+ * Writes delta, xnorm, rnorm, optionally Z (NULL to skip), and raises
+ * stats->delta_max_key to the batch maximum.  stats must have been zeroed by the caller
+ * (etr_layer_forward does it) — the call only ever raises the key. */
+etr_status etr_affinity(const etr_config* cfg, const void* X, const float* R, float* delta,
+                        float* Z, float* xnorm, float* rnorm, etr_stats* stats, void* stream);
+
+/* Bidirectional selection ("Routing Strategy": Top-l experts per token, then each expert
+ * keeps C of its assigned tokens, highest affinity first) under the capacity
+ *   C = capacity, or clamp(ceil((1/E) exp{d dm^2/(2-dm^2)}), c_floor, capacity) when adaptive
+ * (Remark of "Dynamic Lower Bound Module for Expert Capacity"), dm = delta_max_override
+ * or the batch maximum left in stats by etr_affinity.  Mode: cfg->mode, or from step.
+ * Ties go to the lower index.  Kept tokens of an expert are stored in ascending token
+ * order.  Fills every member of route and stats->{mode,C,dropped,unrouted,delta_max,
+ * rows_total}.  ws: etr_workspace_bytes. */
+etr_status etr_select(const etr_config* cfg, const float* delta, etr_stats* stats,
+                      const etr_route* route, void* ws, void* stream);
+
+/* Token rearrangement: Xp[r,:] = X[slot_token[r],:] for rows in use, 0 for pad rows. */
+etr_status etr_dispatch(const etr_config* cfg, const void* X, const etr_route* route, void* Xp,
+                        void* stream);
+
+/* Expert networks as a grouped GEMM over the rows in use (SwiGLU FFN, no bias):
+ *   G = Xp W1g_i^T, U = Xp W1u_i^T, H = silu(G) * U, O = H W2_i^T   for expert i's rows.
+ * G, U, H are kept for the backward pass. */
+etr_status etr_expert_ffn(const etr_config* cfg, const etr_route* route, const void* Xp,
+                          const void* W1g, const void* W1u, const void* W2,
+                          void* G, void* U, void* H, void* O, etr_stats* stats, void* ws,
+                          void* stream);
+
+/* Gate-weighted sum of the general MoE form, MoE(x) = sum_t sum_i G_i(x_t) E_i(x_t), with
+ * the affinity as the gate:  Y[t,:] = sum_{r in rows(t)} gate[r] O[r,:]  (0 if no rows). */
+etr_status etr_combine(const etr_config* cfg, const etr_route* route, const void* O, void* Y,
+                       void* stream);
+
+/* ---- backward stages (the paper states no backward; these are the derivatives of the
+ *      forward definitions above with the selection held constant) -------------------- */
+
+/* dO[r,:] = gate[r] dY[t(r),:];  dgate[r] = <dY[t(r),:], O[r,:]>;  pad rows get 0. */
+etr_status etr_combine_bwd(const etr_config* cfg, const etr_route* route, const void* dY,
+                           const void* O, void* dO, float* dgate, void* stream);
+
+/* dH = dO W2_i;  dG = dH*U*s*(1+G*(1-s)), dU = dH*G*s with s = sigmoid(G);
+ * dXp = dG W1g_i + dU W1u_i;  dW2_i = dO^T H;  dW1g_i = dG^T Xp;  dW1u_i = dU^T Xp.
+ * Experts with no rows get zero weight gradients. */
+etr_status etr_expert_ffn_bwd(const etr_config* cfg, const etr_route* route, const void* dO,
+                              const void* Xp, const void* G, const void* U, const void* H,
+                              const void* W1g, const void* W1u, const void* W2,
+                              void* dG, void* dU, void* dXp,
+                              void* dW1g, void* dW1u, void* dW2, etr_stats* stats, void* ws,
+                              void* stream);
+
+/* dX[t,:] = sum_{r in rows(t)} dXp[r,:]  (overwrites dX). */
+etr_status etr_dispatch_bwd(const etr_config* cfg, const etr_route* route, const void* dXp,
+                            void* dX, void* stream);
+
+/* d delta is non-zero only on selected pairs, where it equals dgate; it is therefore
+ * represented by (route, dgate) and this call only checks its arguments. */
+etr_status etr_select_bwd(const etr_config* cfg, const etr_route* route, const float* dgate);
+
+/* Router gradient.  With a = ||x_t||, b = ||R_i||, c = sqrt(D)/(a b), over selected pairs:
+ *   dX[t,q] += sum_i dgate_ti ( c R_i[q/D]/D - delta_ti x_t[q]/a^2 )      (ADDS to dX)
+ *   dR[i,j]  = sum_t dgate_ti ( c z_t[j]     - delta_ti R_i[j]/b^2 )      (overwrites dR)
+ * ws: etr_workspace_bytes. */
+etr_status etr_affinity_bwd(const etr_config* cfg, const void* X, const float* R,
+                            const float* delta, const float* Z, const float* xnorm,
+                            const float* rnorm, const etr_route* route, const float* dgate,
+                            void* dX, float* dR, void* ws, void* stream);
+
+/* ---- whole layer ---------------------------------------------------------------------- */
+
+/* Zeroes stats, then affinity, select, dispatch, expert_ffn, combine, in that order. */
+etr_status etr_layer_forward(const etr_config* cfg, const void* X, const float* R,
+                             const void* W1g, const void* W1u, const void* W2,
+                             const etr_buffers* buf, void* Y, void* stream);
+
+/* combine_bwd, expert_ffn_bwd, dispatch_bwd, affinity_bwd, in that order, on the buffers
+ * a preceding etr_layer_forward filled. */
+etr_status etr_layer_backward(const etr_config* cfg, const void* X, const float* R,
+                              const void* W1g, const void* W1u, const void* W2,
+                              const void* dY, const etr_buffers* buf,
+                              void* dX, float* dR, void* dW1g, void* dW1u, void* dW2,
+                              void* stream);
+
+/* One training step from HOST activations: copies X_host and dY_host (host, ideally pinned)
+ * to buf->X_dev / dY_dev, runs forward and backward, copies Y and dX back to Y_host and
+ * dX_host (host), and synchronises the stream.  Parameters and their gradients stay on
+ * the device.  buf must have been bound with host staging. */
+etr_status etr_layer_step_host(const etr_config* cfg, const void* X_host, const void* dY_host,
+                               const float* R, const void* W1g, const void* W1u, const void* W2,
+                               const etr_buffers* buf, void* Y_host, void* dX_host,
+                               float* dR, void* dW1g, void* dW1u, void* dW2, void* stream);
+
+/* Copies the device stats to the host and synchronises the stream.  Returns
+ * ETR_ERR_TIMEOUT if a kernel recorded an expired wait. */
+etr_status etr_read_stats(const etr_stats* stats_dev, etr_stats* stats_host, void* stream);
+
+/* Number of kernels launched by this library in the calling process so far. */
+int64_t etr_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ETR_H_ */

@@ -1,0 +1,347 @@
+// GrAP pooling + cosine affinity (forward) and the router gradient (backward).
+//
+// Forward, one CTA per tile of TB tokens:
+//   phase 0  R -> shared memory (rows padded so 128-bit reads of 8 different rows hit
+//            32 different banks), ||R_i|| by one warp per row
+//   phase 1  each warp streams its tokens' rows of X once with 16-byte loads, pools the
+//            D-groups in registers, accumulates ||x||^2, leaves z_t in shared memory
+//   phase 2  s = Z R^T register-tiled (2 tokens x 4 experts per thread, float4 operands),
+//            delta = sqrt(D) s / (||x|| ||R||), batch max through one atomicMax on the
+//            order-preserving integer image (exact and order independent)
+#include "common.cuh"
+
+namespace etr {
+
+constexpr int AFF_TB = 32;        // tokens per CTA
+constexpr int AFF_THREADS = 256;
+
+template <class T>
+__device__ inline void pool_token(const T* __restrict__ x, float* __restrict__ zrow, int d, int D,
+                                  int m, int lane, float& sumsq) {
+  const float invD = 1.0f / (float)D;
+  float sq = 0.f;
+  if (D % 8 == 0) {                 // a lane owns whole groups: D/8 vectors each
+    const int vpg = D / 8;
+#pragma unroll 4
+    for (int j = lane; j < m; j += 32) {
+      float s = 0.f;
+      for (int v = 0; v < vpg; ++v) {
+        Vec8<T> q = Vec8<T>::load(x + (size_t)j * D + v * 8);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) { s += q.v[e]; sq += q.v[e] * q.v[e]; }
+      }
+      zrow[j] = s * invD;
+    }
+  } else if (8 % D == 0) {          // a vector holds 8/D whole groups
+    const int gpv = 8 / D;
+#pragma unroll 4
+    for (int v = lane; v < d / 8; v += 32) {
+      Vec8<T> q = Vec8<T>::load(x + (size_t)v * 8);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) sq += q.v[e] * q.v[e];
+      for (int g = 0; g < gpv; ++g) {
+        float s = 0.f;
+        for (int r = 0; r < D; ++r) s += q.v[g * D + r];
+        zrow[v * gpv + g] = s * invD;
+      }
+    }
+  } else {                          // any other group size: scalar
+    for (int j = lane; j < m; j += 32) {
+      float s = 0.f;
+      for (int r = 0; r < D; ++r) { float v = to_f32<T>(x[(size_t)j * D + r]); s += v; sq += v * v; }
+      zrow[j] = s * invD;
+    }
+  }
+  sumsq = warp_sum(sq);
+}
+
+template <class T>
+__global__ void __launch_bounds__(AFF_THREADS)
+affinity_fwd_kernel(const T* __restrict__ X, const float* __restrict__ R, float* __restrict__ delta,
+                    float* __restrict__ Z, float* __restrict__ xnorm, float* __restrict__ rnorm,
+                    etr_stats* stats, int Ttok, int d, int D, int E, int m, int ldm, int Epad) {
+  extern __shared__ __align__(16) float smem[];
+  float* Rs = smem;                          // [Epad][ldm]
+  float* Zs = Rs + (size_t)Epad * ldm;       // [TB][ldm]
+  float* xn = Zs + (size_t)AFF_TB * ldm;     // [TB]
+  float* rn = xn + AFF_TB;                   // [Epad]
+  __shared__ uint32_t red[AFF_THREADS / 32];
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int t0 = blockIdx.x * AFF_TB;
+
+  // phase 0
+  for (int idx = tid; idx < Epad * ldm; idx += AFF_THREADS) {
+    const int i = idx / ldm, j = idx - i * ldm;
+    Rs[idx] = (i < E && j < m) ? R[(size_t)i * m + j] : 0.f;
+  }
+  for (int idx = tid; idx < AFF_TB * ldm; idx += AFF_THREADS) Zs[idx] = 0.f;
+  __syncthreads();
+  for (int i = warp; i < Epad; i += AFF_THREADS / 32) {
+    float s = 0.f;
+    for (int j = lane; j < m; j += 32) s += Rs[i * ldm + j] * Rs[i * ldm + j];
+    s = warp_sum(s);
+    if (lane == 0) {
+      rn[i] = sqrtf(s);
+      if (blockIdx.x == 0 && i < E) rnorm[i] = rn[i];
+    }
+  }
+
+  // phase 1
+  for (int tt = warp; tt < AFF_TB; tt += AFF_THREADS / 32) {
+    const int t = t0 + tt;
+    if (t < Ttok) {
+      float sq;
+      pool_token<T>(X + (size_t)t * d, Zs + (size_t)tt * ldm, d, D, m, lane, sq);
+      if (lane == 0) { xn[tt] = sqrtf(sq); xnorm[t] = xn[tt]; }
+    } else if (lane == 0) {
+      xn[tt] = 0.f;
+    }
+  }
+  __syncthreads();
+  if (Z != nullptr) {
+    for (int idx = tid; idx < AFF_TB * m; idx += AFF_THREADS) {
+      const int tt = idx / m, j = idx - tt * m;
+      if (t0 + tt < Ttok) Z[(size_t)(t0 + tt) * m + j] = Zs[tt * ldm + j];
+    }
+  }
+
+  // phase 2
+  const int nq = Epad / 4;
+  const float sqD = sqrtf((float)D);
+  const int mr4 = (m + 3) / 4;
+  float best = -INFINITY;
+  for (int item = tid; item < nq * (AFF_TB / 2); item += AFF_THREADS) {
+    const int q = item % nq, tp = item / nq;
+    const float4* z0 = reinterpret_cast<const float4*>(Zs + (size_t)(2 * tp) * ldm);
+    const float4* z1 = reinterpret_cast<const float4*>(Zs + (size_t)(2 * tp + 1) * ldm);
+    const float4* r0 = reinterpret_cast<const float4*>(Rs + (size_t)(4 * q) * ldm);
+    const int rs = ldm / 4;
+    float acc[2][4] = {};
+#pragma unroll 2
+    for (int j = 0; j < mr4; ++j) {
+      const float4 a = z0[j], b = z1[j];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const float4 r = r0[e * rs + j];
+        acc[0][e] = fmaf(a.x, r.x, acc[0][e]); acc[0][e] = fmaf(a.y, r.y, acc[0][e]);
+        acc[0][e] = fmaf(a.z, r.z, acc[0][e]); acc[0][e] = fmaf(a.w, r.w, acc[0][e]);
+        acc[1][e] = fmaf(b.x, r.x, acc[1][e]); acc[1][e] = fmaf(b.y, r.y, acc[1][e]);
+        acc[1][e] = fmaf(b.z, r.z, acc[1][e]); acc[1][e] = fmaf(b.w, r.w, acc[1][e]);
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+      const int tt = 2 * tp + u, t = t0 + tt;
+      if (t >= Ttok) continue;
+      float out[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const float den = xn[tt] * rn[4 * q + e];
+        out[e] = den == 0.f ? 0.f : sqD * acc[u][e] / den;
+        if (4 * q + e < E) best = fmaxf(best, out[e]);
+      }
+      float* dst = delta + (size_t)t * E + 4 * q;
+      if ((E & 3) == 0) {
+        *reinterpret_cast<float4*>(dst) = make_float4(out[0], out[1], out[2], out[3]);
+      } else {
+        for (int e = 0; e < 4; ++e) if (4 * q + e < E) dst[e] = out[e];
+      }
+    }
+  }
+  uint32_t key = best == -INFINITY ? 0u : ordered_key(best);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) key = max(key, __shfl_xor_sync(0xffffffffu, key, o));
+  if (lane == 0) red[warp] = key;
+  __syncthreads();
+  if (tid == 0) {
+    for (int w = 1; w < AFF_THREADS / 32; ++w) key = max(key, red[w]);
+    if (key) atomicMax(&stats->delta_max_key, key);
+  }
+}
+
+// ---- backward -----------------------------------------------------------------------------
+// dX[t,:] += cz[q/D] - beta x[t,:]  with  cz = sum_r (dgate_r sqrt(D)/(a b_i D)) R_i,
+// beta = sum_r dgate_r delta_ti / a^2 over the rows r of token t.  One warp per token.
+template <class T>
+__global__ void __launch_bounds__(256)
+affinity_bwd_dx_kernel(const T* __restrict__ X, const float* __restrict__ R,
+                       const float* __restrict__ delta, const float* __restrict__ xnorm,
+                       const float* __restrict__ rnorm, const int32_t* __restrict__ tok_ptr,
+                       const int32_t* __restrict__ tok_row, const float* __restrict__ dgate,
+                       T* __restrict__ dX, int Ttok, int d, int D, int E, int m, int C_stride) {
+  extern __shared__ __align__(16) float smem[];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  float* cz = smem + (size_t)warp * m;
+  const int t = blockIdx.x * 8 + warp;
+  if (t >= Ttok) return;
+  const int beg = tok_ptr[t], end = tok_ptr[t + 1];
+  const float a = xnorm[t];
+  if (beg == end || a == 0.f) return;
+  for (int j = lane; j < m; j += 32) cz[j] = 0.f;
+  float beta = 0.f;
+  const float sqD = sqrtf((float)D);
+  for (int q = beg; q < end; ++q) {
+    const int r = tok_row[q], i = r / C_stride;
+    const float b = rnorm[i], dg = dgate[r];
+    if (b == 0.f) continue;
+    const float w = dg * sqD / (a * b) / (float)D;
+    beta += dg * delta[(size_t)t * E + i];
+    for (int j = lane; j < m; j += 32) cz[j] = fmaf(w, R[(size_t)i * m + j], cz[j]);
+  }
+  beta /= (a * a);
+  __syncwarp();
+  const T* x = X + (size_t)t * d;
+  T* g = dX + (size_t)t * d;
+  for (int v = lane; v < d / 8; v += 32) {
+    Vec8<T> xv = Vec8<T>::load(x + v * 8), gv = Vec8<T>::load(g + v * 8);
+    float out[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) out[e] = gv.v[e] + (cz[(v * 8 + e) / D] - beta * xv.v[e]);
+    Vec8<T>::store(g + v * 8, out);
+  }
+}
+
+// Partial dR over chunks of 128 slots of one expert (fixed order inside a chunk):
+//   part[i][ch][j] = sum_p w_p Z[t_p][j], w_p = dgate_p sqrt(D)/(a_t b_i);
+//   part[i][ch][m] = sum_p dgate_p delta_ti
+constexpr int DR_CHUNK = 128;
+constexpr int DR_MAXJ = 16;     // m <= 256 * DR_MAXJ
+__global__ void __launch_bounds__(256)
+affinity_bwd_dr_partial_kernel(const float* __restrict__ Z, const float* __restrict__ delta,
+                               const float* __restrict__ xnorm, const float* __restrict__ rnorm,
+                               const int32_t* __restrict__ counts,
+                               const int32_t* __restrict__ slot_token,
+                               const float* __restrict__ dgate, float* __restrict__ part,
+                               int E, int m, int C_stride, int nch, float sqD) {
+  __shared__ int s_t[DR_CHUNK];
+  __shared__ float s_w[DR_CHUNK], s_dd[DR_CHUNK];
+  const int i = blockIdx.x, ch = blockIdx.y, tid = threadIdx.x;
+  const int n = counts[i];
+  const int p0 = ch * DR_CHUNK;
+  float* out = part + ((size_t)i * nch + ch) * (m + 1);
+  const int np = min(DR_CHUNK, n - p0);
+  if (np <= 0) {
+    for (int j = tid; j <= m; j += 256) out[j] = 0.f;
+    return;
+  }
+  const float b = rnorm[i];
+  if (tid < np) {
+    const size_t r = (size_t)i * C_stride + p0 + tid;
+    const int t = slot_token[r];
+    const float a = xnorm[t], dg = dgate[r];
+    const bool dead = (a == 0.f || b == 0.f);
+    s_t[tid] = t;
+    s_w[tid] = dead ? 0.f : dg * sqD / (a * b);
+    s_dd[tid] = dead ? 0.f : dg * delta[(size_t)t * E + i];
+  }
+  __syncthreads();
+  float acc[DR_MAXJ];
+#pragma unroll
+  for (int u = 0; u < DR_MAXJ; ++u) acc[u] = 0.f;
+  float sdd = 0.f;
+  for (int p = 0; p < np; ++p) {
+    const int t = s_t[p];
+    const float w = s_w[p];
+    sdd += s_dd[p];
+#pragma unroll
+    for (int u = 0; u < DR_MAXJ; ++u) {
+      const int j = tid + u * 256;
+      if (j < m) acc[u] = fmaf(w, Z[(size_t)t * m + j], acc[u]);
+    }
+  }
+#pragma unroll
+  for (int u = 0; u < DR_MAXJ; ++u) {
+    const int j = tid + u * 256;
+    if (j < m) out[j] = acc[u];
+  }
+  if (tid == 0) out[m] = sdd;
+}
+
+// dR[i][j] = sum_ch part[i][ch][j] - (sum_ch part[i][ch][m]) R[i][j] / b_i^2, chunks in order.
+__global__ void __launch_bounds__(256)
+affinity_bwd_dr_final_kernel(const float* __restrict__ part, const float* __restrict__ R,
+                             const float* __restrict__ rnorm, float* __restrict__ dR, int m, int nch) {
+  const int i = blockIdx.x;
+  const float b = rnorm[i];
+  const float* base = part + (size_t)i * nch * (m + 1);
+  float sdd = 0.f;
+  for (int ch = 0; ch < nch; ++ch) sdd += base[(size_t)ch * (m + 1) + m];
+  for (int j = threadIdx.x; j < m; j += 256) {
+    float acc = 0.f;
+    for (int ch = 0; ch < nch; ++ch) acc += base[(size_t)ch * (m + 1) + j];
+    dR[(size_t)i * m + j] = b == 0.f ? 0.f : acc - sdd * R[(size_t)i * m + j] / (b * b);
+  }
+}
+
+// ---- host side ---------------------------------------------------------------------------------
+static size_t affinity_smem_bytes(int E, int m, int* ldm_out, int* Epad_out) {
+  const int ldm = (m + 3) / 4 * 4 + 4, Epad = (E + 3) / 4 * 4;
+  *ldm_out = ldm; *Epad_out = Epad;
+  return ((size_t)(Epad + AFF_TB) * ldm + AFF_TB + Epad) * sizeof(float);
+}
+
+etr_status affinity_forward(const etr_config* c, const void* X, const float* R, float* delta,
+                            float* Z, float* xnorm, float* rnorm, etr_stats* stats,
+                            cudaStream_t st) {
+  const int m = c->d / c->D;
+  int ldm, Epad;
+  const size_t smem = affinity_smem_bytes(c->E, m, &ldm, &Epad);
+  if (smem > 200 * 1024) return ETR_ERR_UNSUPPORTED;
+  const int grid = ceil_div(c->T, AFF_TB);
+  if (c->dtype == ETR_BF16) {
+    auto k = affinity_fwd_kernel<__nv_bfloat16>;
+    if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+      return ETR_ERR_CUDA;
+    k<<<grid, AFF_THREADS, smem, st>>>((const __nv_bfloat16*)X, R, delta, Z, xnorm, rnorm, stats,
+                                       c->T, c->d, c->D, c->E, m, ldm, Epad);
+  } else {
+    auto k = affinity_fwd_kernel<float>;
+    if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+      return ETR_ERR_CUDA;
+    k<<<grid, AFF_THREADS, smem, st>>>((const float*)X, R, delta, Z, xnorm, rnorm, stats, c->T,
+                                       c->d, c->D, c->E, m, ldm, Epad);
+  }
+  ETR_LAUNCH_CHECK();
+  return ETR_OK;
+}
+
+size_t affinity_bwd_workspace_bytes(const etr_config* c) {
+  const int m = c->d / c->D, nch = c_stride_of(c) / DR_CHUNK;
+  return (size_t)c->E * nch * (m + 1) * sizeof(float);
+}
+
+etr_status affinity_backward(const etr_config* c, const void* X, const float* R, const float* delta,
+                             const float* Z, const float* xnorm, const float* rnorm,
+                             const etr_route* rt, const float* dgate, void* dX, float* dR,
+                             void* ws, cudaStream_t st) {
+  const int m = c->d / c->D, Cs = c_stride_of(c), nch = Cs / DR_CHUNK;
+  if (m > 256 * DR_MAXJ) return ETR_ERR_UNSUPPORTED;
+  const size_t smem = (size_t)8 * m * sizeof(float);
+  if (smem > 200 * 1024) return ETR_ERR_UNSUPPORTED;
+  const int grid = ceil_div(c->T, 8);
+  if (c->dtype == ETR_BF16) {
+    auto k = affinity_bwd_dx_kernel<__nv_bfloat16>;
+    if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+      return ETR_ERR_CUDA;
+    k<<<grid, 256, smem, st>>>((const __nv_bfloat16*)X, R, delta, xnorm, rnorm, rt->tok_ptr,
+                               rt->tok_row, dgate, (__nv_bfloat16*)dX, c->T, c->d, c->D, c->E, m, Cs);
+  } else {
+    auto k = affinity_bwd_dx_kernel<float>;
+    if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+      return ETR_ERR_CUDA;
+    k<<<grid, 256, smem, st>>>((const float*)X, R, delta, xnorm, rnorm, rt->tok_ptr, rt->tok_row,
+                               dgate, (float*)dX, c->T, c->d, c->D, c->E, m, Cs);
+  }
+  ETR_LAUNCH_CHECK();
+  float* part = (float*)ws;
+  affinity_bwd_dr_partial_kernel<<<dim3(c->E, nch), 256, 0, st>>>(
+      Z, delta, xnorm, rnorm, rt->counts, rt->slot_token, dgate, part, c->E, m, Cs, nch,
+      sqrtf((float)c->D));
+  ETR_LAUNCH_CHECK();
+  affinity_bwd_dr_final_kernel<<<c->E, 256, 0, st>>>(part, R, rnorm, dR, m, nch);
+  ETR_LAUNCH_CHECK();
+  return ETR_OK;
+}
+
+}  // namespace etr

@@ -1,0 +1,307 @@
+// C ABI of libetr: argument checks, buffer carving, stage wrappers, whole-layer calls.
+#include <atomic>
+#include <cstring>
+
+#include "common.cuh"
+
+namespace etr {
+
+static std::atomic<long long> g_launches{0};
+void note_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+static bool use_tc(const etr_config* c) {
+  if (c->gemm_impl == ETR_GEMM_SIMT) return false;
+  if (c->gemm_impl == ETR_GEMM_TCGEN05) return true;
+  return c->dtype == ETR_BF16;
+}
+
+static etr_status check_ptrs(std::initializer_list<const void*> ps) {
+  for (const void* p : ps) {
+    if (p == nullptr) return ETR_ERR_ARG;
+    if (!aligned16(p)) return ETR_ERR_ALIGN;
+  }
+  return ETR_OK;
+}
+
+static etr_status check_route(const etr_route* r) {
+  if (r == nullptr) return ETR_ERR_ARG;
+  return check_ptrs({r->topk_idx, r->counts, r->slot_token, r->gate, r->tok_ptr, r->tok_row});
+}
+
+struct Carver {
+  char* base; size_t off;
+  void* take(size_t bytes) {
+    off = align_up(off, 256);
+    void* p = base ? base + off : nullptr;
+    off += bytes;
+    return p;
+  }
+};
+
+static void carve(const etr_config* c, int staging, char* base, etr_buffers* b, size_t* total) {
+  const size_t T = c->T, E = c->E, d = c->d, h = c->h, m = c->d / c->D, k = c->k;
+  const size_t rows = E * (size_t)c_stride_of(c), eb = elem_bytes(c->dtype);
+  size_t ws = 0;
+  etr_workspace_bytes(c, &ws);
+  Carver cv{base, 0};
+  etr_buffers t;
+  memset(&t, 0, sizeof(t));
+  t.stats = (etr_stats*)cv.take(sizeof(etr_stats));
+  t.route.topk_idx = (int32_t*)cv.take(T * k * 4);
+  t.route.counts = (int32_t*)cv.take(E * 4);
+  t.route.slot_token = (int32_t*)cv.take(rows * 4);
+  t.route.gate = (float*)cv.take(rows * 4);
+  t.route.tok_ptr = (int32_t*)cv.take((T + 1) * 4);
+  t.route.tok_row = (int32_t*)cv.take(rows * 4);
+  t.delta = (float*)cv.take(T * E * 4);
+  t.Z = (float*)cv.take(T * m * 4);
+  t.xnorm = (float*)cv.take(T * 4);
+  t.rnorm = (float*)cv.take(E * 4);
+  t.Xp = cv.take(rows * d * eb);
+  t.G = cv.take(rows * h * eb);
+  t.U = cv.take(rows * h * eb);
+  t.H = cv.take(rows * h * eb);
+  t.O = cv.take(rows * d * eb);
+  t.dO = cv.take(rows * d * eb);
+  t.dG = cv.take(rows * h * eb);
+  t.dU = cv.take(rows * h * eb);
+  t.dXp = cv.take(rows * d * eb);
+  t.dgate = (float*)cv.take(rows * 4);
+  t.ws = cv.take(ws);
+  t.ws_bytes = ws;
+  if (staging) {
+    t.X_dev = cv.take(T * d * eb);
+    t.dY_dev = cv.take(T * d * eb);
+    t.Y_dev = cv.take(T * d * eb);
+    t.dX_dev = cv.take(T * d * eb);
+  }
+  if (b) *b = t;
+  *total = align_up(cv.off, 256);
+}
+
+}  // namespace etr
+
+using namespace etr;
+
+extern "C" {
+
+const char* etr_status_string(etr_status s) {
+  switch (s) {
+    case ETR_OK: return "ok";
+    case ETR_ERR_ARG: return "bad argument (NULL pointer, non-positive size or bad enum)";
+    case ETR_ERR_SHAPE: return "sizes violate the shape rules";
+    case ETR_ERR_ALIGN: return "pointer not 16-byte aligned";
+    case ETR_ERR_WORKSPACE: return "buffer too small";
+    case ETR_ERR_CUDA: return "CUDA call failed";
+    case ETR_ERR_TIMEOUT: return "a bounded device-side wait expired";
+    case ETR_ERR_UNSUPPORTED: return "unsupported configuration";
+  }
+  return "unknown status";
+}
+
+etr_status etr_validate(const etr_config* c) {
+  if (c == nullptr) return ETR_ERR_ARG;
+  if (c->T < 1 || c->d < 1 || c->D < 1 || c->E < 1 || c->k < 1 || c->h < 1 || c->capacity < 1)
+    return ETR_ERR_ARG;
+  if (c->dtype != ETR_F32 && c->dtype != ETR_BF16) return ETR_ERR_ARG;
+  if (c->mode < ETR_MODE_AUTO || c->mode > ETR_MODE_ECR) return ETR_ERR_ARG;
+  if (c->gemm_impl < ETR_GEMM_AUTO || c->gemm_impl > ETR_GEMM_TCGEN05) return ETR_ERR_ARG;
+  if (c->d % c->D != 0 || c->d % 8 != 0 || c->h % 8 != 0) return ETR_ERR_SHAPE;
+  if (c->k > c->E || c->E > 256 || c->E > c->d / c->D) return ETR_ERR_SHAPE;
+  if ((long long)c->T * c->E >= (1ll << 31)) return ETR_ERR_SHAPE;
+  if ((long long)c->E * c_stride_of(c) >= (1ll << 31)) return ETR_ERR_SHAPE;
+  if (use_tc(c)) {
+    if (c->dtype != ETR_BF16) return ETR_ERR_UNSUPPORTED;
+    if (c->d % 64 != 0 || c->h % 64 != 0) return ETR_ERR_UNSUPPORTED;
+  }
+  return ETR_OK;
+}
+
+int32_t etr_c_stride(const etr_config* c) { return c ? c_stride_of(c) : 0; }
+
+etr_status etr_workspace_bytes(const etr_config* c, size_t* bytes) {
+  if (bytes == nullptr) return ETR_ERR_ARG;
+  ETR_TRY(etr_validate(c));
+  size_t w = select_workspace_bytes(c);
+  w = w > affinity_bwd_workspace_bytes(c) ? w : affinity_bwd_workspace_bytes(c);
+  if (use_tc(c)) w = w > tc_workspace_bytes(c) ? w : tc_workspace_bytes(c);
+  *bytes = align_up(w, 256);
+  return ETR_OK;
+}
+
+etr_status etr_buffers_bytes(const etr_config* c, int with_host_staging, size_t* bytes) {
+  if (bytes == nullptr) return ETR_ERR_ARG;
+  ETR_TRY(etr_validate(c));
+  carve(c, with_host_staging, nullptr, nullptr, bytes);
+  return ETR_OK;
+}
+
+etr_status etr_buffers_bind(const etr_config* c, int with_host_staging, void* base, size_t bytes,
+                            etr_buffers* out) {
+  if (base == nullptr || out == nullptr) return ETR_ERR_ARG;
+  ETR_TRY(etr_validate(c));
+  if (reinterpret_cast<uintptr_t>(base) & 255u) return ETR_ERR_ALIGN;
+  size_t need = 0;
+  carve(c, with_host_staging, nullptr, nullptr, &need);
+  if (bytes < need) return ETR_ERR_WORKSPACE;
+  carve(c, with_host_staging, (char*)base, out, &need);
+  return ETR_OK;
+}
+
+etr_status etr_affinity(const etr_config* c, const void* X, const float* R, float* delta, float* Z,
+                        float* xnorm, float* rnorm, etr_stats* stats, void* stream) {
+  ETR_TRY(etr_validate(c));
+  ETR_TRY(check_ptrs({X, R, delta, xnorm, rnorm, stats}));
+  if (Z && !aligned16(Z)) return ETR_ERR_ALIGN;
+  return affinity_forward(c, X, R, delta, Z, xnorm, rnorm, stats, (cudaStream_t)stream);
+}
+
+etr_status etr_select(const etr_config* c, const float* delta, etr_stats* stats,
+                      const etr_route* route, void* ws, void* stream) {
+  ETR_TRY(etr_validate(c));
+  ETR_TRY(check_ptrs({delta, stats, ws}));
+  ETR_TRY(check_route(route));
+  return select_forward(c, delta, stats, route, ws, (cudaStream_t)stream);
+}
+
+etr_status etr_dispatch(const etr_config* c, const void* X, const etr_route* route, void* Xp,
+                        void* stream) {
+  ETR_TRY(etr_validate(c));
+  ETR_TRY(check_ptrs({X, Xp}));
+  ETR_TRY(check_route(route));
+  return dispatch_forward(c, X, route, Xp, (cudaStream_t)stream);
+}
+
+etr_status etr_expert_ffn(const etr_config* c, const etr_route* route, const void* Xp,
+                          const void* W1g, const void* W1u, const void* W2, void* G, void* U,
+                          void* H, void* O, etr_stats* stats, void* ws, void* stream) {
+  ETR_TRY(etr_validate(c));
+  ETR_TRY(check_ptrs({Xp, W1g, W1u, W2, G, U, H, O}));
+  ETR_TRY(check_route(route));
+  if (use_tc(c)) {
+    ETR_TRY(check_ptrs({stats, ws}));
+    return tc_ffn_forward(c, route, Xp, W1g, W1u, W2, G, U, H, O, stats, ws, (cudaStream_t)stream);
+  }
+  return simt_ffn_forward(c, route, Xp, W1g, W1u, W2, G, U, H, O, (cudaStream_t)stream);
+}
+
+etr_status etr_combine(const etr_config* c, const etr_route* route, const void* O, void* Y,
+                       void* stream) {
+  ETR_TRY(etr_validate(c));
+  ETR_TRY(check_ptrs({O, Y}));
+  ETR_TRY(check_route(route));
+  return combine_forward(c, route, O, Y, (cudaStream_t)stream);
+}
+
+etr_status etr_combine_bwd(const etr_config* c, const etr_route* route, const void* dY,
+                           const void* O, void* dO, float* dgate, void* stream) {
+  ETR_TRY(etr_validate(c));
+  ETR_TRY(check_ptrs({dY, O, dO, dgate}));
+  ETR_TRY(check_route(route));
+  return combine_backward(c, route, dY, O, dO, dgate, (cudaStream_t)stream);
+}
+
+etr_status etr_expert_ffn_bwd(const etr_config* c, const etr_route* route, const void* dO,
+                              const void* Xp, const void* G, const void* U, const void* H,
+                              const void* W1g, const void* W1u, const void* W2, void* dG, void* dU,
+                              void* dXp, void* dW1g, void* dW1u, void* dW2, etr_stats* stats,
+                              void* ws, void* stream) {
+  ETR_TRY(etr_validate(c));
+  ETR_TRY(check_ptrs({dO, Xp, G, U, H, W1g, W1u, W2, dG, dU, dXp, dW1g, dW1u, dW2}));
+  ETR_TRY(check_route(route));
+  if (use_tc(c)) {
+    ETR_TRY(check_ptrs({stats, ws}));
+    return tc_ffn_backward(c, route, dO, Xp, G, U, H, W1g, W1u, W2, dG, dU, dXp, dW1g, dW1u, dW2,
+                           stats, ws, (cudaStream_t)stream);
+  }
+  return simt_ffn_backward(c, route, dO, Xp, G, U, H, W1g, W1u, W2, dG, dU, dXp, dW1g, dW1u, dW2,
+                           (cudaStream_t)stream);
+}
+
+etr_status etr_dispatch_bwd(const etr_config* c, const etr_route* route, const void* dXp, void* dX,
+                            void* stream) {
+  ETR_TRY(etr_validate(c));
+  ETR_TRY(check_ptrs({dXp, dX}));
+  ETR_TRY(check_route(route));
+  return dispatch_backward(c, route, dXp, dX, (cudaStream_t)stream);
+}
+
+etr_status etr_select_bwd(const etr_config* c, const etr_route* route, const float* dgate) {
+  ETR_TRY(etr_validate(c));
+  ETR_TRY(check_ptrs({dgate}));
+  return check_route(route);
+}
+
+etr_status etr_affinity_bwd(const etr_config* c, const void* X, const float* R, const float* delta,
+                            const float* Z, const float* xnorm, const float* rnorm,
+                            const etr_route* route, const float* dgate, void* dX, float* dR,
+                            void* ws, void* stream) {
+  ETR_TRY(etr_validate(c));
+  ETR_TRY(check_ptrs({X, R, delta, Z, xnorm, rnorm, dgate, dX, dR, ws}));
+  ETR_TRY(check_route(route));
+  return affinity_backward(c, X, R, delta, Z, xnorm, rnorm, route, dgate, dX, dR, ws,
+                           (cudaStream_t)stream);
+}
+
+etr_status etr_layer_forward(const etr_config* c, const void* X, const float* R, const void* W1g,
+                             const void* W1u, const void* W2, const etr_buffers* b, void* Y,
+                             void* stream) {
+  if (b == nullptr) return ETR_ERR_ARG;
+  ETR_TRY(etr_validate(c));
+  ETR_TRY(check_ptrs({b->stats}));
+  if (cudaMemsetAsync(b->stats, 0, sizeof(etr_stats), (cudaStream_t)stream) != cudaSuccess)
+    return ETR_ERR_CUDA;
+  ETR_TRY(etr_affinity(c, X, R, b->delta, b->Z, b->xnorm, b->rnorm, b->stats, stream));
+  ETR_TRY(etr_select(c, b->delta, b->stats, &b->route, b->ws, stream));
+  ETR_TRY(etr_dispatch(c, X, &b->route, b->Xp, stream));
+  ETR_TRY(etr_expert_ffn(c, &b->route, b->Xp, W1g, W1u, W2, b->G, b->U, b->H, b->O, b->stats, b->ws,
+                         stream));
+  return etr_combine(c, &b->route, b->O, Y, stream);
+}
+
+etr_status etr_layer_backward(const etr_config* c, const void* X, const float* R, const void* W1g,
+                              const void* W1u, const void* W2, const void* dY, const etr_buffers* b,
+                              void* dX, float* dR, void* dW1g, void* dW1u, void* dW2, void* stream) {
+  if (b == nullptr) return ETR_ERR_ARG;
+  ETR_TRY(etr_combine_bwd(c, &b->route, dY, b->O, b->dO, b->dgate, stream));
+  ETR_TRY(etr_expert_ffn_bwd(c, &b->route, b->dO, b->Xp, b->G, b->U, b->H, W1g, W1u, W2, b->dG, b->dU,
+                             b->dXp, dW1g, dW1u, dW2, b->stats, b->ws, stream));
+  ETR_TRY(etr_dispatch_bwd(c, &b->route, b->dXp, dX, stream));
+  ETR_TRY(etr_select_bwd(c, &b->route, b->dgate));
+  return etr_affinity_bwd(c, X, R, b->delta, b->Z, b->xnorm, b->rnorm, &b->route, b->dgate, dX, dR,
+                          b->ws, stream);
+}
+
+etr_status etr_layer_step_host(const etr_config* c, const void* X_host, const void* dY_host,
+                               const float* R, const void* W1g, const void* W1u, const void* W2,
+                               const etr_buffers* b, void* Y_host, void* dX_host, float* dR,
+                               void* dW1g, void* dW1u, void* dW2, void* stream) {
+  if (b == nullptr || X_host == nullptr || dY_host == nullptr || Y_host == nullptr || dX_host == nullptr)
+    return ETR_ERR_ARG;
+  ETR_TRY(etr_validate(c));
+  if (!b->X_dev || !b->dY_dev || !b->Y_dev || !b->dX_dev) return ETR_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)stream;
+  const size_t bytes = (size_t)c->T * c->d * elem_bytes(c->dtype);
+  if (cudaMemcpyAsync(b->X_dev, X_host, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return ETR_ERR_CUDA;
+  if (cudaMemcpyAsync(b->dY_dev, dY_host, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return ETR_ERR_CUDA;
+  ETR_TRY(etr_layer_forward(c, b->X_dev, R, W1g, W1u, W2, b, b->Y_dev, stream));
+  if (cudaMemcpyAsync(Y_host, b->Y_dev, bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return ETR_ERR_CUDA;
+  ETR_TRY(etr_layer_backward(c, b->X_dev, R, W1g, W1u, W2, b->dY_dev, b, b->dX_dev, dR, dW1g, dW1u,
+                             dW2, stream));
+  if (cudaMemcpyAsync(dX_host, b->dX_dev, bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return ETR_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return ETR_ERR_CUDA;
+  return ETR_OK;
+}
+
+etr_status etr_read_stats(const etr_stats* dev, etr_stats* host, void* stream) {
+  if (dev == nullptr || host == nullptr) return ETR_ERR_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (cudaMemcpyAsync(host, dev, sizeof(etr_stats), cudaMemcpyDeviceToHost, st) != cudaSuccess)
+    return ETR_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return ETR_ERR_CUDA;
+  return host->error_word ? ETR_ERR_TIMEOUT : ETR_OK;
+}
+
+int64_t etr_launch_count(void) { return (int64_t)g_launches.load(); }
+
+}  // extern "C"

@@ -1,0 +1,141 @@
+// Shared device/host helpers of libetr (sm_100a only).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/etr.h"
+
+namespace etr {
+
+// ---- launch accounting and error mapping ------------------------------------------------
+void note_launch(int n = 1);
+#define ETR_LAUNCH_CHECK()                                  \
+  do {                                                      \
+    ::etr::note_launch();                                   \
+    cudaError_t e__ = cudaGetLastError();                   \
+    if (e__ != cudaSuccess) return ETR_ERR_CUDA;            \
+  } while (0)
+#define ETR_TRY(expr)                                       \
+  do {                                                      \
+    etr_status s__ = (expr);                                \
+    if (s__ != ETR_OK) return s__;                          \
+  } while (0)
+
+inline int c_stride_of(const etr_config* c) { return (c->capacity + 127) / 128 * 128; }
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline size_t elem_bytes(int dtype) { return dtype == ETR_BF16 ? 2 : 4; }
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
+
+// ---- order-preserving map float -> uint32 (larger float <=> larger key; key 0 is below
+//      every finite float and is used as "not a candidate") --------------------------------
+__host__ __device__ inline uint32_t ordered_key(float f) {
+  uint32_t u;
+#ifdef __CUDA_ARCH__
+  u = __float_as_uint(f);
+#else
+  union { float f; uint32_t u; } c; c.f = f; u = c.u;
+#endif
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__host__ __device__ inline float key_to_float(uint32_t k) {
+  uint32_t u = (k & 0x80000000u) ? (k & 0x7fffffffu) : ~k;
+#ifdef __CUDA_ARCH__
+  return __uint_as_float(u);
+#else
+  union { float f; uint32_t u; } c; c.u = u; return c.f;
+#endif
+}
+
+// ---- 8-element vectors of the activation dtype -----------------------------------------------
+template <class T> struct Vec8;
+template <> struct Vec8<float> {
+  float v[8];
+  __device__ static Vec8 load(const float* p) {
+    Vec8 r;
+    float4 a = *reinterpret_cast<const float4*>(p), b = *reinterpret_cast<const float4*>(p + 4);
+    r.v[0] = a.x; r.v[1] = a.y; r.v[2] = a.z; r.v[3] = a.w;
+    r.v[4] = b.x; r.v[5] = b.y; r.v[6] = b.z; r.v[7] = b.w;
+    return r;
+  }
+  __device__ static void store(float* p, const float* f) {
+    *reinterpret_cast<float4*>(p) = make_float4(f[0], f[1], f[2], f[3]);
+    *reinterpret_cast<float4*>(p + 4) = make_float4(f[4], f[5], f[6], f[7]);
+  }
+};
+template <> struct Vec8<__nv_bfloat16> {
+  float v[8];
+  __device__ static Vec8 load(const __nv_bfloat16* p) {
+    Vec8 r;
+    uint4 q = *reinterpret_cast<const uint4*>(p);
+    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      r.v[2 * i] = __uint_as_float(w[i] << 16);
+      r.v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+    }
+    return r;
+  }
+  __device__ static void store(__nv_bfloat16* p, const float* f) {
+    uint32_t w[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      __nv_bfloat162 b = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
+      w[i] = *reinterpret_cast<uint32_t*>(&b);
+    }
+    *reinterpret_cast<uint4*>(p) = make_uint4(w[0], w[1], w[2], w[3]);
+  }
+};
+
+template <class T> __device__ inline float to_f32(T v);
+template <> __device__ inline float to_f32<float>(float v) { return v; }
+template <> __device__ inline float to_f32<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+template <class T> __device__ inline T from_f32(float v);
+template <> __device__ inline float from_f32<float>(float v) { return v; }
+template <> __device__ inline __nv_bfloat16 from_f32<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+
+__device__ inline float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// ---- stage entry points, one translation unit each ------------------------------------------
+etr_status affinity_forward(const etr_config* c, const void* X, const float* R, float* delta,
+                            float* Z, float* xnorm, float* rnorm, etr_stats* stats, cudaStream_t st);
+size_t affinity_bwd_workspace_bytes(const etr_config* c);
+etr_status affinity_backward(const etr_config* c, const void* X, const float* R, const float* delta,
+                             const float* Z, const float* xnorm, const float* rnorm,
+                             const etr_route* rt, const float* dgate, void* dX, float* dR, void* ws,
+                             cudaStream_t st);
+size_t select_workspace_bytes(const etr_config* c);
+int resolve_mode(const etr_config* c);
+etr_status select_forward(const etr_config* c, const float* delta, etr_stats* stats,
+                          const etr_route* rt, void* ws, cudaStream_t st);
+etr_status dispatch_forward(const etr_config* c, const void* X, const etr_route* rt, void* Xp, cudaStream_t st);
+etr_status combine_forward(const etr_config* c, const etr_route* rt, const void* O, void* Y, cudaStream_t st);
+etr_status combine_backward(const etr_config* c, const etr_route* rt, const void* dY, const void* O,
+                            void* dO, float* dgate, cudaStream_t st);
+etr_status dispatch_backward(const etr_config* c, const etr_route* rt, const void* dXp, void* dX, cudaStream_t st);
+
+// SIMT grouped GEMMs (fp32 or bf16 storage, fp32 accumulate).
+etr_status simt_ffn_forward(const etr_config* cfg, const etr_route* route, const void* Xp,
+                            const void* W1g, const void* W1u, const void* W2, void* G, void* U,
+                            void* H, void* O, cudaStream_t st);
+etr_status simt_ffn_backward(const etr_config* cfg, const etr_route* route, const void* dO,
+                             const void* Xp, const void* G, const void* U, const void* H,
+                             const void* W1g, const void* W1u, const void* W2, void* dG, void* dU,
+                             void* dXp, void* dW1g, void* dW1u, void* dW2, cudaStream_t st);
+// tcgen05 grouped GEMMs (bf16 only).
+etr_status tc_ffn_forward(const etr_config* cfg, const etr_route* route, const void* Xp,
+                          const void* W1g, const void* W1u, const void* W2, void* G, void* U,
+                          void* H, void* O, etr_stats* stats, void* ws, cudaStream_t st);
+etr_status tc_ffn_backward(const etr_config* cfg, const etr_route* route, const void* dO,
+                           const void* Xp, const void* G, const void* U, const void* H,
+                           const void* W1g, const void* W1u, const void* W2, void* dG, void* dU,
+                           void* dXp, void* dW1g, void* dW1u, void* dW2, etr_stats* stats,
+                           void* ws, cudaStream_t st);
+size_t tc_workspace_bytes(const etr_config* cfg);
+
+}  // namespace etr

@@ -1,0 +1,135 @@
+// Token rearrangement and gate-weighted combine, forward and backward.  All four kernels
+// are pure streaming: 16-byte vectors, one pass over every byte they must touch.
+#include "common.cuh"
+
+namespace etr {
+
+// Xp[r,:] = X[slot_token[r],:] for rows in use; pad rows (up to the next multiple of 128
+// after counts[i]) are zero-filled; rows beyond are left alone.  One warp per row.
+template <class T>
+__global__ void __launch_bounds__(256)
+dispatch_kernel(const T* __restrict__ X, const int32_t* __restrict__ counts,
+                const int32_t* __restrict__ slot_token, T* __restrict__ Xp, int d, int C_stride,
+                int n_rows) {
+  const int r = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (r >= n_rows) return;
+  const int i = r / C_stride, p = r - i * C_stride;
+  const int lim = (counts[i] + 127) & ~127;
+  if (p >= lim) return;
+  const int t = slot_token[r];
+  uint4* dst = reinterpret_cast<uint4*>(Xp + (size_t)r * d);
+  const int nv = d * (int)sizeof(T) / 16;
+  if (t >= 0) {
+    const uint4* src = reinterpret_cast<const uint4*>(X + (size_t)t * d);
+#pragma unroll 4
+    for (int v = lane; v < nv; v += 32) dst[v] = __ldg(src + v);
+  } else {
+    for (int v = lane; v < nv; v += 32) dst[v] = make_uint4(0, 0, 0, 0);
+  }
+}
+
+// Y[t,:] = sum_{r in rows(t)} gate[r] O[r,:]   (gate == nullptr: plain sum, used for dX).
+// One thread per 8 consecutive elements of a token.
+template <class T>
+__global__ void __launch_bounds__(256)
+combine_kernel(const T* __restrict__ O, const float* __restrict__ gate,
+               const int32_t* __restrict__ tok_ptr, const int32_t* __restrict__ tok_row,
+               T* __restrict__ Y, int Ttok, int d) {
+  const int vpt = d / 8;
+  const long long idx = (long long)blockIdx.x * 256 + threadIdx.x;
+  if (idx >= (long long)Ttok * vpt) return;
+  const int t = (int)(idx / vpt), v = (int)(idx - (long long)t * vpt);
+  float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+  const int beg = tok_ptr[t], end = tok_ptr[t + 1];
+  for (int q = beg; q < end; ++q) {
+    const int r = tok_row[q];
+    const float g = gate ? gate[r] : 1.0f;
+    Vec8<T> o = Vec8<T>::load(O + (size_t)r * d + v * 8);
+#pragma unroll
+    for (int e = 0; e < 8; ++e) acc[e] = fmaf(g, o.v[e], acc[e]);
+  }
+  Vec8<T>::store(Y + (size_t)t * d + v * 8, acc);
+}
+
+// dO[r,:] = gate[r] dY[t(r),:], dgate[r] = <dY[t(r),:], O[r,:]>; pad rows zero.  Warp per row.
+template <class T>
+__global__ void __launch_bounds__(256)
+combine_bwd_kernel(const T* __restrict__ dY, const T* __restrict__ O,
+                   const int32_t* __restrict__ counts, const int32_t* __restrict__ slot_token,
+                   const float* __restrict__ gate, T* __restrict__ dO, float* __restrict__ dgate,
+                   int d, int C_stride, int n_rows) {
+  const int r = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (r >= n_rows) return;
+  const int i = r / C_stride, p = r - i * C_stride;
+  const int lim = (counts[i] + 127) & ~127;
+  if (p >= lim) return;
+  const int t = slot_token[r];
+  T* dst = dO + (size_t)r * d;
+  if (t < 0) {
+    const int nv = d * (int)sizeof(T) / 16;
+    for (int v = lane; v < nv; v += 32) reinterpret_cast<uint4*>(dst)[v] = make_uint4(0, 0, 0, 0);
+    if (lane == 0) dgate[r] = 0.f;
+    return;
+  }
+  const float g = gate[r];
+  const T* gy = dY + (size_t)t * d;
+  const T* o = O + (size_t)r * d;
+  float dot = 0.f;
+#pragma unroll 2
+  for (int v = lane; v < d / 8; v += 32) {
+    Vec8<T> a = Vec8<T>::load(gy + v * 8), b = Vec8<T>::load(o + v * 8);
+    float out[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) { out[e] = g * a.v[e]; dot = fmaf(a.v[e], b.v[e], dot); }
+    Vec8<T>::store(dst + v * 8, out);
+  }
+  dot = warp_sum(dot);
+  if (lane == 0) dgate[r] = dot;
+}
+
+template <class T>
+static etr_status permute_launch(int which, const etr_config* c, const etr_route* rt, const void* a,
+                                 const void* b, void* out, float* dgate, cudaStream_t st) {
+  const int Cs = c_stride_of(c), n_rows = c->E * Cs;
+  switch (which) {
+    case 0:
+      dispatch_kernel<T><<<ceil_div(n_rows, 8), 256, 0, st>>>((const T*)a, rt->counts, rt->slot_token,
+                                                             (T*)out, c->d, Cs, n_rows);
+      break;
+    case 1:
+    case 3: {
+      const long long n = (long long)c->T * (c->d / 8);
+      combine_kernel<T><<<(unsigned)((n + 255) / 256), 256, 0, st>>>(
+          (const T*)a, which == 1 ? rt->gate : nullptr, rt->tok_ptr, rt->tok_row, (T*)out, c->T, c->d);
+      break;
+    }
+    case 2:
+      combine_bwd_kernel<T><<<ceil_div(n_rows, 8), 256, 0, st>>>(
+          (const T*)a, (const T*)b, rt->counts, rt->slot_token, rt->gate, (T*)out, dgate, c->d, Cs, n_rows);
+      break;
+  }
+  ETR_LAUNCH_CHECK();
+  return ETR_OK;
+}
+
+static etr_status permute_dispatch(int which, const etr_config* c, const etr_route* rt, const void* a,
+                                   const void* b, void* out, float* dgate, cudaStream_t st) {
+  return c->dtype == ETR_BF16 ? permute_launch<__nv_bfloat16>(which, c, rt, a, b, out, dgate, st)
+                              : permute_launch<float>(which, c, rt, a, b, out, dgate, st);
+}
+
+etr_status dispatch_forward(const etr_config* c, const void* X, const etr_route* rt, void* Xp, cudaStream_t st) {
+  return permute_dispatch(0, c, rt, X, nullptr, Xp, nullptr, st);
+}
+etr_status combine_forward(const etr_config* c, const etr_route* rt, const void* O, void* Y, cudaStream_t st) {
+  return permute_dispatch(1, c, rt, O, nullptr, Y, nullptr, st);
+}
+etr_status combine_backward(const etr_config* c, const etr_route* rt, const void* dY, const void* O,
+                            void* dO, float* dgate, cudaStream_t st) {
+  return permute_dispatch(2, c, rt, dY, O, dO, dgate, st);
+}
+etr_status dispatch_backward(const etr_config* c, const etr_route* rt, const void* dXp, void* dX, cudaStream_t st) {
+  return permute_dispatch(3, c, rt, dXp, nullptr, dX, nullptr, st);
+}
+
+}  // namespace etr

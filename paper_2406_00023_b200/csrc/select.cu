@@ -1,0 +1,285 @@
+// Bidirectional selection: token-side top-k, expert-side top-C, routing maps.
+//
+// All decisions are taken on order-preserving 32-bit integer images of the fp32
+// affinities, so there is no floating-point arithmetic here and the result is exact:
+//   1. token side (one warp per token): the k best experts by (key desc, index asc);
+//      writes topk_idx and the transposed key matrix keyT[E][T] (0 = not a candidate;
+//      in expert choice every pair is a candidate).  Block 0 also fixes mode and C.
+//   2. expert side (one CTA per expert): 4-pass 8-bit radix select over the expert's row
+//      of keyT finds the C-th largest key tau; tokens with key > tau are kept, and of the
+//      tokens with key == tau the lowest token ids fill the remaining quota; a ballot
+//      scan in token order assigns slots (ascending token id).  The row of keyT is
+//      overwritten with the slot position (or -1).
+//   3. token-major CSR from the position matrix: count, exclusive scan, fill.
+#include "common.cuh"
+
+namespace etr {
+
+constexpr int SEL_TB = 32;         // tokens per CTA on the token side
+constexpr int SEL_MAX_EPL = 8;     // experts per lane: E <= 256
+
+struct SelectParams {
+  int T, E, k, d, C_stride, capacity, c_floor, adaptive, mode;
+  float delta_max_override;
+};
+
+// C = capacity, or clamp(ceil((1/E) exp{d dm^2/(2-dm^2)}), c_floor, capacity).
+__device__ inline int capacity_from_delta(const SelectParams& p, float delta_max) {
+  if (!p.adaptive) return p.capacity;
+  double ds = p.delta_max_override >= 0.f ? (double)p.delta_max_override : (double)delta_max;
+  ds = fmin(1.0, fmax(0.0, ds));
+  const double y = (double)p.d * ds * ds / (2.0 - ds * ds);
+  const double cmin = ceil(exp(y) / (double)p.E);
+  const double c = fmin((double)p.capacity, fmax((double)p.c_floor, cmin));
+  return (int)c;
+}
+
+__global__ void __launch_bounds__(256)
+select_token_side_kernel(const float* __restrict__ delta, int32_t* __restrict__ topk_idx,
+                         uint32_t* __restrict__ keyT, etr_stats* stats, SelectParams p) {
+  __shared__ uint32_t tile[256 * (SEL_TB + 1)];      // [E][33]
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int t0 = blockIdx.x * SEL_TB;
+  if (blockIdx.x == 0 && tid == 0) {
+    const uint32_t mk = stats->delta_max_key;
+    const float dm = mk ? key_to_float(mk) : 0.f;
+    stats->delta_max = dm;
+    stats->mode = p.mode;
+    stats->C = capacity_from_delta(p, dm);
+  }
+  for (int tt = warp; tt < SEL_TB; tt += 8) {
+    const int t = t0 + tt;
+    uint32_t key[SEL_MAX_EPL];
+    bool cand[SEL_MAX_EPL];
+#pragma unroll
+    for (int u = 0; u < SEL_MAX_EPL; ++u) {
+      const int i = lane + 32 * u;
+      key[u] = (t < p.T && i < p.E) ? ordered_key(delta[(size_t)t * p.E + i]) : 0u;
+      cand[u] = (p.mode == ETR_MODE_ECR);
+    }
+    if (p.mode == ETR_MODE_TCR && t < p.T) {
+      for (int j = 0; j < p.k; ++j) {
+        // arg-max over (key, lower index wins) among experts not yet taken
+        unsigned long long best = 0ull;
+#pragma unroll
+        for (int u = 0; u < SEL_MAX_EPL; ++u) {
+          const int i = lane + 32 * u;
+          if (i < p.E && !cand[u]) {
+            const unsigned long long v = ((unsigned long long)key[u] << 32) | (uint32_t)(0x7fffffff - i);
+            best = v > best ? v : best;
+          }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+          const unsigned long long other = __shfl_xor_sync(0xffffffffu, best, o);
+          best = other > best ? other : best;
+        }
+        const int win = 0x7fffffff - (int)(uint32_t)(best & 0xffffffffull);
+        if (lane == (win & 31)) {
+#pragma unroll
+          for (int u = 0; u < SEL_MAX_EPL; ++u) if (u == (win >> 5)) cand[u] = true;
+        }
+        if (lane == 0) topk_idx[(size_t)t * p.k + j] = win;
+      }
+    } else if (t < p.T) {
+      for (int j = lane; j < p.k; j += 32) topk_idx[(size_t)t * p.k + j] = -1;
+    }
+#pragma unroll
+    for (int u = 0; u < SEL_MAX_EPL; ++u) {
+      const int i = lane + 32 * u;
+      if (i < p.E) tile[i * (SEL_TB + 1) + tt] = cand[u] ? key[u] : 0u;
+    }
+  }
+  __syncthreads();
+  for (int idx = tid; idx < p.E * SEL_TB; idx += 256) {
+    const int i = idx / SEL_TB, tt = idx % SEL_TB;
+    if (t0 + tt < p.T) keyT[(size_t)i * p.T + t0 + tt] = tile[i * (SEL_TB + 1) + tt];
+  }
+}
+
+// One CTA (1024 threads) per expert.
+__global__ void __launch_bounds__(1024)
+select_expert_side_kernel(uint32_t* __restrict__ keyT, const etr_stats* __restrict__ stats,
+                          int32_t* __restrict__ counts, int32_t* __restrict__ slot_token,
+                          float* __restrict__ gate, int T, int C_stride) {
+  __shared__ uint32_t hist[256];
+  __shared__ uint32_t s_prefix, s_remaining, s_ncand;
+  __shared__ uint32_t warp_gt[32], warp_eq[32];
+  __shared__ uint32_t base_sel, base_eq;
+  const int i = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  uint32_t* row = keyT + (size_t)i * T;
+  int32_t* my_slot = slot_token + (size_t)i * C_stride;
+  float* my_gate = gate + (size_t)i * C_stride;
+  const int C = stats->C;
+
+  // candidates = keys > 0
+  if (tid == 0) s_ncand = 0;
+  __syncthreads();
+  uint32_t nc = 0;
+  for (int t = tid; t < T; t += 1024) nc += row[t] != 0u;
+  for (int o = 16; o > 0; o >>= 1) nc += __shfl_xor_sync(0xffffffffu, nc, o);
+  if (lane == 0 && nc) atomicAdd(&s_ncand, nc);
+  __syncthreads();
+  const uint32_t n_keep = min((uint32_t)C, s_ncand);
+
+  // radix select: the n_keep-th largest key
+  uint32_t tau = 0, quota = 0;
+  if (n_keep > 0) {
+    if (tid == 0) { s_prefix = 0; s_remaining = n_keep; }
+    for (int pass = 0; pass < 4; ++pass) {
+      const int shift = 24 - 8 * pass;
+      if (tid < 256) hist[tid] = 0;
+      __syncthreads();
+      const uint32_t prefix = s_prefix;
+      const uint32_t pmask = pass == 0 ? 0u : (0xffffffffu << (shift + 8));
+      for (int t = tid; t < T; t += 1024) {
+        const uint32_t kx = row[t];
+        if ((kx & pmask) == prefix) atomicAdd(&hist[(kx >> shift) & 0xff], 1u);
+      }
+      __syncthreads();
+      if (tid == 0) {
+        uint32_t rem = s_remaining;
+        int b = 255;
+        for (; b > 0; --b) {
+          if (hist[b] >= rem) break;
+          rem -= hist[b];
+        }
+        s_prefix = prefix | ((uint32_t)b << shift);
+        s_remaining = rem;        // after the last pass: how many keys == tau are admitted
+      }
+      __syncthreads();
+    }
+    tau = s_prefix;
+    quota = s_remaining;
+  }
+
+  // slot assignment in ascending token order
+  if (tid == 0) { base_sel = 0; base_eq = 0; }
+  __syncthreads();
+  for (int c0 = 0; c0 < T; c0 += 1024) {
+    const int t = c0 + tid;
+    const uint32_t kx = t < T ? row[t] : 0u;
+    const bool gt = n_keep > 0 && kx > tau;
+    const bool eq = n_keep > 0 && kx == tau && kx != 0u;
+    const uint32_t b_gt = __ballot_sync(0xffffffffu, gt), b_eq = __ballot_sync(0xffffffffu, eq);
+    if (lane == 0) { warp_gt[warp] = __popc(b_gt); warp_eq[warp] = __popc(b_eq); }
+    __syncthreads();
+    uint32_t pre_gt = 0, pre_eq = 0, tot_gt = 0, tot_eq = 0;
+    for (int w = 0; w < 32; ++w) {
+      const uint32_t g = warp_gt[w], e = warp_eq[w];
+      if (w < warp) { pre_gt += g; pre_eq += e; }
+      tot_gt += g; tot_eq += e;
+    }
+    const uint32_t lt_mask = (1u << lane) - 1u;
+    const uint32_t eq_rank = base_eq + pre_eq + __popc(b_eq & lt_mask);   // rank among key == tau
+    const uint32_t gt_rank = pre_gt + __popc(b_gt & lt_mask);             // within this chunk
+    const uint32_t eq_before_chunk = min(base_eq, quota);
+    const uint32_t eq_adm_before_me = min(eq_rank, quota) - eq_before_chunk;
+    const bool sel = gt || (eq && eq_rank < quota);
+    int pos = -1;
+    if (sel) {
+      pos = (int)(base_sel + gt_rank + eq_adm_before_me);
+      my_slot[pos] = t;
+      my_gate[pos] = key_to_float(kx);
+    }
+    if (t < T) row[t] = (uint32_t)pos;
+    __syncthreads();
+    if (tid == 0) {
+      const uint32_t eq_after = min(base_eq + tot_eq, quota);
+      base_sel += tot_gt + (eq_after - eq_before_chunk);
+      base_eq += tot_eq;
+    }
+    __syncthreads();
+  }
+  for (int p = (int)n_keep + tid; p < C_stride; p += 1024) { my_slot[p] = -1; my_gate[p] = 0.f; }
+  if (tid == 0) counts[i] = (int)n_keep;
+}
+
+// rows per token (tok_ptr[t+1] = count), plus the number of unrouted tokens
+__global__ void __launch_bounds__(256)
+csr_count_kernel(const int32_t* __restrict__ posT, int32_t* __restrict__ tok_ptr, etr_stats* stats,
+                 int T, int E) {
+  const int t = blockIdx.x * 256 + threadIdx.x;
+  int n = 0;
+  if (t < T) {
+    for (int i = 0; i < E; ++i) n += posT[(size_t)i * T + t] >= 0;
+    tok_ptr[t + 1] = n;
+  }
+  const uint32_t un = __ballot_sync(0xffffffffu, t < T && n == 0);
+  if ((threadIdx.x & 31) == 0 && un) atomicAdd(&stats->unrouted, __popc(un));
+}
+
+// in-place inclusive scan of tok_ptr[1..T] (single CTA), i.e. exclusive offsets in tok_ptr[0..T]
+__global__ void __launch_bounds__(1024)
+csr_scan_kernel(int32_t* __restrict__ tok_ptr, etr_stats* stats, int T, int n_cand) {
+  __shared__ int wsum[32];
+  __shared__ int carry;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (tid == 0) { carry = 0; tok_ptr[0] = 0; }
+  __syncthreads();
+  for (int c0 = 0; c0 < T; c0 += 1024) {
+    const int t = c0 + tid;
+    const int v = t < T ? tok_ptr[t + 1] : 0;
+    int inc = v;
+    for (int o = 1; o < 32; o <<= 1) {
+      const int y = __shfl_up_sync(0xffffffffu, inc, o);
+      if (lane >= o) inc += y;
+    }
+    if (lane == 31) wsum[warp] = inc;
+    __syncthreads();
+    int pre = carry;
+    for (int w = 0; w < warp; ++w) pre += wsum[w];
+    if (t < T) tok_ptr[t + 1] = pre + inc;
+    __syncthreads();
+    if (tid == 1023) carry = pre + inc;
+    __syncthreads();
+  }
+  if (tid == 0) {
+    stats->rows_total = carry;
+    stats->dropped = n_cand - carry;
+  }
+}
+
+__global__ void __launch_bounds__(256)
+csr_fill_kernel(const int32_t* __restrict__ posT, const int32_t* __restrict__ tok_ptr,
+                int32_t* __restrict__ tok_row, int T, int E, int C_stride) {
+  const int t = blockIdx.x * 256 + threadIdx.x;
+  if (t >= T) return;
+  int q = tok_ptr[t];
+  for (int i = 0; i < E; ++i) {
+    const int pos = posT[(size_t)i * T + t];
+    if (pos >= 0) tok_row[q++] = i * C_stride + pos;
+  }
+}
+
+size_t select_workspace_bytes(const etr_config* c) { return (size_t)c->T * c->E * sizeof(uint32_t); }
+
+int resolve_mode(const etr_config* c) {
+  if (c->mode == ETR_MODE_TCR || c->mode == ETR_MODE_ECR) return c->mode;
+  return c->step < c->switch_step ? ETR_MODE_TCR : ETR_MODE_ECR;
+}
+
+etr_status select_forward(const etr_config* c, const float* delta, etr_stats* stats,
+                          const etr_route* rt, void* ws, cudaStream_t st) {
+  SelectParams p;
+  p.T = c->T; p.E = c->E; p.k = c->k; p.d = c->d; p.C_stride = c_stride_of(c);
+  p.capacity = c->capacity; p.c_floor = c->c_floor < 1 ? 1 : c->c_floor; p.adaptive = c->adaptive;
+  p.mode = resolve_mode(c); p.delta_max_override = c->delta_max_override;
+  uint32_t* keyT = (uint32_t*)ws;
+  select_token_side_kernel<<<ceil_div(c->T, SEL_TB), 256, 0, st>>>(delta, rt->topk_idx, keyT, stats, p);
+  ETR_LAUNCH_CHECK();
+  select_expert_side_kernel<<<c->E, 1024, 0, st>>>(keyT, stats, rt->counts, rt->slot_token, rt->gate,
+                                                   c->T, p.C_stride);
+  ETR_LAUNCH_CHECK();
+  csr_count_kernel<<<ceil_div(c->T, 256), 256, 0, st>>>((const int32_t*)keyT, rt->tok_ptr, stats, c->T, c->E);
+  ETR_LAUNCH_CHECK();
+  const int n_cand = p.mode == ETR_MODE_TCR ? c->T * c->k : c->T * c->E;
+  csr_scan_kernel<<<1, 1024, 0, st>>>(rt->tok_ptr, stats, c->T, n_cand);
+  ETR_LAUNCH_CHECK();
+  csr_fill_kernel<<<ceil_div(c->T, 256), 256, 0, st>>>((const int32_t*)keyT, rt->tok_ptr, rt->tok_row,
+                                                       c->T, c->E, p.C_stride);
+  ETR_LAUNCH_CHECK();
+  return ETR_OK;
+}
+
+}  // namespace etr
