@@ -12,7 +12,7 @@ void note_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 static bool use_tc(const etr_config* c) {
   if (c->gemm_impl == ETR_GEMM_SIMT) return false;
   if (c->gemm_impl == ETR_GEMM_TCGEN05) return true;
-  return c->dtype == ETR_BF16;
+  return c->dtype == ETR_BF16 && tc_available();
 }
 
 static etr_status check_ptrs(std::initializer_list<const void*> ps) {

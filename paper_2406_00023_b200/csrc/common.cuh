@@ -137,5 +137,6 @@ etr_status tc_ffn_backward(const etr_config* cfg, const etr_route* route, const 
                            void* dXp, void* dW1g, void* dW1u, void* dW2, etr_stats* stats,
                            void* ws, cudaStream_t st);
 size_t tc_workspace_bytes(const etr_config* cfg);
+bool tc_available();
 
 }  // namespace etr
