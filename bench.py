@@ -1,0 +1,337 @@
+"""Benchmark of the ETR MoE layer: forward + backward tokens/s on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload large] [--impl reference]
+
+A step is one pass of the whole hot path (affinity, selection, dispatch, expert FFN,
+combine and every backward stage) over one batch of seeded synthetic tokens.  With N > 1
+(launched by torch.distributed.run) every rank runs an independent replica of the layer on
+its own tokens: the path has no exchange step, so there is no data-path collective and the
+scaling is weak.  Rank 0 prints one JSON line.
+
+`--impl reference` times the CPU oracle (oracle/) on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+from dataclasses import replace
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+import torch  # noqa: E402
+
+from gen import workloads as gw  # noqa: E402
+
+METRIC = "etr_moe_layer_fwd_bwd_tokens_per_sec"
+UNIT = "tokens/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture summarised
+# under profiles/ (None: not captured for the current version of that kernel).
+NCU_TRAFFIC_BYTES = {}
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {k: float(d[k]) for k in FALLBACK_PEAKS if k in d} | {"source": "measured"}
+    return dict(FALLBACK_PEAKS, source="fallback")
+
+
+def mode_name(w):
+    if w.mode in ("tcr", "ecr"):
+        return w.mode
+    return "tcr" if w.step < w.switch_step else "ecr"
+
+
+# ---- algorithmic work per kernel and step (what the method itself must move / compute) ----
+def algorithmic_work(w, rows, kernel):
+    """(amount, "bytes"|"flops") for all launches of `kernel` in one step."""
+    b = 2 if w.dtype == "bf16" else 4
+    T, d, E, h, m = w.T, w.d, w.E, w.h, w.m
+    table = {
+        "affinity_fwd_kernel": (T * d * b + T * E * 4 + T * m * 4 + T * 4, "bytes"),
+        "select_token_side_kernel": (2 * T * E * 4, "bytes"),
+        "select_expert_side_kernel": (T * E * 4 + rows * 8, "bytes"),
+        "csr_count_kernel": (T * E * 4, "bytes"),
+        "csr_scan_kernel": (T * 8, "bytes"),
+        "csr_fill_kernel": (T * E * 4 + rows * 4, "bytes"),
+        "dispatch_kernel": (2 * rows * d * b, "bytes"),
+        "combine_kernel": (2 * (rows * d * b + T * d * b), "bytes"),       # combine + dispatch_bwd
+        "combine_bwd_kernel": (3 * rows * d * b, "bytes"),
+        "affinity_bwd_dx_kernel": (3 * T * d * b, "bytes"),
+        "affinity_bwd_dr_partial_kernel": (rows * m * 4, "bytes"),
+        "affinity_bwd_dr_final_kernel": (E * m * 8, "bytes"),
+        "gemm_simt_kernel": (18 * rows * d * h, "flops"),
+    }
+    return table.get(kernel, (0, "bytes"))
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
+                 "--format=csv,noheader,nounits", "-lms", "200"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=lambda: self.lines.extend(self.proc.stdout), daemon=True)
+            self.t.start()
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.25)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        self.t.join(timeout=2)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(mx) if mx else None, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def oracle_sample_run(w, inputs_host, weights_host, Ts, steps, warmup):
+    """Times the CPU oracle (as it stands) on the first Ts tokens of the workload."""
+    from oracle import binding as ob
+    cores = ob.set_threads(os.cpu_count() or 1)
+    o = ob.Oracle("f32")
+    ws = replace(w, T=Ts)
+    X, dY, R = inputs_host["X"][:Ts], inputs_host["dY"][:Ts], inputs_host["R"]
+    W1g, W1u, W2 = weights_host
+    mode = ob.MODE_TCR if mode_name(w) == "tcr" else ob.MODE_ECR
+    times = []
+    for it in range(warmup + steps):
+        t0 = time.perf_counter()
+        fw = o.forward(X, R, W1g, W1u, W2, D=w.D, k=w.k, capacity=ws.capacity, mode=mode,
+                       adaptive=w.adaptive)
+        o.backward(fw, X, R, W1g, W1u, W2, dY)
+        if it >= warmup:
+            times.append(time.perf_counter() - t0)
+    sec = sum(times) / len(times)
+    return {"value": Ts / sec, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"first {Ts} tokens of the workload, all {w.E} experts, capacity "
+                      f"{ws.capacity}, full forward+backward, {len(times)} step(s) of {sec:.2f} s"}, sec
+
+
+def device_weights(w, device, seed):
+    """Expert weights ~ N(0, 1/d) drawn on the device (seeded); bf16 or fp32 per workload."""
+    g = torch.Generator(device=device)
+    g.manual_seed(seed)
+    dt = torch.bfloat16 if w.dtype == "bf16" else torch.float32
+    std = 1.0 / np.sqrt(w.d)
+    out = []
+    for shape in ((w.E, w.h, w.d), (w.E, w.h, w.d), (w.E, w.d, w.h)):
+        t = torch.empty(shape, dtype=dt, device=device)
+        for e in range(w.E):                       # per expert: bounded fp32 temporaries
+            t[e] = (torch.randn(shape[1:], generator=g, device=device) * std).to(dt)
+        out.append(t)
+    return out
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="large", choices=list(gw.WORKLOADS))
+    ap.add_argument("--gemm", default="auto", choices=["auto", "simt", "tcgen05"])
+    ap.add_argument("--cpu-tokens", type=int, default=128, help="tokens in the CPU-oracle sample")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    w0 = gw.WORKLOADS[args.workload]
+    config = {"workload": f"{w0.name} (config {w0.config_id}): T={w0.T} d={w0.d} D={w0.D} E={w0.E} "
+                          f"k={w0.k} h={w0.h} cf={w0.cf} {mode_name(w0)} adaptive={int(w0.adaptive)} "
+                          f"x={w0.x_kind}",
+              "T": w0.T, "d": w0.d, "D": w0.D, "E": w0.E, "k": w0.k, "h": w0.h,
+              "capacity": w0.capacity, "mode": mode_name(w0), "adaptive": bool(w0.adaptive),
+              "l2": "inputs larger than L2 (no flush)", "parallelism": f"replicas x{world}"}
+
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        w = w0
+        Ts = min(args.cpu_tokens, w.T)
+        inp = gw.make_inputs(replace(w, T=Ts), weights=False)
+        inp["R"] = gw.expert_embeddings(w)
+        W = gw.expert_weights(w)
+        base, sec = oracle_sample_run(w, inp, W, Ts, max(1, args.steps), args.warmup)
+        print(json.dumps({
+            "impl": "reference", "metric": METRIC, "value": base["value"], "unit": UNIT,
+            "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": config,
+            "cpu_baseline": base,
+            "e2e": {"value": base["value"], "unit": UNIT, "h2d_bytes_per_step": 0,
+                    "d2h_bytes_per_step": 0}}))
+        return
+
+    from paper_2406_00023_b200 import etr
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    w = replace(w0, config_id=w0.config_id + 1000 * rank)       # each replica: its own tokens
+
+    inp = gw.make_inputs(w, weights=False)
+    act = torch.bfloat16 if w.dtype == "bf16" else torch.float32
+    Xh = torch.from_numpy(inp["X"]).to(act).pin_memory()
+    dYh = torch.from_numpy(inp["dY"]).to(act).pin_memory()
+    Yh, dXh = torch.empty_like(Xh).pin_memory(), torch.empty_like(Xh).pin_memory()
+    X, dY = Xh.to(dev), dYh.to(dev)
+    R = torch.from_numpy(inp["R"]).to(dev)
+    W1g, W1u, W2 = device_weights(w, dev, w.seed)
+    impl = {"auto": etr.GEMM_AUTO, "simt": etr.GEMM_SIMT, "tcgen05": etr.GEMM_TCGEN05}[args.gemm]
+    cfg = etr.make_config(T=w.T, d=w.d, D=w.D, E=w.E, k=w.k, h=w.h, capacity=w.capacity,
+                          dtype=etr.BF16 if w.dtype == "bf16" else etr.F32,
+                          mode=etr.MODE_TCR if mode_name(w) == "tcr" else etr.MODE_ECR,
+                          step=w.step, switch_step=w.switch_step, adaptive=w.adaptive, gemm_impl=impl)
+    buf = etr.LayerBuffers(cfg, host_staging=True, device=dev)
+    Y, dX = torch.empty_like(X), torch.empty_like(X)
+    dR = torch.empty_like(R)
+    dW1g, dW1u, dW2 = torch.empty_like(W1g), torch.empty_like(W1u), torch.empty_like(W2)
+
+    def step():
+        etr.layer_forward(cfg, X, R, W1g, W1u, W2, buf, Y)
+        etr.layer_backward(cfg, X, R, W1g, W1u, W2, dY, buf, dX, dR, dW1g, dW1u, dW2)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    st = buf.read_stats()
+    assert st.error_word == 0, "a device-side wait expired during warm-up"
+    rows = st.rows_total
+
+    sampler = ClockSampler(local)
+    sampler.start()
+    etr.timing_enable(True)
+    n0 = etr.launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    barrier()
+    launches = etr.launch_count() - n0
+    ms_total = e0.elapsed_time(e1)
+    clocks = sampler.stop()
+    recs = etr.timing_collect()
+    etr.timing_enable(False)
+    assert buf.read_stats().error_word == 0
+
+    # end to end through the host-buffer entry point (H2D and D2H inside the timed region)
+    e2e_steps = max(1, min(args.steps, 5))
+    etr.layer_step_host(cfg, Xh, dYh, R, W1g, W1u, W2, buf, Yh, dXh, dR, dW1g, dW1u, dW2)
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        etr.layer_step_host(cfg, Xh, dYh, R, W1g, W1u, W2, buf, Yh, dXh, dR, dW1g, dW1u, dW2)
+    torch.cuda.synchronize()
+    e2e_ms = (time.perf_counter() - t0) * 1e3 / e2e_steps
+
+    t = torch.tensor([ms_total, e2e_ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_total, e2e_ms = float(t[0]), float(t[1])
+    ms_step = ms_total / args.steps
+
+    # per-kernel table and the roofline of the dominant kernel
+    per = {}
+    for name, ms in recs:
+        if ms >= 0:
+            a = per.setdefault(name, [0, 0.0])
+            a[0] += 1; a[1] += ms
+    peaks = load_peaks()
+    kernels = []
+    for name, (n, ms) in sorted(per.items(), key=lambda kv: -kv[1][1]):
+        amount, kind = algorithmic_work(w, rows, name)
+        per_launch = amount * args.steps / n if n else 0.0
+        avg_ms = ms / n
+        if kind == "flops":
+            ach, peak, unit, bound = per_launch / (avg_ms * 1e-3) / 1e12, peaks["bf16_tflops_sustained"], "TFLOP/s", "tensor"
+        else:
+            ach, peak, unit, bound = per_launch / (avg_ms * 1e-3) / 1e9, peaks["hbm_gbs"], "GB/s", "hbm"
+        kernels.append({"kernel": name, "launches_per_step": n / args.steps, "ms_per_step": ms / args.steps,
+                        "share": ms / sum(v[1] for v in per.values()), "bound": bound,
+                        "achieved": ach, "peak": peak, "unit": unit, "frac": ach / peak})
+    top = kernels[0] if kernels else None
+    roofline = None
+    if top:
+        roofline = {"kernel": top["kernel"], "bound": top["bound"], "achieved": top["achieved"],
+                    "peak": top["peak"], "unit": top["unit"], "frac": top["frac"],
+                    "traffic": NCU_TRAFFIC_BYTES.get(top["kernel"]),
+                    "peak_source": peaks["source"] + (" (sustained)" if top["bound"] == "tensor" else "")}
+
+    out = {"metric": METRIC, "value": world * w.T / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world,
+           "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step,
+           "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+           "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic", "config": config,
+           "clocks": clocks, "gpu_launches": int(launches),
+           "e2e": {"value": world * w.T / (e2e_ms * 1e-3), "unit": UNIT,
+                   "h2d_bytes_per_step": int(2 * Xh.numel() * Xh.element_size()),
+                   "d2h_bytes_per_step": int(2 * Xh.numel() * Xh.element_size()),
+                   "ms_per_step": e2e_ms},
+           "roofline": roofline, "kernels": kernels,
+           "routing": {"C": st.C, "rows": rows, "dropped": st.dropped, "unrouted": st.unrouted,
+                       "delta_max": st.delta_max}}
+
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        Ts = min(args.cpu_tokens, w.T)
+        Wh = [t.float().cpu().numpy() for t in (W1g, W1u, W2)]
+        base, _ = oracle_sample_run(w, {"X": inp["X"], "dY": inp["dY"], "R": inp["R"]}, Wh, Ts, 1, 0)
+        out["cpu_baseline"] = base
+    if rank == 0:
+        print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -235,6 +235,15 @@ etr_status etr_read_stats(const etr_stats* stats_dev, etr_stats* stats_host, voi
 /* Number of kernels launched by this library in the calling process so far. */
 int64_t etr_launch_count(void);
 
+/* Per-kernel timing for benchmarks.  While enabled, every kernel the library launches is
+ * bracketed by a CUDA event pair recorded on the launch stream (host-side objects; no
+ * device memory).  etr_timing_enable clears earlier records.  etr_timing_collect waits for
+ * the recorded events, writes up to max_records kernel names into `names` (host, one per
+ * line, NUL-terminated) and their durations in milliseconds into `ms` (host; -1 where the
+ * time could not be read), clears the records and returns how many it wrote. */
+etr_status etr_timing_enable(int on);
+int64_t etr_timing_collect(char* names, size_t names_bytes, float* ms, int64_t max_records);
+
 #ifdef __cplusplus
 }
 #endif

@@ -293,12 +293,14 @@ etr_status affinity_forward(const etr_config* c, const void* X, const float* R, 
     auto k = affinity_fwd_kernel<__nv_bfloat16>;
     if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
       return ETR_ERR_CUDA;
+    ETR_TIME_BEGIN("affinity_fwd_kernel");
     k<<<grid, AFF_THREADS, smem, st>>>((const __nv_bfloat16*)X, R, delta, Z, xnorm, rnorm, stats,
                                        c->T, c->d, c->D, c->E, m, ldm, Epad);
   } else {
     auto k = affinity_fwd_kernel<float>;
     if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
       return ETR_ERR_CUDA;
+    ETR_TIME_BEGIN("affinity_fwd_kernel");
     k<<<grid, AFF_THREADS, smem, st>>>((const float*)X, R, delta, Z, xnorm, rnorm, stats, c->T,
                                        c->d, c->D, c->E, m, ldm, Epad);
   }
@@ -324,21 +326,25 @@ etr_status affinity_backward(const etr_config* c, const void* X, const float* R,
     auto k = affinity_bwd_dx_kernel<__nv_bfloat16>;
     if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
       return ETR_ERR_CUDA;
+    ETR_TIME_BEGIN("affinity_bwd_dx_kernel");
     k<<<grid, 256, smem, st>>>((const __nv_bfloat16*)X, R, delta, xnorm, rnorm, rt->tok_ptr,
                                rt->tok_row, dgate, (__nv_bfloat16*)dX, c->T, c->d, c->D, c->E, m, Cs);
   } else {
     auto k = affinity_bwd_dx_kernel<float>;
     if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
       return ETR_ERR_CUDA;
+    ETR_TIME_BEGIN("affinity_bwd_dx_kernel");
     k<<<grid, 256, smem, st>>>((const float*)X, R, delta, xnorm, rnorm, rt->tok_ptr, rt->tok_row,
                                dgate, (float*)dX, c->T, c->d, c->D, c->E, m, Cs);
   }
   ETR_LAUNCH_CHECK();
   float* part = (float*)ws;
+  ETR_TIME_BEGIN("affinity_bwd_dr_partial_kernel");
   affinity_bwd_dr_partial_kernel<<<dim3(c->E, nch), 256, 0, st>>>(
       Z, delta, xnorm, rnorm, rt->counts, rt->slot_token, dgate, part, c->E, m, Cs, nch,
       sqrtf((float)c->D));
   ETR_LAUNCH_CHECK();
+  ETR_TIME_BEGIN("affinity_bwd_dr_final_kernel");
   affinity_bwd_dr_final_kernel<<<c->E, 256, 0, st>>>(part, R, rnorm, dR, m, nch);
   ETR_LAUNCH_CHECK();
   return ETR_OK;

@@ -1,6 +1,9 @@
 // C ABI of libetr: argument checks, buffer carving, stage wrappers, whole-layer calls.
 #include <atomic>
 #include <cstring>
+#include <mutex>
+#include <string>
+#include <vector>
 
 #include "common.cuh"
 
@@ -8,6 +11,32 @@ namespace etr {
 
 static std::atomic<long long> g_launches{0};
 void note_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+// ---- optional per-kernel timing: one CUDA event pair per launch, on the launch stream ----
+struct TimingRecord { const char* name; cudaEvent_t beg, end; };
+static std::mutex g_timing_mu;
+static bool g_timing_on = false;
+static std::vector<TimingRecord> g_records;
+static std::vector<cudaEvent_t> g_event_pool;
+
+static cudaEvent_t take_event() {
+  if (!g_event_pool.empty()) { cudaEvent_t e = g_event_pool.back(); g_event_pool.pop_back(); return e; }
+  cudaEvent_t e = nullptr;
+  cudaEventCreate(&e);
+  return e;
+}
+void timing_begin(const char* name, cudaStream_t st) {
+  if (!g_timing_on) return;
+  std::lock_guard<std::mutex> lk(g_timing_mu);
+  TimingRecord r{name, take_event(), take_event()};
+  if (r.beg) cudaEventRecord(r.beg, st);
+  g_records.push_back(r);
+}
+void timing_end(cudaStream_t st) {
+  if (!g_timing_on) return;
+  std::lock_guard<std::mutex> lk(g_timing_mu);
+  if (!g_records.empty() && g_records.back().end) cudaEventRecord(g_records.back().end, st);
+}
 
 static bool use_tc(const etr_config* c) {
   if (c->gemm_impl == ETR_GEMM_SIMT) return false;
@@ -303,5 +332,38 @@ etr_status etr_read_stats(const etr_stats* dev, etr_stats* host, void* stream) {
 }
 
 int64_t etr_launch_count(void) { return (int64_t)g_launches.load(); }
+
+etr_status etr_timing_enable(int on) {
+  std::lock_guard<std::mutex> lk(g_timing_mu);
+  for (auto& r : g_records) { g_event_pool.push_back(r.beg); g_event_pool.push_back(r.end); }
+  g_records.clear();
+  g_timing_on = on != 0;
+  return ETR_OK;
+}
+
+int64_t etr_timing_collect(char* names, size_t names_bytes, float* ms, int64_t max_records) {
+  std::lock_guard<std::mutex> lk(g_timing_mu);
+  int64_t n = 0;
+  size_t off = 0;
+  if (names && names_bytes) names[0] = 0;
+  for (auto& r : g_records) {
+    if (n >= max_records) break;
+    float t = -1.f;
+    if (!r.beg || !r.end || cudaEventSynchronize(r.end) != cudaSuccess ||
+        cudaEventElapsedTime(&t, r.beg, r.end) != cudaSuccess)
+      t = -1.f;
+    const size_t len = strlen(r.name);
+    if (!names || off + len + 2 > names_bytes) break;
+    memcpy(names + off, r.name, len);
+    names[off + len] = '\n';
+    names[off + len + 1] = 0;
+    off += len + 1;
+    if (ms) ms[n] = t;
+    ++n;
+  }
+  for (auto& r : g_records) { g_event_pool.push_back(r.beg); g_event_pool.push_back(r.end); }
+  g_records.clear();
+  return n;
+}
 
 }  // extern "C"

@@ -10,8 +10,13 @@ namespace etr {
 
 // ---- launch accounting and error mapping ------------------------------------------------
 void note_launch(int n = 1);
+// Optional per-kernel timing (etr_timing_enable): an event pair around every launch.
+void timing_begin(const char* kernel_name, cudaStream_t st);
+void timing_end(cudaStream_t st);
+#define ETR_TIME_BEGIN(name) ::etr::timing_begin(name, st)
 #define ETR_LAUNCH_CHECK()                                  \
   do {                                                      \
+    ::etr::timing_end(st);                                  \
     ::etr::note_launch();                                   \
     cudaError_t e__ = cudaGetLastError();                   \
     if (e__ != cudaSuccess) return ETR_ERR_CUDA;            \

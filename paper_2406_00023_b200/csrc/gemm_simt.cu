@@ -114,6 +114,7 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(GemmArgs g) {
 template <class T, int EPI>
 static etr_status launch(const GemmArgs& g, int E, cudaStream_t st) {
   dim3 grid(ceil_div(g.N, 64), ceil_div(g.dyn == DYN_M ? g.m_cap : g.M, 64), E);
+  ETR_TIME_BEGIN("gemm_simt_kernel");
   gemm_simt_kernel<T, EPI><<<grid, 256, 0, st>>>(g);
   ETR_LAUNCH_CHECK();
   return ETR_OK;

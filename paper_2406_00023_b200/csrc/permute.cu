@@ -93,17 +93,20 @@ static etr_status permute_launch(int which, const etr_config* c, const etr_route
   const int Cs = c_stride_of(c), n_rows = c->E * Cs;
   switch (which) {
     case 0:
+      ETR_TIME_BEGIN("dispatch_kernel");
       dispatch_kernel<T><<<ceil_div(n_rows, 8), 256, 0, st>>>((const T*)a, rt->counts, rt->slot_token,
                                                              (T*)out, c->d, Cs, n_rows);
       break;
     case 1:
     case 3: {
       const long long n = (long long)c->T * (c->d / 8);
+      ETR_TIME_BEGIN("combine_kernel");
       combine_kernel<T><<<(unsigned)((n + 255) / 256), 256, 0, st>>>(
           (const T*)a, which == 1 ? rt->gate : nullptr, rt->tok_ptr, rt->tok_row, (T*)out, c->T, c->d);
       break;
     }
     case 2:
+      ETR_TIME_BEGIN("combine_bwd_kernel");
       combine_bwd_kernel<T><<<ceil_div(n_rows, 8), 256, 0, st>>>(
           (const T*)a, (const T*)b, rt->counts, rt->slot_token, rt->gate, (T*)out, dgate, c->d, Cs, n_rows);
       break;

@@ -266,16 +266,21 @@ etr_status select_forward(const etr_config* c, const float* delta, etr_stats* st
   p.capacity = c->capacity; p.c_floor = c->c_floor < 1 ? 1 : c->c_floor; p.adaptive = c->adaptive;
   p.mode = resolve_mode(c); p.delta_max_override = c->delta_max_override;
   uint32_t* keyT = (uint32_t*)ws;
+  ETR_TIME_BEGIN("select_token_side_kernel");
   select_token_side_kernel<<<ceil_div(c->T, SEL_TB), 256, 0, st>>>(delta, rt->topk_idx, keyT, stats, p);
   ETR_LAUNCH_CHECK();
+  ETR_TIME_BEGIN("select_expert_side_kernel");
   select_expert_side_kernel<<<c->E, 1024, 0, st>>>(keyT, stats, rt->counts, rt->slot_token, rt->gate,
                                                    c->T, p.C_stride);
   ETR_LAUNCH_CHECK();
+  ETR_TIME_BEGIN("csr_count_kernel");
   csr_count_kernel<<<ceil_div(c->T, 256), 256, 0, st>>>((const int32_t*)keyT, rt->tok_ptr, stats, c->T, c->E);
   ETR_LAUNCH_CHECK();
   const int n_cand = p.mode == ETR_MODE_TCR ? c->T * c->k : c->T * c->E;
+  ETR_TIME_BEGIN("csr_scan_kernel");
   csr_scan_kernel<<<1, 1024, 0, st>>>(rt->tok_ptr, stats, c->T, n_cand);
   ETR_LAUNCH_CHECK();
+  ETR_TIME_BEGIN("csr_fill_kernel");
   csr_fill_kernel<<<ceil_div(c->T, 256), 256, 0, st>>>((const int32_t*)keyT, rt->tok_ptr, rt->tok_row,
                                                        c->T, c->E, p.C_stride);
   ETR_LAUNCH_CHECK();

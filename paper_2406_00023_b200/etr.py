@@ -24,7 +24,7 @@ EXPORTS = [
     "etr_buffers_bind", "etr_affinity", "etr_select", "etr_dispatch", "etr_expert_ffn", "etr_combine",
     "etr_combine_bwd", "etr_expert_ffn_bwd", "etr_dispatch_bwd", "etr_select_bwd", "etr_affinity_bwd",
     "etr_layer_forward", "etr_layer_backward", "etr_layer_step_host", "etr_read_stats",
-    "etr_launch_count",
+    "etr_launch_count", "etr_timing_enable", "etr_timing_collect",
 ]
 
 
@@ -85,6 +85,20 @@ def status_string(code: int) -> str:
 
 def launch_count() -> int:
     return int(lib().etr_launch_count())
+
+
+def timing_enable(on: bool) -> None:
+    lib().etr_timing_enable(int(bool(on)))
+
+
+def timing_collect(max_records: int = 1 << 16):
+    """[(kernel name, milliseconds)] for every launch since timing was enabled."""
+    names = C.create_string_buffer(max_records * 48)
+    ms = (C.c_float * max_records)()
+    f = lib().etr_timing_collect
+    f.restype = C.c_int64
+    n = f(names, C.c_size_t(len(names)), ms, C.c_int64(max_records))
+    return list(zip(names.value.decode().split("\n")[:n], [float(ms[i]) for i in range(n)]))
 
 
 def _check(code, where):

@@ -1,0 +1,45 @@
+"""The C-ABI library builds without a GPU, loads, and exports every function include/etr.h
+declares; host-side argument checks work with no device present."""
+import ctypes
+import os
+import re
+
+from paper_2406_00023_b200 import build as etr_build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "etr.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(etr_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol():
+    lib = ctypes.CDLL(etr_build.build())
+    names = declared_functions()
+    assert len(names) >= 23
+    for n in names:
+        assert hasattr(lib, n), f"{n} declared in etr.h but not exported"
+
+
+def test_binding_lists_the_same_entry_points():
+    from paper_2406_00023_b200 import etr
+    assert sorted(etr.EXPORTS) == declared_functions()
+
+
+def test_host_side_validation_needs_no_gpu():
+    from paper_2406_00023_b200 import etr
+    good = etr.make_config(T=512, d=256, D=4, E=8, k=2, h=512, capacity=160, dtype=etr.F32)
+    assert etr.validate(good) == etr.OK
+    assert etr.c_stride(good) == 256
+    assert etr.workspace_bytes(good) > 0
+    assert etr.validate(etr.make_config(T=512, d=256, D=3, E=8, k=2, h=512, capacity=160, dtype=etr.F32)) == etr.ERR_SHAPE
+    assert etr.validate(etr.make_config(T=512, d=256, D=4, E=8, k=9, h=512, capacity=160, dtype=etr.F32)) == etr.ERR_SHAPE
+    assert etr.validate(etr.make_config(T=512, d=256, D=4, E=8, k=2, h=512, capacity=0, dtype=etr.F32)) == etr.ERR_ARG
+    assert etr.validate(etr.make_config(T=512, d=256, D=4, E=8, k=2, h=512, capacity=160, dtype=5)) == etr.ERR_ARG
+    assert "aligned" in etr.status_string(etr.ERR_ALIGN)
+    n = ctypes.c_size_t(0)
+    assert etr.lib().etr_buffers_bytes(ctypes.byref(good), 1, ctypes.byref(n)) == etr.OK and n.value > 1 << 20
+    # struct layouts the binding relies on
+    assert ctypes.sizeof(etr.Config) == 72 and ctypes.sizeof(etr.Stats) == 64
