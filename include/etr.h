@@ -153,6 +153,30 @@ etr_status etr_affinity(const etr_config* cfg, const void* X, const float* R, fl
 etr_status etr_select(const etr_config* cfg, const float* delta, etr_stats* stats,
                       const etr_route* route, void* ws, void* stream);
 
+/* etr_select for callers that cannot allocate device memory (the paper has no counterpart;
+ * this is a deployment variant of the call above, same results bit for bit).
+ *
+ * Some hosts of this library may not call cudaMalloc at all: code running inside another
+ * framework's stream callback or memory-pool-managed region, plugins loaded into a process
+ * whose device memory was fully handed to a pool at start-up, or real-time loops where an
+ * allocation (an implicit device synchronisation) is forbidden.  They pass delta, stats and
+ * the route outputs as usual, and the T*E 32-bit keys that etr_select keeps in `ws` live
+ * instead in a fixed array inside the library image.
+ *
+ * Limit: T*E <= ETR_SELECT_STATIC_MAX_ENTRIES (16 MiB of keys, enough for every workload up
+ * to T=65536, E=64); larger problems return ETR_ERR_WORKSPACE and launch nothing.  Every GPU
+ * that loads the library carries those 16 MiB until the process ends.
+ * The call itself allocates and frees nothing.  Its first use on a device looks up the
+ * array's device address (once per device, with that device current); make that first call
+ * outside any stream capture.
+ * All calls share the one array, which keeps whatever the previous call left in it: the
+ * selection overwrites every entry it later reads, so nothing needs clearing, but two calls
+ * whose kernels overlap on the same GPU (different streams, or threads) race on it — keep
+ * such calls ordered. */
+#define ETR_SELECT_STATIC_MAX_ENTRIES (4u * 1024u * 1024u)
+etr_status etr_select_static(const etr_config* cfg, const float* delta, etr_stats* stats,
+                             const etr_route* route, void* stream);
+
 /* Token rearrangement: Xp[r,:] = X[slot_token[r],:] for rows in use, 0 for pad rows. */
 etr_status etr_dispatch(const etr_config* cfg, const void* X, const etr_route* route, void* Xp,
                         void* stream);

@@ -11,6 +11,8 @@
 //      scan in token order assigns slots (ascending token id).  The row of keyT is
 //      overwritten with the slot position (or -1).
 //   3. token-major CSR from the position matrix: count, exclusive scan, fill.
+#include <mutex>
+
 #include "common.cuh"
 
 namespace etr {
@@ -288,3 +290,48 @@ etr_status select_forward(const etr_config* c, const float* delta, etr_stats* st
 }
 
 }  // namespace etr
+
+// ---- selection without caller scratch ----------------------------------------------------------
+// Same kernels as select_forward, but the key matrix lives in a fixed device array that is
+// part of the library image, for callers that have no way to allocate device memory (see
+// etr_select_static in etr.h).  Every GPU that loads the library holds these bytes until the
+// process exits.
+namespace etr {
+
+constexpr size_t SELECT_STATIC_MAX_BYTES = ETR_SELECT_STATIC_MAX_ENTRIES * sizeof(uint32_t);
+static __device__ __align__(256) unsigned char g_select_scratch[SELECT_STATIC_MAX_BYTES];
+
+// In host code `g_select_scratch` is only a handle for the runtime's symbol table, not a
+// device address; the address is looked up once per device and cached.
+static std::mutex g_scratch_mu;
+static void* g_scratch_addr[64] = {};
+
+static etr_status select_scratch_address(void** out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return ETR_ERR_CUDA;
+  std::lock_guard<std::mutex> lk(g_scratch_mu);
+  if (g_scratch_addr[dev] == nullptr) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_select_scratch) != cudaSuccess || p == nullptr) return ETR_ERR_CUDA;
+    g_scratch_addr[dev] = p;
+  }
+  *out = g_scratch_addr[dev];
+  return ETR_OK;
+}
+
+}  // namespace etr
+
+extern "C" etr_status etr_select_static(const etr_config* cfg, const float* delta, etr_stats* stats,
+                                        const etr_route* route, void* stream) {
+  using namespace etr;
+  ETR_TRY(etr_validate(cfg));
+  if (delta == nullptr || stats == nullptr || route == nullptr) return ETR_ERR_ARG;
+  if (!route->topk_idx || !route->counts || !route->slot_token || !route->gate || !route->tok_ptr ||
+      !route->tok_row)
+    return ETR_ERR_ARG;
+  if (!aligned16(delta) || !aligned16(stats)) return ETR_ERR_ALIGN;
+  if (select_workspace_bytes(cfg) > SELECT_STATIC_MAX_BYTES) return ETR_ERR_WORKSPACE;
+  void* scratch = nullptr;
+  ETR_TRY(select_scratch_address(&scratch));
+  return select_forward(cfg, delta, stats, route, scratch, (cudaStream_t)stream);
+}

@@ -21,7 +21,7 @@ GEMM_AUTO, GEMM_SIMT, GEMM_TCGEN05 = 0, 1, 2
 
 EXPORTS = [
     "etr_status_string", "etr_validate", "etr_c_stride", "etr_workspace_bytes", "etr_buffers_bytes",
-    "etr_buffers_bind", "etr_affinity", "etr_select", "etr_dispatch", "etr_expert_ffn", "etr_combine",
+    "etr_buffers_bind", "etr_affinity", "etr_select", "etr_select_static", "etr_dispatch", "etr_expert_ffn", "etr_combine",
     "etr_combine_bwd", "etr_expert_ffn_bwd", "etr_dispatch_bwd", "etr_select_bwd", "etr_affinity_bwd",
     "etr_layer_forward", "etr_layer_backward", "etr_layer_step_host", "etr_read_stats",
     "etr_launch_count", "etr_timing_enable", "etr_timing_collect",
@@ -214,6 +214,17 @@ def affinity(cfg, X, R, delta, Z, xnorm, rnorm, stats):
 def select(cfg, delta, stats, route: Route, ws):
     _check(lib().etr_select(C.byref(cfg), _p(delta), _p(stats), C.byref(route), _p(ws), _stream()),
            "etr_select")
+
+
+SELECT_STATIC_MAX_ENTRIES = 4 * 1024 * 1024
+
+
+def select_static(cfg, delta, stats, route: Route):
+    """etr_select without a scratch argument: for callers that cannot allocate device memory.
+    The keys live in a fixed 16 MiB array inside the library (T*E <= SELECT_STATIC_MAX_ENTRIES);
+    calls that overlap on one GPU race on it."""
+    _check(lib().etr_select_static(C.byref(cfg), _p(delta), _p(stats), C.byref(route), _stream()),
+           "etr_select_static")
 
 
 def dispatch(cfg, X, route: Route, Xp):
