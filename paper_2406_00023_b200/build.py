@@ -25,7 +25,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     if stale:
         nvcc = os.environ.get("NVCC", "nvcc")
         cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-o", LIB] + \
-              [os.path.join(CSRC, s) for s in SOURCES] + ["-lcuda"]
+              [os.path.join(CSRC, s) for s in SOURCES]
         subprocess.check_call(cmd)
     return LIB
 

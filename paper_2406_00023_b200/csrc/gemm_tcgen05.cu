@@ -1,15 +1,556 @@
-// placeholder until the tcgen05 kernels land
+// Grouped GEMMs of the expert FFN on the 5th-generation tensor cores (bf16 in, fp32
+// accumulate in tensor memory).  One persistent, warp-specialised kernel serves all six
+// contractions of the forward and backward pass:
+//
+//   warp 0      TMA producer: 64x64-element boxes (128-byte swizzle) into a 4-stage ring
+//   warp 1      allocates tensor memory, issues tcgen05.mma (128 x 256 x 16 per instruction)
+//   warps 2-5   epilogue: tcgen05.ld of the fp32 accumulator, fused SwiGLU / its derivative,
+//               bf16 stores; two accumulator stages so it overlaps the next tile's MMAs
+//
+// Every operand is fetched as 64x64 boxes of its row-major tensor, so one tensor map per
+// tensor serves both uses of it: "K-major" (the contraction index is contiguous in memory)
+// and "MN-major" (the output index is contiguous: weight-gradient GEMMs, which contract over
+// rows, and the data-gradient GEMMs, which read the weights transposed).  Only the
+// shared-memory matrix descriptor differs.
+//
+// Tiles never straddle experts: the per-expert row count is read from `counts` on the
+// device, and tiles are dealt round-robin to the CTAs of a persistent grid.  All waits on
+// mbarriers are bounded; on expiry the kernel records a code in etr_stats.error_word,
+// stops issuing work, releases its tensor memory and returns.
+#include <cuda.h>
+
+#include <mutex>
+
 #include "common.cuh"
+
 namespace etr {
+
+constexpr int TC_BM = 128;
+constexpr int TC_BK = 64;
+constexpr int TC_STAGES = 4;
+constexpr int TC_THREADS = 192;
+constexpr uint32_t TC_BOX_BYTES = 64 * 64 * 2;
+constexpr long long TC_WAIT_LIMIT_CYCLES = 4000000000ll;   // about two seconds
+
+enum { TC_EPI_STORE = 0, TC_EPI_SWIGLU = 1, TC_EPI_DSWIGLU = 2 };
+enum { TC_DYN_M = 1, TC_DYN_K = 2 };
+
+struct TcParams {
+  int a_mn, b_mn;        // 1: operand is MN-major in memory
+  int dual_b;            // SwiGLU: accumulator columns [0,128) from B0, [128,256) from B1
+  int k1_blocks;         // > 0: K blocks [0,k1) use (A0,B0), the rest (A1,B1)
+  int M, N, K;           // per-expert extents (DYN_M: M = C_stride cap; DYN_K: K unused)
+  int dyn, E;
+  const int32_t* counts;
+  __nv_bfloat16* out0; __nv_bfloat16* out1; __nv_bfloat16* out2;
+  const __nv_bfloat16* in0; const __nv_bfloat16* in1;
+  long long out_bs;      // elements between experts in the outputs (and in0/in1)
+  int ld_out;
+  uint32_t idesc;
+  etr_stats* stats;
+};
+
+// ---- PTX wrappers -----------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait: false if this or another thread of the CTA gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  for (uint32_t it = 1;; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((it & 255u) == 0u) {
+      if (*abort_flag) return false;
+      if (clock64() - t0 > TC_WAIT_LIMIT_CYCLES) { *abort_flag = 1; return false; }
+    }
+  }
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0,
+                                            int c1, int c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
+      " [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                       uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]),
+        "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]),
+        "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]),
+        "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr));
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor, 128-byte swizzle, tile base 1024-byte aligned.
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  uint64_t d = (uint64_t)((addr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)(lbo_bytes >> 4) << 16;
+  d |= (uint64_t)(sbo_bytes >> 4) << 32;
+  d |= 1ull << 46;     // descriptor version of this architecture
+  d |= 2ull << 61;     // 128-byte swizzle
+  return d;
+}
+
+__device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+__device__ __forceinline__ void store32(__nv_bfloat16* dst, const float* v) {
+  uint4* p = reinterpret_cast<uint4*>(dst);
+#pragma unroll
+  for (int q = 0; q < 4; ++q)
+    p[q] = make_uint4(pack_bf16(v[8 * q], v[8 * q + 1]), pack_bf16(v[8 * q + 2], v[8 * q + 3]),
+                      pack_bf16(v[8 * q + 4], v[8 * q + 5]), pack_bf16(v[8 * q + 6], v[8 * q + 7]));
+}
+__device__ __forceinline__ void load32(const __nv_bfloat16* src, float* v) {
+  const uint4* p = reinterpret_cast<const uint4*>(src);
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const uint4 w = p[q];
+    const uint32_t u[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      v[8 * q + 2 * i] = __uint_as_float(u[i] << 16);
+      v[8 * q + 2 * i + 1] = __uint_as_float(u[i] & 0xffff0000u);
+    }
+  }
+}
+
+struct TileCoord { int e, m0, n0, kblocks, m_lim; };
+
+// Tile index -> coordinates.  tile_prefix[e] = first tile of expert e.
+__device__ __forceinline__ bool tile_coord(const TcParams& p, const int* tile_prefix, int tile, int& e_cur,
+                                           int n_tile_cols, TileCoord& tc) {
+  if (tile >= tile_prefix[p.E]) return false;
+  while (tile >= tile_prefix[e_cur + 1]) ++e_cur;
+  const int local = tile - tile_prefix[e_cur];
+  const int n_e = p.counts[e_cur];
+  int mt_count;
+  if (p.dyn == TC_DYN_M) {
+    mt_count = (min(n_e, p.M) + TC_BM - 1) / TC_BM;
+    tc.kblocks = (p.K + TC_BK - 1) / TC_BK;
+    tc.m_lim = mt_count * TC_BM;
+  } else {
+    mt_count = (p.M + TC_BM - 1) / TC_BM;
+    tc.kblocks = (n_e + TC_BK - 1) / TC_BK;
+    tc.m_lim = p.M;
+  }
+  tc.e = e_cur;
+  tc.m0 = (local % mt_count) * TC_BM;
+  tc.n0 = (local / mt_count) * n_tile_cols;
+  (void)n_tile_cols;
+  return true;
+}
+
+template <int BN, int EPI>
+__global__ void __launch_bounds__(TC_THREADS, 1)
+tc_grouped_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtensorMap mapA1,
+                       const __grid_constant__ CUtensorMap mapB0, const __grid_constant__ CUtensorMap mapB1,
+                       const TcParams p) {
+  constexpr int B_BOXES = BN / 64;
+  constexpr uint32_t STAGE_BYTES = (2 + B_BOXES) * TC_BOX_BYTES;
+  constexpr int N_TILE_COLS = (EPI == TC_EPI_SWIGLU) ? BN / 2 : BN;
+  constexpr uint32_t TMEM_COLS = 512;
+
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t bars[2 * TC_STAGES + 4];
+  __shared__ uint32_t tmem_base_slot;
+  __shared__ int abort_flag_s;
+  __shared__ int tile_prefix[257];
+
+  volatile int* abort_flag = &abort_flag_s;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const uint32_t tiles_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t full_bar = smem_u32(&bars[0]);                   // [TC_STAGES]
+  const uint32_t empty_bar = smem_u32(&bars[TC_STAGES]);          // [TC_STAGES]
+  const uint32_t tfull_bar = smem_u32(&bars[2 * TC_STAGES]);      // [2]
+  const uint32_t tempty_bar = smem_u32(&bars[2 * TC_STAGES + 2]); // [2]
+
+  // ---- set-up ---------------------------------------------------------------------------------
+  if (tid == 0) {
+    abort_flag_s = 0;
+    for (int s = 0; s < TC_STAGES; ++s) { mbar_init(full_bar + 8 * s, 1); mbar_init(empty_bar + 8 * s, 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar + 8 * a, 1); mbar_init(tempty_bar + 8 * a, 4); }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    const int nt = (p.N + N_TILE_COLS - 1) / N_TILE_COLS;
+    int acc = 0;
+    for (int e = 0; e < p.E; ++e) {
+      tile_prefix[e] = acc;
+      const int n_e = p.counts[e];
+      const int mt = p.dyn == TC_DYN_M ? (min(n_e, p.M) + TC_BM - 1) / TC_BM : (p.M + TC_BM - 1) / TC_BM;
+      acc += mt * nt;
+    }
+    tile_prefix[p.E] = acc;
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"(TMEM_COLS) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_slot;
+
+  if (warp == 0) {
+    // ---- TMA producer ---------------------------------------------------------------------------
+    if (lane == 0) {
+      int e_cur = 0, stage = 0;
+      uint32_t phase = 0;
+      TileCoord tc;
+      bool ok = true;
+      for (int tile = blockIdx.x; ok && tile_coord(p, tile_prefix, tile, e_cur, N_TILE_COLS, tc); tile += gridDim.x) {
+        for (int kb = 0; kb < tc.kblocks; ++kb) {
+          if (!mbar_wait(empty_bar + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
+          const uint32_t fb = full_bar + 8 * stage;
+          mbar_expect_tx(fb, STAGE_BYTES);
+          const bool second = p.k1_blocks > 0 && kb >= p.k1_blocks;
+          const int k0 = (second ? kb - p.k1_blocks : kb) * TC_BK;
+          const CUtensorMap* ma = second ? &mapA1 : &mapA0;
+          const uint32_t sa = tiles_base + stage * STAGE_BYTES;
+          const uint32_t sb = sa + 2 * TC_BOX_BYTES;
+#pragma unroll
+          for (int j = 0; j < 2; ++j) {
+            if (p.a_mn) tma_load_3d(sa + j * TC_BOX_BYTES, ma, fb, tc.m0 + 64 * j, k0, tc.e);
+            else        tma_load_3d(sa + j * TC_BOX_BYTES, ma, fb, k0, tc.m0 + 64 * j, tc.e);
+          }
+#pragma unroll
+          for (int j = 0; j < B_BOXES; ++j) {
+            const CUtensorMap* mb = &mapB0;
+            int nn = tc.n0 + 64 * j;
+            if (p.dual_b) {
+              if (j >= B_BOXES / 2) { mb = &mapB1; nn = tc.n0 + 64 * (j - B_BOXES / 2); }
+            } else if (second) {
+              mb = &mapB1;
+            }
+            if (p.b_mn) tma_load_3d(sb + j * TC_BOX_BYTES, mb, fb, nn, k0, tc.e);
+            else        tma_load_3d(sb + j * TC_BOX_BYTES, mb, fb, k0, nn, tc.e);
+          }
+          if (++stage == TC_STAGES) { stage = 0; phase ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---- MMA issuer ------------------------------------------------------------------------------
+    if (lane == 0) {
+      int e_cur = 0, stage = 0, acc_stage = 0;
+      uint32_t phase = 0, acc_phase = 0;
+      TileCoord tc;
+      bool ok = true;
+      const uint32_t a_lbo = p.a_mn ? TC_BOX_BYTES : 16u, b_lbo = p.b_mn ? TC_BOX_BYTES : 16u;
+      const uint32_t a_kstep = p.a_mn ? 2048u : 32u, b_kstep = p.b_mn ? 2048u : 32u;
+      for (int tile = blockIdx.x; ok && tile_coord(p, tile_prefix, tile, e_cur, N_TILE_COLS, tc); tile += gridDim.x) {
+        if (tc.kblocks == 0) continue;
+        if (!mbar_wait(tempty_bar + 8 * acc_stage, acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc_stage * 256);
+        for (int kb = 0; kb < tc.kblocks; ++kb) {
+          if (!mbar_wait(full_bar + 8 * stage, phase, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sa = tiles_base + stage * STAGE_BYTES;
+          const uint32_t sb = sa + 2 * TC_BOX_BYTES;
+#pragma unroll
+          for (int kk = 0; kk < TC_BK / 16; ++kk) {
+            const uint64_t ad = make_smem_desc(sa + kk * a_kstep, a_lbo, 1024u);
+            const uint64_t bd = make_smem_desc(sb + kk * b_kstep, b_lbo, 1024u);
+            tc_mma(d_tmem, ad, bd, p.idesc, (kb > 0 || kk > 0) ? 1u : 0u);
+          }
+          tc_commit(empty_bar + 8 * stage);          // frees the stage when these MMAs retire
+          if (++stage == TC_STAGES) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        tc_commit(tfull_bar + 8 * acc_stage);        // accumulator complete
+        if (++acc_stage == 2) { acc_stage = 0; acc_phase ^= 1u; }
+      }
+    }
+  } else {
+    // ---- epilogue warps ---------------------------------------------------------------------------
+    const int q = warp & 3;
+    const int row_in_tile = 32 * q + lane;
+    int e_cur = 0, acc_stage = 0;
+    uint32_t acc_phase = 0;
+    TileCoord tc;
+    bool ok = true;
+    for (int tile = blockIdx.x; ok && tile_coord(p, tile_prefix, tile, e_cur, N_TILE_COLS, tc); tile += gridDim.x) {
+      const int grow = tc.m0 + row_in_tile;
+      const bool row_ok = grow < tc.m_lim;
+      const long long obase = (long long)tc.e * p.out_bs + (long long)grow * p.ld_out + tc.n0;
+      if (tc.kblocks == 0) {        // nothing to contract: the block of the output is zero
+        if (row_ok) {
+          float z[32];
+#pragma unroll
+          for (int i = 0; i < 32; ++i) z[i] = 0.f;
+          for (int c = 0; c < N_TILE_COLS / 32 && tc.n0 + 32 * c < p.N; ++c) store32(p.out0 + obase + 32 * c, z);
+        }
+        continue;
+      }
+      if (!mbar_wait(tfull_bar + 8 * acc_stage, acc_phase, abort_flag)) { ok = false; break; }
+      tc_fence_after();
+      const uint32_t taddr = tmem_base + (uint32_t)(acc_stage * 256) + ((uint32_t)(32 * q) << 16);
+#pragma unroll 1
+      for (int c = 0; c < N_TILE_COLS / 32; ++c) {
+        if (tc.n0 + 32 * c >= p.N) break;
+        __syncwarp();               // tcgen05.ld is warp-collective: reconverge after masked stores
+        uint32_t r0[32];
+        float v[32];
+        tc_ld32(taddr + 32 * c, r0);
+        if (EPI == TC_EPI_SWIGLU) {
+          uint32_t r1[32];
+          tc_ld32(taddr + BN / 2 + 32 * c, r1);
+          tc_wait_ld();
+          if (row_ok) {
+            float hv[32];
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+              const float g = __uint_as_float(r0[i]), u = __uint_as_float(r1[i]);
+              hv[i] = g / (1.0f + __expf(-g)) * u;
+              v[i] = g;
+            }
+            store32(p.out0 + obase + 32 * c, v);
+            store32(p.out2 + obase + 32 * c, hv);
+#pragma unroll
+            for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r1[i]);
+            store32(p.out1 + obase + 32 * c, v);
+          }
+        } else if (EPI == TC_EPI_DSWIGLU) {
+          tc_wait_ld();
+          if (row_ok) {
+            float g[32], u[32], dg[32];
+            load32(p.in0 + obase + 32 * c, g);
+            load32(p.in1 + obase + 32 * c, u);
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+              const float dh = __uint_as_float(r0[i]);
+              const float s = 1.0f / (1.0f + __expf(-g[i]));
+              dg[i] = dh * u[i] * s * (1.0f + g[i] * (1.0f - s));
+              v[i] = dh * g[i] * s;
+            }
+            store32(p.out0 + obase + 32 * c, dg);
+            store32(p.out1 + obase + 32 * c, v);
+          }
+        } else {
+          tc_wait_ld();
+          if (row_ok) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r0[i]);
+            store32(p.out0 + obase + 32 * c, v);
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(tempty_bar + 8 * acc_stage);
+      if (++acc_stage == 2) { acc_stage = 0; acc_phase ^= 1u; }
+    }
+  }
+
+  // ---- teardown -----------------------------------------------------------------------------------
+  __syncwarp();
+  if (*abort_flag) {
+    // give copies that are still in flight time to land before the CTA's memory is released
+    const long long t0 = clock64();
+    while (clock64() - t0 < 2000000ll) { }
+    if (tid == 0) atomicExch(&p.stats->error_word, 0x7c05);
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+  }
+}
+
+// ---- host side --------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = (EncodeTiledFn)p;
+  });
+  return fn;
+}
+
+// Row-major bf16 tensor [E, rows, cols] as a 3-D map (cols, rows, E), 64x64 boxes, 128-byte swizzle.
+static etr_status make_map(CUtensorMap* m, const void* base, int cols, int rows, int E) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return ETR_ERR_CUDA;
+  const cuuint64_t dims[3] = {(cuuint64_t)cols, (cuuint64_t)rows, (cuuint64_t)E};
+  const cuuint64_t strides[2] = {(cuuint64_t)cols * 2, (cuuint64_t)cols * 2 * (cuuint64_t)rows};
+  const cuuint32_t box[3] = {64, 64, 1};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  const CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box,
+                        estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                        CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? ETR_OK : ETR_ERR_CUDA;
+}
+
+static uint32_t make_idesc(int a_mn, int b_mn, int n) {
+  uint32_t d = 0;
+  d |= 1u << 4;                     // accumulator fp32
+  d |= 1u << 7;                     // A bf16
+  d |= 1u << 10;                    // B bf16
+  d |= (uint32_t)(a_mn ? 1 : 0) << 15;
+  d |= (uint32_t)(b_mn ? 1 : 0) << 16;
+  d |= (uint32_t)(n >> 3) << 17;
+  d |= (uint32_t)(TC_BM >> 4) << 24;
+  return d;
+}
+
+static int sm_count() {
+  static int n = 0;
+  if (n == 0) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+    if (n <= 0) n = 148;
+  }
+  return n;
+}
+
+template <int BN, int EPI>
+static etr_status tc_launch(const char* name, const CUtensorMap& a0, const CUtensorMap& a1,
+                            const CUtensorMap& b0, const CUtensorMap& b1, TcParams p, int max_tiles,
+                            cudaStream_t st) {
+  constexpr size_t smem = (size_t)TC_STAGES * (2 + BN / 64) * TC_BOX_BYTES + 1024;
+  auto k = tc_grouped_gemm_kernel<BN, EPI>;
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+      return ETR_ERR_CUDA;
+    attr_set = true;
+  }
+  p.idesc = make_idesc(p.a_mn, p.b_mn, BN);
+  const int grid = max_tiles < sm_count() ? (max_tiles < 1 ? 1 : max_tiles) : sm_count();
+  ETR_TIME_BEGIN(name);
+  k<<<grid, TC_THREADS, smem, st>>>(a0, a1, b0, b1, p);
+  ETR_LAUNCH_CHECK();
+  return ETR_OK;
+}
+
 size_t tc_workspace_bytes(const etr_config*) { return 0; }
-bool tc_available() { return false; }
-etr_status tc_ffn_forward(const etr_config*, const etr_route*, const void*, const void*, const void*,
-                          const void*, void*, void*, void*, void*, etr_stats*, void*, cudaStream_t) {
-  return ETR_ERR_UNSUPPORTED;
+bool tc_available() { return true; }
+
+etr_status tc_ffn_forward(const etr_config* c, const etr_route* rt, const void* Xp, const void* W1g,
+                          const void* W1u, const void* W2, void* G, void* U, void* H, void* O,
+                          etr_stats* stats, void*, cudaStream_t st) {
+  const int d = c->d, h = c->h, Cs = c_stride_of(c), E = c->E;
+  CUtensorMap mXp, mW1g, mW1u, mW2, mH;
+  ETR_TRY(make_map(&mXp, Xp, d, Cs, E));
+  ETR_TRY(make_map(&mW1g, W1g, d, h, E));
+  ETR_TRY(make_map(&mW1u, W1u, d, h, E));
+  ETR_TRY(make_map(&mW2, W2, h, d, E));
+  ETR_TRY(make_map(&mH, H, h, Cs, E));
+  const int mt = Cs / TC_BM;
+  {  // G, U, H = SwiGLU(Xp W1g^T, Xp W1u^T)
+    TcParams p = {};
+    p.dual_b = 1; p.M = Cs; p.N = h; p.K = d; p.dyn = TC_DYN_M; p.E = E; p.counts = rt->counts;
+    p.out0 = (__nv_bfloat16*)G; p.out1 = (__nv_bfloat16*)U; p.out2 = (__nv_bfloat16*)H;
+    p.out_bs = (long long)Cs * h; p.ld_out = h; p.stats = stats;
+    ETR_TRY((tc_launch<256, TC_EPI_SWIGLU>("tc_gemm_swiglu", mXp, mXp, mW1g, mW1u, p,
+                                           E * mt * ceil_div(h, 128), st)));
+  }
+  {  // O = H W2^T
+    TcParams p = {};
+    p.M = Cs; p.N = d; p.K = h; p.dyn = TC_DYN_M; p.E = E; p.counts = rt->counts;
+    p.out0 = (__nv_bfloat16*)O; p.out_bs = (long long)Cs * d; p.ld_out = d; p.stats = stats;
+    ETR_TRY((tc_launch<256, TC_EPI_STORE>("tc_gemm_down", mH, mH, mW2, mW2, p, E * mt * ceil_div(d, 256), st)));
+  }
+  return ETR_OK;
 }
-etr_status tc_ffn_backward(const etr_config*, const etr_route*, const void*, const void*, const void*,
-                           const void*, const void*, const void*, const void*, const void*, void*,
-                           void*, void*, void*, void*, void*, etr_stats*, void*, cudaStream_t) {
-  return ETR_ERR_UNSUPPORTED;
+
+etr_status tc_ffn_backward(const etr_config* c, const etr_route* rt, const void* dO, const void* Xp,
+                           const void* G, const void* U, const void* H, const void* W1g,
+                           const void* W1u, const void* W2, void* dG, void* dU, void* dXp, void* dW1g,
+                           void* dW1u, void* dW2, etr_stats* stats, void*, cudaStream_t st) {
+  const int d = c->d, h = c->h, Cs = c_stride_of(c), E = c->E;
+  CUtensorMap mdO, mXp, mH, mdG, mdU, mW1g, mW1u, mW2;
+  ETR_TRY(make_map(&mdO, dO, d, Cs, E));
+  ETR_TRY(make_map(&mXp, Xp, d, Cs, E));
+  ETR_TRY(make_map(&mH, H, h, Cs, E));
+  ETR_TRY(make_map(&mdG, dG, h, Cs, E));
+  ETR_TRY(make_map(&mdU, dU, h, Cs, E));
+  ETR_TRY(make_map(&mW1g, W1g, d, h, E));
+  ETR_TRY(make_map(&mW1u, W1u, d, h, E));
+  ETR_TRY(make_map(&mW2, W2, h, d, E));
+  const int mt = Cs / TC_BM;
+  {  // dH = dO W2 (W2 read with its output index contiguous), then dG, dU
+    TcParams p = {};
+    p.b_mn = 1; p.M = Cs; p.N = h; p.K = d; p.dyn = TC_DYN_M; p.E = E; p.counts = rt->counts;
+    p.out0 = (__nv_bfloat16*)dG; p.out1 = (__nv_bfloat16*)dU;
+    p.in0 = (const __nv_bfloat16*)G; p.in1 = (const __nv_bfloat16*)U;
+    p.out_bs = (long long)Cs * h; p.ld_out = h; p.stats = stats;
+    ETR_TRY((tc_launch<256, TC_EPI_DSWIGLU>("tc_gemm_dswiglu", mdO, mdO, mW2, mW2, p,
+                                            E * mt * ceil_div(h, 256), st)));
+  }
+  {  // dXp = dG W1g + dU W1u: one contraction over 2h
+    TcParams p = {};
+    p.b_mn = 1; p.k1_blocks = ceil_div(h, TC_BK); p.M = Cs; p.N = d; p.K = 2 * h; p.dyn = TC_DYN_M;
+    p.E = E; p.counts = rt->counts;
+    p.out0 = (__nv_bfloat16*)dXp; p.out_bs = (long long)Cs * d; p.ld_out = d; p.stats = stats;
+    ETR_TRY((tc_launch<256, TC_EPI_STORE>("tc_gemm_dxp", mdG, mdU, mW1g, mW1u, p,
+                                          E * mt * ceil_div(d, 256), st)));
+  }
+  {  // dW2 = dO^T H: contraction over the expert's rows, both operands MN-major
+    TcParams p = {};
+    p.a_mn = 1; p.b_mn = 1; p.M = d; p.N = h; p.dyn = TC_DYN_K; p.E = E; p.counts = rt->counts;
+    p.out0 = (__nv_bfloat16*)dW2; p.out_bs = (long long)d * h; p.ld_out = h; p.stats = stats;
+    ETR_TRY((tc_launch<256, TC_EPI_STORE>("tc_gemm_dw2", mdO, mdO, mH, mH, p,
+                                          E * ceil_div(d, TC_BM) * ceil_div(h, 256), st)));
+  }
+  for (int which = 0; which < 2; ++which) {  // dW1g = dG^T Xp, dW1u = dU^T Xp
+    TcParams p = {};
+    p.a_mn = 1; p.b_mn = 1; p.M = h; p.N = d; p.dyn = TC_DYN_K; p.E = E; p.counts = rt->counts;
+    p.out0 = (__nv_bfloat16*)(which ? dW1u : dW1g); p.out_bs = (long long)h * d; p.ld_out = d; p.stats = stats;
+    const CUtensorMap& ma = which ? mdU : mdG;
+    ETR_TRY((tc_launch<256, TC_EPI_STORE>("tc_gemm_dw1", ma, ma, mXp, mXp, p,
+                                          E * ceil_div(h, TC_BM) * ceil_div(d, 256), st)));
+  }
+  return ETR_OK;
 }
+
 }  // namespace etr
