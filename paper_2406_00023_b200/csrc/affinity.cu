@@ -8,6 +8,8 @@
 //   phase 2  s = Z R^T register-tiled (2 tokens x 4 experts per thread, float4 operands),
 //            delta = sqrt(D) s / (||x|| ||R||), batch max through one atomicMax on the
 //            order-preserving integer image (exact and order independent)
+#include <algorithm>
+
 #include "common.cuh"
 
 namespace etr {
@@ -15,14 +17,74 @@ namespace etr {
 constexpr int AFF_TB = 32;        // tokens per CTA
 constexpr int AFF_THREADS = 256;
 
+// Raw 16-byte pieces of a row, converted only when consumed (keeps a batch of loads cheap
+// in registers).
+template <class T> struct Raw16;
+template <> struct Raw16<__nv_bfloat16> {          // 8 elements
+  static constexpr int ELEMS = 8;
+  uint4 w;
+  __device__ void load(const __nv_bfloat16* p) { w = __ldg(reinterpret_cast<const uint4*>(p)); }
+  __device__ void reduce(float& s, float& sq) const {
+    const uint32_t u[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const float a = __uint_as_float(u[i] << 16), b = __uint_as_float(u[i] & 0xffff0000u);
+      s += a; s += b; sq = fmaf(a, a, sq); sq = fmaf(b, b, sq);
+    }
+  }
+};
+template <> struct Raw16<float> {                  // 4 elements
+  static constexpr int ELEMS = 4;
+  float4 w;
+  __device__ void load(const float* p) { w = __ldg(reinterpret_cast<const float4*>(p)); }
+  __device__ void reduce(float& s, float& sq) const {
+    s += w.x; s += w.y; s += w.z; s += w.w;
+    sq = fmaf(w.x, w.x, sq); sq = fmaf(w.y, w.y, sq); sq = fmaf(w.z, w.z, sq); sq = fmaf(w.w, w.w, sq);
+  }
+};
+
+// Whole groups owned by a lane, PPG 16-byte pieces per group.  Loads are issued in batches of
+// 8 independent pieces per lane before any is consumed, so one warp keeps 4 KiB in flight.
+// Out-of-range groups re-read the lane's first group and are discarded (no predicated loads).
+template <class T, int PPG>
+__device__ inline float pool_groups(const T* __restrict__ x, float* __restrict__ zrow, int m, int lane,
+                                    float invD) {
+  constexpr int GB = PPG >= 8 ? 1 : 8 / PPG;      // groups per batch
+  constexpr int D = Raw16<T>::ELEMS * PPG;
+  float sq = 0.f;
+  for (int j0 = lane; j0 < m; j0 += 32 * GB) {
+    Raw16<T> q[GB][PPG];
+#pragma unroll
+    for (int g = 0; g < GB; ++g) {
+      const int j = j0 + 32 * g;
+      const T* src = x + (size_t)(j < m ? j : lane) * D;
+#pragma unroll
+      for (int v = 0; v < PPG; ++v) q[g][v].load(src + v * Raw16<T>::ELEMS);
+    }
+#pragma unroll
+    for (int g = 0; g < GB; ++g) {
+      const int j = j0 + 32 * g;
+      float s = 0.f, q2 = 0.f;
+#pragma unroll
+      for (int v = 0; v < PPG; ++v) q[g][v].reduce(s, q2);
+      if (j < m) { zrow[j] = s * invD; sq += q2; }
+    }
+  }
+  return sq;
+}
+
+// Pools one token row into zrow[0..m) (lane-strided) and returns this lane's share of ||x||^2.
 template <class T>
-__device__ inline void pool_token(const T* __restrict__ x, float* __restrict__ zrow, int d, int D,
-                                  int m, int lane, float& sumsq) {
+__device__ inline float pool_token_partial(const T* __restrict__ x, float* __restrict__ zrow, int d,
+                                           int D, int m, int lane) {
   const float invD = 1.0f / (float)D;
+  constexpr int PE = Raw16<T>::ELEMS;
+  if (D == PE) return pool_groups<T, 1>(x, zrow, m, lane, invD);
+  if (D == 2 * PE) return pool_groups<T, 2>(x, zrow, m, lane, invD);
+  if (D == 4 * PE) return pool_groups<T, 4>(x, zrow, m, lane, invD);
   float sq = 0.f;
   if (D % 8 == 0) {                 // a lane owns whole groups: D/8 vectors each
     const int vpg = D / 8;
-#pragma unroll 4
     for (int j = lane; j < m; j += 32) {
       float s = 0.f;
       for (int v = 0; v < vpg; ++v) {
@@ -52,9 +114,133 @@ __device__ inline void pool_token(const T* __restrict__ x, float* __restrict__ z
       zrow[j] = s * invD;
     }
   }
-  sumsq = warp_sum(sq);
+  return sq;
 }
 
+template <class T>
+__device__ inline void pool_token(const T* __restrict__ x, float* __restrict__ zrow, int d, int D,
+                                  int m, int lane, float& sumsq) {
+  sumsq = warp_sum(pool_token_partial<T>(x, zrow, d, D, m, lane));
+}
+
+// ---- forward, warp-autonomous persistent form (the default) ------------------------------------
+// R stays in shared memory for the life of the CTA; every warp owns a private slice for the
+// pooled rows of TPG tokens and loops on its own: pool TPG tokens (16-byte loads, one pass
+// over X), then s = z R^T with lane = expert (EPL experts per lane, TPG x EPL accumulators,
+// float4 operands: R rows conflict-free, z rows broadcast), then coalesced stores of delta.
+// No block-wide barrier after set-up, so the loads of some warps overlap the FMAs of others.
+template <class T, int EPL, int TPG>
+__global__ void __launch_bounds__(512, 1)
+affinity_fwd_warp_kernel(const T* __restrict__ X, const float* __restrict__ R,
+                         float* __restrict__ delta, float* __restrict__ Z, float* __restrict__ xnorm,
+                         float* __restrict__ rnorm, etr_stats* stats, int Ttok, int d, int D, int E,
+                         int m, int ldm) {
+  extern __shared__ __align__(16) float smem[];
+  constexpr int EROWS = 32 * EPL;
+  const int nw = blockDim.x >> 5;
+  float* Rs = smem;                               // [EROWS][ldm]
+  float* rn = Rs + (size_t)EROWS * ldm;           // [EROWS]
+  float* Zall = rn + EROWS;                       // [nw][TPG][ldm]
+  __shared__ uint32_t red[16];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+  for (int idx = tid; idx < EROWS * ldm; idx += blockDim.x) {
+    const int i = idx / ldm, j = idx - i * ldm;
+    Rs[idx] = (i < E && j < m) ? R[(size_t)i * m + j] : 0.f;
+  }
+  float* zs = Zall + (size_t)warp * TPG * ldm;
+  for (int idx = lane; idx < TPG * ldm; idx += 32) zs[idx] = 0.f;
+  __syncthreads();
+  for (int i = warp; i < EROWS; i += nw) {
+    float s = 0.f;
+    for (int j = lane; j < m; j += 32) s += Rs[i * ldm + j] * Rs[i * ldm + j];
+    s = warp_sum(s);
+    if (lane == 0) {
+      rn[i] = sqrtf(s);
+      if (blockIdx.x == 0 && i < E) rnorm[i] = rn[i];
+    }
+  }
+  __syncthreads();
+
+  const float sqD = sqrtf((float)D);
+  const int mr4 = (m + 3) / 4, rs4 = ldm / 4;
+  const int ngroups = (Ttok + TPG - 1) / TPG;
+  float best = -INFINITY;
+  for (int g = blockIdx.x * nw + warp; g < ngroups; g += gridDim.x * nw) {
+    const int t0 = g * TPG;
+    // pooling, one token at a time (its loads are batched inside); ||x_t|| is parked in the
+    // last pad column of the token's slice row, which the product below never reads
+#pragma unroll 1
+    for (int u = 0; u < TPG; ++u) {
+      const int t = t0 + u;
+      float part = 0.f;
+      if (t < Ttok) {
+        part = pool_token_partial<T>(X + (size_t)t * d, zs + (size_t)u * ldm, d, D, m, lane);
+      } else {
+        for (int j = lane; j < m; j += 32) zs[(size_t)u * ldm + j] = 0.f;
+      }
+      part = warp_sum(part);
+      if (lane == 0) zs[(size_t)u * ldm + ldm - 1] = sqrtf(part);
+    }
+    __syncwarp();
+    if (Z != nullptr) {
+#pragma unroll
+      for (int u = 0; u < TPG; ++u)
+        if (t0 + u < Ttok)
+          for (int j = lane; j < m; j += 32) Z[(size_t)(t0 + u) * m + j] = zs[(size_t)u * ldm + j];
+    }
+    float acc[TPG][EPL];
+#pragma unroll
+    for (int u = 0; u < TPG; ++u)
+#pragma unroll
+      for (int e = 0; e < EPL; ++e) acc[u][e] = 0.f;
+    const float4* r4 = reinterpret_cast<const float4*>(Rs) + (size_t)lane * rs4;
+    const float4* z4 = reinterpret_cast<const float4*>(zs);
+#pragma unroll 2
+    for (int j = 0; j < mr4; ++j) {
+      float4 r[EPL];
+#pragma unroll
+      for (int e = 0; e < EPL; ++e) r[e] = r4[(size_t)(32 * e) * rs4 + j];
+#pragma unroll
+      for (int u = 0; u < TPG; ++u) {
+        const float4 z = z4[(size_t)u * rs4 + j];
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) {
+          acc[u][e] = fmaf(z.x, r[e].x, acc[u][e]); acc[u][e] = fmaf(z.y, r[e].y, acc[u][e]);
+          acc[u][e] = fmaf(z.z, r[e].z, acc[u][e]); acc[u][e] = fmaf(z.w, r[e].w, acc[u][e]);
+        }
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < TPG; ++u) {
+      const int t = t0 + u;
+      if (t >= Ttok) continue;
+#pragma unroll
+      for (int e = 0; e < EPL; ++e) {
+        const int i = lane + 32 * e;
+        if (i < E) {
+          const float den = zs[(size_t)u * ldm + ldm - 1] * rn[i];
+          const float v = den == 0.f ? 0.f : sqD * acc[u][e] / den;
+          delta[(size_t)t * E + i] = v;
+          best = fmaxf(best, v);
+        }
+      }
+      if (lane == 0) xnorm[t] = zs[(size_t)u * ldm + ldm - 1];
+    }
+    __syncwarp();        // the slice is rewritten by the next group's pooling
+  }
+  uint32_t key = best == -INFINITY ? 0u : ordered_key(best);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) key = max(key, __shfl_xor_sync(0xffffffffu, key, o));
+  if (lane == 0) red[warp] = key;
+  __syncthreads();
+  if (tid == 0) {
+    for (int w = 1; w < nw; ++w) key = max(key, red[w]);
+    if (key) atomicMax(&stats->delta_max_key, key);
+  }
+}
+
+// ---- forward, tiled form (fallback for shapes whose R does not fit next to the warp slices) ----
 template <class T>
 __global__ void __launch_bounds__(AFF_THREADS)
 affinity_fwd_kernel(const T* __restrict__ X, const float* __restrict__ R, float* __restrict__ delta,
@@ -281,10 +467,61 @@ static size_t affinity_smem_bytes(int E, int m, int* ldm_out, int* Epad_out) {
   return ((size_t)(Epad + AFF_TB) * ldm + AFF_TB + Epad) * sizeof(float);
 }
 
+static int device_sm_count() {
+  static int n = 0;
+  if (n == 0) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+    if (n <= 0) n = 148;
+  }
+  return n;
+}
+
+template <class T, int EPL, int TPG>
+static etr_status launch_affinity_warp(const etr_config* c, const void* X, const float* R, float* delta,
+                                       float* Z, float* xnorm, float* rnorm, etr_stats* stats,
+                                       cudaStream_t st, bool* done) {
+  const int m = c->d / c->D, ldm = (m + 3) / 4 * 4 + 4;
+  *done = false;
+  for (int nw = 16; nw >= 8; nw /= 2) {
+    const size_t smem = ((size_t)(32 * EPL + nw * TPG) * ldm + 32 * EPL) * sizeof(float);
+    if (smem > 220 * 1024) continue;
+    auto k = affinity_fwd_warp_kernel<T, EPL, TPG>;
+    if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+      return ETR_ERR_CUDA;
+    const int ngroups = ceil_div(c->T, TPG);
+    const int grid = std::min(device_sm_count(), ceil_div(ngroups, nw));
+    ETR_TIME_BEGIN("affinity_fwd_warp_kernel");
+    k<<<grid, nw * 32, smem, st>>>((const T*)X, R, delta, Z, xnorm, rnorm, stats, c->T, c->d, c->D,
+                                   c->E, m, ldm);
+    ETR_LAUNCH_CHECK();
+    *done = true;
+    return ETR_OK;
+  }
+  return ETR_OK;
+}
+
+template <class T>
+static etr_status affinity_forward_warp(const etr_config* c, const void* X, const float* R, float* delta,
+                                        float* Z, float* xnorm, float* rnorm, etr_stats* stats,
+                                        cudaStream_t st, bool* done) {
+  if (c->E <= 32) return launch_affinity_warp<T, 1, 8>(c, X, R, delta, Z, xnorm, rnorm, stats, st, done);
+  if (c->E <= 64) return launch_affinity_warp<T, 2, 8>(c, X, R, delta, Z, xnorm, rnorm, stats, st, done);
+  if (c->E <= 128) return launch_affinity_warp<T, 4, 4>(c, X, R, delta, Z, xnorm, rnorm, stats, st, done);
+  return launch_affinity_warp<T, 8, 2>(c, X, R, delta, Z, xnorm, rnorm, stats, st, done);
+}
+
 etr_status affinity_forward(const etr_config* c, const void* X, const float* R, float* delta,
                             float* Z, float* xnorm, float* rnorm, etr_stats* stats,
                             cudaStream_t st) {
   const int m = c->d / c->D;
+  bool done = false;
+  if (c->dtype == ETR_BF16)
+    ETR_TRY(affinity_forward_warp<__nv_bfloat16>(c, X, R, delta, Z, xnorm, rnorm, stats, st, &done));
+  else
+    ETR_TRY(affinity_forward_warp<float>(c, X, R, delta, Z, xnorm, rnorm, stats, st, &done));
+  if (done) return ETR_OK;
   int ldm, Epad;
   const size_t smem = affinity_smem_bytes(c->E, m, &ldm, &Epad);
   if (smem > 200 * 1024) return ETR_ERR_UNSUPPORTED;

@@ -4,8 +4,9 @@
 //
 //   warp 0      TMA producer: 64x64-element boxes (128-byte swizzle) into a 4-stage ring
 //   warp 1      allocates tensor memory, issues tcgen05.mma (128 x 256 x 16 per instruction)
-//   warps 2-5   epilogue: tcgen05.ld of the fp32 accumulator, fused SwiGLU / its derivative,
-//               bf16 stores; two accumulator stages so it overlaps the next tile's MMAs
+//   warps 2-9   epilogue: tcgen05.ld of the fp32 accumulator, fused SwiGLU / its derivative,
+//               bf16 stores (two warps per 32-lane quarter of tensor memory, half of the
+//               columns each); two accumulator stages so it overlaps the next tile's MMAs
 //
 // Every operand is fetched as 64x64 boxes of its row-major tensor, so one tensor map per
 // tensor serves both uses of it: "K-major" (the contraction index is contiguous in memory)
@@ -28,7 +29,7 @@ namespace etr {
 constexpr int TC_BM = 128;
 constexpr int TC_BK = 64;
 constexpr int TC_STAGES = 4;
-constexpr int TC_THREADS = 192;
+constexpr int TC_THREADS = 320;        // TMA warp, MMA warp, 8 epilogue warps
 constexpr uint32_t TC_BOX_BYTES = 64 * 64 * 2;
 constexpr long long TC_WAIT_LIMIT_CYCLES = 4000000000ll;   // about two seconds
 
@@ -207,7 +208,7 @@ tc_grouped_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_c
   if (tid == 0) {
     abort_flag_s = 0;
     for (int s = 0; s < TC_STAGES; ++s) { mbar_init(full_bar + 8 * s, 1); mbar_init(empty_bar + 8 * s, 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar + 8 * a, 1); mbar_init(tempty_bar + 8 * a, 4); }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar + 8 * a, 1); mbar_init(tempty_bar + 8 * a, 8); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     const int nt = (p.N + N_TILE_COLS - 1) / N_TILE_COLS;
     int acc = 0;
@@ -301,7 +302,9 @@ tc_grouped_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_c
     }
   } else {
     // ---- epilogue warps ---------------------------------------------------------------------------
-    const int q = warp & 3;
+    const int q = warp & 3;                        // quarter of tensor memory this warp may read
+    const int half = (warp - 2) >> 2;              // which half of the tile's columns it handles
+    constexpr int NCH = N_TILE_COLS / 32 / 2;      // 32-column chunks per warp
     const int row_in_tile = 32 * q + lane;
     int e_cur = 0, acc_stage = 0;
     uint32_t acc_phase = 0;
@@ -310,21 +313,31 @@ tc_grouped_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_c
     for (int tile = blockIdx.x; ok && tile_coord(p, tile_prefix, tile, e_cur, N_TILE_COLS, tc); tile += gridDim.x) {
       const int grow = tc.m0 + row_in_tile;
       const bool row_ok = grow < tc.m_lim;
+      const int c_beg = half * NCH;
       const long long obase = (long long)tc.e * p.out_bs + (long long)grow * p.ld_out + tc.n0;
       if (tc.kblocks == 0) {        // nothing to contract: the block of the output is zero
         if (row_ok) {
           float z[32];
 #pragma unroll
           for (int i = 0; i < 32; ++i) z[i] = 0.f;
-          for (int c = 0; c < N_TILE_COLS / 32 && tc.n0 + 32 * c < p.N; ++c) store32(p.out0 + obase + 32 * c, z);
+          for (int c = c_beg; c < c_beg + NCH && tc.n0 + 32 * c < p.N; ++c) store32(p.out0 + obase + 32 * c, z);
         }
         continue;
+      }
+      // SwiGLU derivative: the saved G and U of the first chunk are fetched before the
+      // accumulator is ready, those of chunk c+1 while chunk c is processed
+      uint4 pg[4], pu[4];
+      if (EPI == TC_EPI_DSWIGLU && row_ok && tc.n0 + 32 * c_beg < p.N) {
+        const uint4* sg = reinterpret_cast<const uint4*>(p.in0 + obase + 32 * c_beg);
+        const uint4* su = reinterpret_cast<const uint4*>(p.in1 + obase + 32 * c_beg);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) { pg[i] = sg[i]; pu[i] = su[i]; }
       }
       if (!mbar_wait(tfull_bar + 8 * acc_stage, acc_phase, abort_flag)) { ok = false; break; }
       tc_fence_after();
       const uint32_t taddr = tmem_base + (uint32_t)(acc_stage * 256) + ((uint32_t)(32 * q) << 16);
 #pragma unroll 1
-      for (int c = 0; c < N_TILE_COLS / 32; ++c) {
+      for (int c = c_beg; c < c_beg + NCH; ++c) {
         if (tc.n0 + 32 * c >= p.N) break;
         __syncwarp();               // tcgen05.ld is warp-collective: reconverge after masked stores
         uint32_t r0[32];
@@ -349,17 +362,28 @@ tc_grouped_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_c
             store32(p.out1 + obase + 32 * c, v);
           }
         } else if (EPI == TC_EPI_DSWIGLU) {
+          uint4 cg[4], cu[4];
+#pragma unroll
+          for (int i = 0; i < 4; ++i) { cg[i] = pg[i]; cu[i] = pu[i]; }
+          if (row_ok && c + 1 < c_beg + NCH && tc.n0 + 32 * (c + 1) < p.N) {
+            const uint4* sg = reinterpret_cast<const uint4*>(p.in0 + obase + 32 * (c + 1));
+            const uint4* su = reinterpret_cast<const uint4*>(p.in1 + obase + 32 * (c + 1));
+#pragma unroll
+            for (int i = 0; i < 4; ++i) { pg[i] = sg[i]; pu[i] = su[i]; }
+          }
           tc_wait_ld();
           if (row_ok) {
-            float g[32], u[32], dg[32];
-            load32(p.in0 + obase + 32 * c, g);
-            load32(p.in1 + obase + 32 * c, u);
+            float dg[32];
 #pragma unroll
             for (int i = 0; i < 32; ++i) {
+              const uint32_t wg = reinterpret_cast<const uint32_t*>(cg)[i >> 1];
+              const uint32_t wu = reinterpret_cast<const uint32_t*>(cu)[i >> 1];
+              const float g = (i & 1) ? __uint_as_float(wg & 0xffff0000u) : __uint_as_float(wg << 16);
+              const float u = (i & 1) ? __uint_as_float(wu & 0xffff0000u) : __uint_as_float(wu << 16);
               const float dh = __uint_as_float(r0[i]);
-              const float s = 1.0f / (1.0f + __expf(-g[i]));
-              dg[i] = dh * u[i] * s * (1.0f + g[i] * (1.0f - s));
-              v[i] = dh * g[i] * s;
+              const float sgm = 1.0f / (1.0f + __expf(-g));
+              dg[i] = dh * u * sgm * (1.0f + g * (1.0f - sgm));
+              v[i] = dh * g * sgm;
             }
             store32(p.out0 + obase + 32 * c, dg);
             store32(p.out1 + obase + 32 * c, v);
