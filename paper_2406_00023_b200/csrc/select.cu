@@ -99,14 +99,33 @@ select_token_side_kernel(const float* __restrict__ delta, int32_t* __restrict__ 
   }
 }
 
-// One CTA (1024 threads) per expert.
+// Histogram add with warp aggregation: lanes holding the same digit elect one leader that
+// adds their number.  Affinity keys share their top bits, so the unaggregated form would
+// serialise on a handful of bins.
+__device__ __forceinline__ void hist_add(uint32_t* hist, uint32_t digit, bool active) {
+  const uint32_t amask = __ballot_sync(0xffffffffu, active);
+  if (active) {
+    const uint32_t peers = __match_any_sync(amask, digit);
+    if ((threadIdx.x & 31) == (uint32_t)(__ffs(peers) - 1)) atomicAdd(&hist[digit], (uint32_t)__popc(peers));
+  }
+}
+
+// One CTA (1024 threads) per expert; every thread owns 4 consecutive tokens per sweep.
+constexpr int SEL_KPT = 4;
+constexpr int SEL_SWEEP = 1024 * SEL_KPT;
+
+__device__ __forceinline__ void load_keys(const uint32_t* __restrict__ row, int t0, int T, uint32_t* k) {
+#pragma unroll
+  for (int u = 0; u < SEL_KPT; ++u) k[u] = t0 + u < T ? row[t0 + u] : 0u;
+}
+
 __global__ void __launch_bounds__(1024)
 select_expert_side_kernel(uint32_t* __restrict__ keyT, const etr_stats* __restrict__ stats,
                           int32_t* __restrict__ counts, int32_t* __restrict__ slot_token,
                           float* __restrict__ gate, int T, int C_stride) {
   __shared__ uint32_t hist[256];
   __shared__ uint32_t s_prefix, s_remaining, s_ncand;
-  __shared__ uint32_t warp_gt[32], warp_eq[32];
+  __shared__ uint32_t warp_tot[32], warp_pre[32];
   __shared__ uint32_t base_sel, base_eq;
   const int i = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   uint32_t* row = keyT + (size_t)i * T;
@@ -114,126 +133,190 @@ select_expert_side_kernel(uint32_t* __restrict__ keyT, const etr_stats* __restri
   float* my_gate = gate + (size_t)i * C_stride;
   const int C = stats->C;
 
-  // candidates = keys > 0
-  if (tid == 0) s_ncand = 0;
-  __syncthreads();
-  uint32_t nc = 0;
-  for (int t = tid; t < T; t += 1024) nc += row[t] != 0u;
-  for (int o = 16; o > 0; o >>= 1) nc += __shfl_xor_sync(0xffffffffu, nc, o);
-  if (lane == 0 && nc) atomicAdd(&s_ncand, nc);
-  __syncthreads();
-  const uint32_t n_keep = min((uint32_t)C, s_ncand);
-
-  // radix select: the n_keep-th largest key
-  uint32_t tau = 0, quota = 0;
-  if (n_keep > 0) {
-    if (tid == 0) { s_prefix = 0; s_remaining = n_keep; }
-    for (int pass = 0; pass < 4; ++pass) {
-      const int shift = 24 - 8 * pass;
-      if (tid < 256) hist[tid] = 0;
-      __syncthreads();
-      const uint32_t prefix = s_prefix;
-      const uint32_t pmask = pass == 0 ? 0u : (0xffffffffu << (shift + 8));
-      for (int t = tid; t < T; t += 1024) {
-        const uint32_t kx = row[t];
-        if ((kx & pmask) == prefix) atomicAdd(&hist[(kx >> shift) & 0xff], 1u);
+  // radix select, 4 passes of 8 bits: the n_keep-th largest key; pass 0 also counts candidates
+  uint32_t tau = 0, quota = 0, n_keep = 0;
+  if (tid == 0) { s_prefix = 0; s_ncand = 0; }
+  for (int pass = 0; pass < 4; ++pass) {
+    const int shift = 24 - 8 * pass;
+    if (tid < 256) hist[tid] = 0;
+    __syncthreads();
+    const uint32_t prefix = s_prefix;
+    const uint32_t pmask = pass == 0 ? 0u : (0xffffffffu << (shift + 8));
+    uint32_t nc = 0;
+    uint32_t cur[SEL_KPT], nxt[SEL_KPT];
+    load_keys(row, tid * SEL_KPT, T, cur);
+    for (int c0 = 0; c0 < T; c0 += SEL_SWEEP) {
+      if (c0 + SEL_SWEEP < T) load_keys(row, c0 + SEL_SWEEP + tid * SEL_KPT, T, nxt);   // prefetch
+#pragma unroll
+      for (int u = 0; u < SEL_KPT; ++u) {
+        const uint32_t kx = cur[u];
+        const bool in_range = c0 + tid * SEL_KPT + u < T;
+        nc += (in_range && kx != 0u);
+        hist_add(hist, (kx >> shift) & 0xffu, in_range && (kx & pmask) == prefix);
       }
-      __syncthreads();
-      if (tid == 0) {
-        uint32_t rem = s_remaining;
-        int b = 255;
-        for (; b > 0; --b) {
-          if (hist[b] >= rem) break;
-          rem -= hist[b];
-        }
-        s_prefix = prefix | ((uint32_t)b << shift);
-        s_remaining = rem;        // after the last pass: how many keys == tau are admitted
-      }
-      __syncthreads();
+#pragma unroll
+      for (int u = 0; u < SEL_KPT; ++u) cur[u] = nxt[u];
     }
-    tau = s_prefix;
-    quota = s_remaining;
+    if (pass == 0) {
+      for (int o = 16; o > 0; o >>= 1) nc += __shfl_xor_sync(0xffffffffu, nc, o);
+      if (lane == 0 && nc) atomicAdd(&s_ncand, nc);
+    }
+    __syncthreads();
+    if (pass == 0) n_keep = min((uint32_t)C, s_ncand);
+    if (n_keep == 0) break;                       // uniform across the CTA
+    if (tid == 0) {
+      uint32_t rem = pass == 0 ? n_keep : s_remaining;
+      int b = 255;
+      for (; b > 0; --b) {
+        if (hist[b] >= rem) break;
+        rem -= hist[b];
+      }
+      s_prefix = prefix | ((uint32_t)b << shift);
+      s_remaining = rem;        // after the last pass: how many keys == tau are admitted
+    }
+    __syncthreads();
   }
+  if (n_keep > 0) { tau = s_prefix; quota = s_remaining; }
 
   // slot assignment in ascending token order
   if (tid == 0) { base_sel = 0; base_eq = 0; }
   __syncthreads();
-  for (int c0 = 0; c0 < T; c0 += 1024) {
-    const int t = c0 + tid;
-    const uint32_t kx = t < T ? row[t] : 0u;
-    const bool gt = n_keep > 0 && kx > tau;
-    const bool eq = n_keep > 0 && kx == tau && kx != 0u;
-    const uint32_t b_gt = __ballot_sync(0xffffffffu, gt), b_eq = __ballot_sync(0xffffffffu, eq);
-    if (lane == 0) { warp_gt[warp] = __popc(b_gt); warp_eq[warp] = __popc(b_eq); }
+  uint32_t cur[SEL_KPT], nxt[SEL_KPT];
+  load_keys(row, tid * SEL_KPT, T, cur);
+  for (int c0 = 0; c0 < T; c0 += SEL_SWEEP) {
+    if (c0 + SEL_SWEEP < T) load_keys(row, c0 + SEL_SWEEP + tid * SEL_KPT, T, nxt);
+    const int tb = c0 + tid * SEL_KPT;
+    uint32_t ngt = 0, neq = 0;
+#pragma unroll
+    for (int u = 0; u < SEL_KPT; ++u) {
+      const bool live = n_keep > 0 && tb + u < T && cur[u] != 0u;
+      ngt += live && cur[u] > tau;
+      neq += live && cur[u] == tau;
+    }
+    // block-wide exclusive scan of (ngt, neq), packed 16 bits apart (each < 2^13 per sweep)
+    const uint32_t mine = ngt | (neq << 16);
+    uint32_t inc = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const uint32_t y = __shfl_up_sync(0xffffffffu, inc, o);
+      if (lane >= o) inc += y;
+    }
+    if (lane == 31) warp_tot[warp] = inc;
     __syncthreads();
-    uint32_t pre_gt = 0, pre_eq = 0, tot_gt = 0, tot_eq = 0;
-    for (int w = 0; w < 32; ++w) {
-      const uint32_t g = warp_gt[w], e = warp_eq[w];
-      if (w < warp) { pre_gt += g; pre_eq += e; }
-      tot_gt += g; tot_eq += e;
+    if (warp == 0) {
+      const uint32_t wt = warp_tot[lane];
+      uint32_t winc = wt;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t y = __shfl_up_sync(0xffffffffu, winc, o);
+        if (lane >= o) winc += y;
+      }
+      warp_pre[lane] = winc - wt;
+      if (lane == 31) warp_tot[0] = winc;          // sweep totals
     }
-    const uint32_t lt_mask = (1u << lane) - 1u;
-    const uint32_t eq_rank = base_eq + pre_eq + __popc(b_eq & lt_mask);   // rank among key == tau
-    const uint32_t gt_rank = pre_gt + __popc(b_gt & lt_mask);             // within this chunk
-    const uint32_t eq_before_chunk = min(base_eq, quota);
-    const uint32_t eq_adm_before_me = min(eq_rank, quota) - eq_before_chunk;
-    const bool sel = gt || (eq && eq_rank < quota);
-    int pos = -1;
-    if (sel) {
-      pos = (int)(base_sel + gt_rank + eq_adm_before_me);
-      my_slot[pos] = t;
-      my_gate[pos] = key_to_float(kx);
+    __syncthreads();
+    const uint32_t excl = warp_pre[warp] + inc - mine;
+    const uint32_t tot = warp_tot[0];
+    uint32_t gt_before = excl & 0xffffu, eq_rank = base_eq + (excl >> 16);
+    const uint32_t eq_before_sweep = min(base_eq, quota);
+    const uint32_t bs = base_sel;
+#pragma unroll
+    for (int u = 0; u < SEL_KPT; ++u) {
+      const int t = tb + u;
+      const uint32_t kx = cur[u];
+      const bool live = n_keep > 0 && t < T && kx != 0u;
+      const bool gt = live && kx > tau, eq = live && kx == tau;
+      int pos = -1;
+      if (gt || (eq && eq_rank < quota)) {
+        pos = (int)(bs + gt_before + (min(eq_rank, quota) - eq_before_sweep));
+        my_slot[pos] = t;
+        my_gate[pos] = key_to_float(kx);
+      }
+      if (t < T) row[t] = (uint32_t)pos;
+      gt_before += gt;
+      eq_rank += eq;
     }
-    if (t < T) row[t] = (uint32_t)pos;
     __syncthreads();
     if (tid == 0) {
+      const uint32_t tot_gt = tot & 0xffffu, tot_eq = tot >> 16;
       const uint32_t eq_after = min(base_eq + tot_eq, quota);
-      base_sel += tot_gt + (eq_after - eq_before_chunk);
+      base_sel += tot_gt + (eq_after - eq_before_sweep);
       base_eq += tot_eq;
     }
     __syncthreads();
+#pragma unroll
+    for (int u = 0; u < SEL_KPT; ++u) cur[u] = nxt[u];
   }
   for (int p = (int)n_keep + tid; p < C_stride; p += 1024) { my_slot[p] = -1; my_gate[p] = 0.f; }
   if (tid == 0) counts[i] = (int)n_keep;
 }
 
-// rows per token (tok_ptr[t+1] = count), plus the number of unrouted tokens
+// Token-major CSR in three small kernels without a long serial scan:
+//   count  per-token row counts, exclusive scan inside each 256-token block (left in
+//          tok_ptr[t+1]), block totals to scratch
+//   scan   exclusive scan of the block totals (one CTA; T/256 values)
+//   fill   tok_row from the position matrix, final tok_ptr
 __global__ void __launch_bounds__(256)
-csr_count_kernel(const int32_t* __restrict__ posT, int32_t* __restrict__ tok_ptr, etr_stats* stats,
-                 int T, int E) {
-  const int t = blockIdx.x * 256 + threadIdx.x;
+csr_count_kernel(const int32_t* __restrict__ posT, int32_t* __restrict__ tok_ptr,
+                 int32_t* __restrict__ block_total, etr_stats* stats, int T, int E) {
+  __shared__ int wsum[8];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int t = blockIdx.x * 256 + tid;
   int n = 0;
-  if (t < T) {
+  if (t < T)
     for (int i = 0; i < E; ++i) n += posT[(size_t)i * T + t] >= 0;
-    tok_ptr[t + 1] = n;
-  }
   const uint32_t un = __ballot_sync(0xffffffffu, t < T && n == 0);
-  if ((threadIdx.x & 31) == 0 && un) atomicAdd(&stats->unrouted, __popc(un));
+  if (lane == 0 && un) atomicAdd(&stats->unrouted, __popc(un));
+  int inc = n;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int y = __shfl_up_sync(0xffffffffu, inc, o);
+    if (lane >= o) inc += y;
+  }
+  if (lane == 31) wsum[warp] = inc;
+  __syncthreads();
+  int pre = 0, tot = 0;
+#pragma unroll
+  for (int w = 0; w < 8; ++w) { if (w < warp) pre += wsum[w]; tot += wsum[w]; }
+  if (t < T) tok_ptr[t + 1] = pre + inc - n;          // exclusive, within the block
+  if (tid == 0) block_total[blockIdx.x] = tot;
 }
 
-// in-place inclusive scan of tok_ptr[1..T] (single CTA), i.e. exclusive offsets in tok_ptr[0..T]
 __global__ void __launch_bounds__(1024)
-csr_scan_kernel(int32_t* __restrict__ tok_ptr, etr_stats* stats, int T, int n_cand) {
-  __shared__ int wsum[32];
+csr_scan_kernel(int32_t* __restrict__ block_total, int32_t* __restrict__ tok_ptr, etr_stats* stats,
+                int nblocks, int n_cand) {
+  __shared__ int wsum[32], wpre[32];
   __shared__ int carry;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   if (tid == 0) { carry = 0; tok_ptr[0] = 0; }
   __syncthreads();
-  for (int c0 = 0; c0 < T; c0 += 1024) {
-    const int t = c0 + tid;
-    const int v = t < T ? tok_ptr[t + 1] : 0;
+  for (int c0 = 0; c0 < nblocks; c0 += 1024) {
+    const int b = c0 + tid;
+    const int v = b < nblocks ? block_total[b] : 0;
     int inc = v;
+#pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
       const int y = __shfl_up_sync(0xffffffffu, inc, o);
       if (lane >= o) inc += y;
     }
     if (lane == 31) wsum[warp] = inc;
     __syncthreads();
-    int pre = carry;
-    for (int w = 0; w < warp; ++w) pre += wsum[w];
-    if (t < T) tok_ptr[t + 1] = pre + inc;
+    if (warp == 0) {
+      const int wt = wsum[lane];
+      int winc = wt;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int y = __shfl_up_sync(0xffffffffu, winc, o);
+        if (lane >= o) winc += y;
+      }
+      wpre[lane] = winc - wt;
+      if (lane == 31) wsum[0] = winc;
+    }
     __syncthreads();
-    if (tid == 1023) carry = pre + inc;
+    if (b < nblocks) block_total[b] = carry + wpre[warp] + inc - v;     // exclusive block offset
+    const int total = wsum[0];
+    __syncthreads();
+    if (tid == 0) carry += total;
     __syncthreads();
   }
   if (tid == 0) {
@@ -243,18 +326,24 @@ csr_scan_kernel(int32_t* __restrict__ tok_ptr, etr_stats* stats, int T, int n_ca
 }
 
 __global__ void __launch_bounds__(256)
-csr_fill_kernel(const int32_t* __restrict__ posT, const int32_t* __restrict__ tok_ptr,
-                int32_t* __restrict__ tok_row, int T, int E, int C_stride) {
+csr_fill_kernel(const int32_t* __restrict__ posT, const int32_t* __restrict__ block_offset,
+                int32_t* __restrict__ tok_ptr, int32_t* __restrict__ tok_row, int T, int E,
+                int C_stride) {
   const int t = blockIdx.x * 256 + threadIdx.x;
   if (t >= T) return;
-  int q = tok_ptr[t];
+  int q = block_offset[blockIdx.x] + tok_ptr[t + 1];
   for (int i = 0; i < E; ++i) {
     const int pos = posT[(size_t)i * T + t];
     if (pos >= 0) tok_row[q++] = i * C_stride + pos;
   }
+  tok_ptr[t + 1] = q;
 }
 
-size_t select_workspace_bytes(const etr_config* c) { return (size_t)c->T * c->E * sizeof(uint32_t); }
+// key / position matrix [E][T], then one int per 256-token block
+static size_t select_keys_bytes(const etr_config* c) { return align_up((size_t)c->T * c->E * sizeof(uint32_t), 256); }
+size_t select_workspace_bytes(const etr_config* c) {
+  return select_keys_bytes(c) + align_up((size_t)ceil_div(c->T, 256) * sizeof(int32_t), 256);
+}
 
 int resolve_mode(const etr_config* c) {
   if (c->mode == ETR_MODE_TCR || c->mode == ETR_MODE_ECR) return c->mode;
@@ -276,15 +365,17 @@ etr_status select_forward(const etr_config* c, const float* delta, etr_stats* st
                                                    c->T, p.C_stride);
   ETR_LAUNCH_CHECK();
   ETR_TIME_BEGIN("csr_count_kernel");
-  csr_count_kernel<<<ceil_div(c->T, 256), 256, 0, st>>>((const int32_t*)keyT, rt->tok_ptr, stats, c->T, c->E);
+  int32_t* block_total = reinterpret_cast<int32_t*>(reinterpret_cast<char*>(ws) + select_keys_bytes(c));
+  const int nblocks = ceil_div(c->T, 256);
+  csr_count_kernel<<<nblocks, 256, 0, st>>>((const int32_t*)keyT, rt->tok_ptr, block_total, stats, c->T, c->E);
   ETR_LAUNCH_CHECK();
   const int n_cand = p.mode == ETR_MODE_TCR ? c->T * c->k : c->T * c->E;
   ETR_TIME_BEGIN("csr_scan_kernel");
-  csr_scan_kernel<<<1, 1024, 0, st>>>(rt->tok_ptr, stats, c->T, n_cand);
+  csr_scan_kernel<<<1, 1024, 0, st>>>(block_total, rt->tok_ptr, stats, nblocks, n_cand);
   ETR_LAUNCH_CHECK();
   ETR_TIME_BEGIN("csr_fill_kernel");
-  csr_fill_kernel<<<ceil_div(c->T, 256), 256, 0, st>>>((const int32_t*)keyT, rt->tok_ptr, rt->tok_row,
-                                                       c->T, c->E, p.C_stride);
+  csr_fill_kernel<<<nblocks, 256, 0, st>>>((const int32_t*)keyT, block_total, rt->tok_ptr, rt->tok_row,
+                                           c->T, c->E, p.C_stride);
   ETR_LAUNCH_CHECK();
   return ETR_OK;
 }
@@ -298,7 +389,8 @@ etr_status select_forward(const etr_config* c, const float* delta, etr_stats* st
 // process exits.
 namespace etr {
 
-constexpr size_t SELECT_STATIC_MAX_BYTES = ETR_SELECT_STATIC_MAX_ENTRIES * sizeof(uint32_t);
+// the keys, plus the per-block scan scratch (one int per 256 tokens; T <= 4 Mi)
+constexpr size_t SELECT_STATIC_MAX_BYTES = ETR_SELECT_STATIC_MAX_ENTRIES * sizeof(uint32_t) + (64u << 10) + 512u;
 static __device__ __align__(256) unsigned char g_select_scratch[SELECT_STATIC_MAX_BYTES];
 
 // In host code `g_select_scratch` is only a handle for the runtime's symbol table, not a
@@ -330,7 +422,9 @@ extern "C" etr_status etr_select_static(const etr_config* cfg, const float* delt
       !route->tok_row)
     return ETR_ERR_ARG;
   if (!aligned16(delta) || !aligned16(stats)) return ETR_ERR_ALIGN;
-  if (select_workspace_bytes(cfg) > SELECT_STATIC_MAX_BYTES) return ETR_ERR_WORKSPACE;
+  if ((unsigned long long)cfg->T * (unsigned long long)cfg->E > ETR_SELECT_STATIC_MAX_ENTRIES ||
+      select_workspace_bytes(cfg) > SELECT_STATIC_MAX_BYTES)
+    return ETR_ERR_WORKSPACE;
   void* scratch = nullptr;
   ETR_TRY(select_scratch_address(&scratch));
   return select_forward(cfg, delta, stats, route, scratch, (cudaStream_t)stream);
