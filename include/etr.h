@@ -247,7 +247,9 @@ etr_status etr_layer_backward(const etr_config* cfg, const void* X, const float*
 /* One training step from HOST activations: copies X_host and dY_host (host, ideally pinned)
  * to buf->X_dev / dY_dev, runs forward and backward, copies Y and dX back to Y_host and
  * dX_host (host), and synchronises the stream.  Parameters and their gradients stay on
- * the device.  buf must have been bound with host staging. */
+ * the device.  buf must have been bound with host staging.  The copy of dY overlaps the
+ * forward pass and the copy of Y overlaps the backward pass, on two side streams the
+ * library creates once per device (host-side objects; still no device allocation). */
 etr_status etr_layer_step_host(const etr_config* cfg, const void* X_host, const void* dY_host,
                                const float* R, const void* W1g, const void* W1u, const void* W2,
                                const etr_buffers* buf, void* Y_host, void* dX_host,

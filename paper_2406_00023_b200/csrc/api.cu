@@ -301,6 +301,31 @@ etr_status etr_layer_backward(const etr_config* c, const void* X, const float* R
                           b->ws, stream);
 }
 
+// Side streams and events for the host-buffer step (host-side objects, created once per device).
+struct HostStepCtx { cudaStream_t up = nullptr, down = nullptr; cudaEvent_t dy_ready = nullptr, fwd_done = nullptr, y_done = nullptr, start = nullptr; };
+static std::mutex g_ctx_mu;
+static HostStepCtx g_ctx[64];
+
+static etr_status host_step_ctx(HostStepCtx** out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return ETR_ERR_CUDA;
+  std::lock_guard<std::mutex> lk(g_ctx_mu);
+  HostStepCtx& c = g_ctx[dev];
+  if (c.up == nullptr) {
+    if (cudaStreamCreateWithFlags(&c.up, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaStreamCreateWithFlags(&c.down, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaEventCreateWithFlags(&c.dy_ready, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&c.fwd_done, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&c.y_done, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&c.start, cudaEventDisableTiming) != cudaSuccess)
+      return ETR_ERR_CUDA;
+  }
+  *out = &c;
+  return ETR_OK;
+}
+
+#define ETR_CUDA(expr) do { if ((expr) != cudaSuccess) return ETR_ERR_CUDA; } while (0)
+
 etr_status etr_layer_step_host(const etr_config* c, const void* X_host, const void* dY_host,
                                const float* R, const void* W1g, const void* W1u, const void* W2,
                                const etr_buffers* b, void* Y_host, void* dX_host, float* dR,
@@ -310,15 +335,27 @@ etr_status etr_layer_step_host(const etr_config* c, const void* X_host, const vo
   ETR_TRY(etr_validate(c));
   if (!b->X_dev || !b->dY_dev || !b->Y_dev || !b->dX_dev) return ETR_ERR_WORKSPACE;
   cudaStream_t st = (cudaStream_t)stream;
+  HostStepCtx* hc = nullptr;
+  ETR_TRY(host_step_ctx(&hc));
   const size_t bytes = (size_t)c->T * c->d * elem_bytes(c->dtype);
-  if (cudaMemcpyAsync(b->X_dev, X_host, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return ETR_ERR_CUDA;
-  if (cudaMemcpyAsync(b->dY_dev, dY_host, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return ETR_ERR_CUDA;
+  // dY goes up on a side stream while X is copied and the forward pass runs; Y comes down on
+  // another side stream while the backward pass runs.
+  ETR_CUDA(cudaEventRecord(hc->start, st));
+  ETR_CUDA(cudaStreamWaitEvent(hc->up, hc->start, 0));
+  ETR_CUDA(cudaMemcpyAsync(b->X_dev, X_host, bytes, cudaMemcpyHostToDevice, st));
+  ETR_CUDA(cudaMemcpyAsync(b->dY_dev, dY_host, bytes, cudaMemcpyHostToDevice, hc->up));
+  ETR_CUDA(cudaEventRecord(hc->dy_ready, hc->up));
   ETR_TRY(etr_layer_forward(c, b->X_dev, R, W1g, W1u, W2, b, b->Y_dev, stream));
-  if (cudaMemcpyAsync(Y_host, b->Y_dev, bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return ETR_ERR_CUDA;
+  ETR_CUDA(cudaEventRecord(hc->fwd_done, st));
+  ETR_CUDA(cudaStreamWaitEvent(hc->down, hc->fwd_done, 0));
+  ETR_CUDA(cudaMemcpyAsync(Y_host, b->Y_dev, bytes, cudaMemcpyDeviceToHost, hc->down));
+  ETR_CUDA(cudaEventRecord(hc->y_done, hc->down));
+  ETR_CUDA(cudaStreamWaitEvent(st, hc->dy_ready, 0));
   ETR_TRY(etr_layer_backward(c, b->X_dev, R, W1g, W1u, W2, b->dY_dev, b, b->dX_dev, dR, dW1g, dW1u,
                              dW2, stream));
-  if (cudaMemcpyAsync(dX_host, b->dX_dev, bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return ETR_ERR_CUDA;
-  if (cudaStreamSynchronize(st) != cudaSuccess) return ETR_ERR_CUDA;
+  ETR_CUDA(cudaMemcpyAsync(dX_host, b->dX_dev, bytes, cudaMemcpyDeviceToHost, st));
+  ETR_CUDA(cudaStreamWaitEvent(st, hc->y_done, 0));
+  ETR_CUDA(cudaStreamSynchronize(st));
   return ETR_OK;
 }
 

@@ -29,26 +29,36 @@ dispatch_kernel(const T* __restrict__ X, const int32_t* __restrict__ counts,
 }
 
 // Y[t,:] = sum_{r in rows(t)} gate[r] O[r,:]   (gate == nullptr: plain sum, used for dX).
-// One thread per 8 consecutive elements of a token.
-template <class T>
+// One thread per NV groups of 8 consecutive elements of a token, half a row apart, so every
+// row contributes NV independent 16-byte loads per thread.
+template <class T, int NV>
 __global__ void __launch_bounds__(256)
 combine_kernel(const T* __restrict__ O, const float* __restrict__ gate,
                const int32_t* __restrict__ tok_ptr, const int32_t* __restrict__ tok_row,
                T* __restrict__ Y, int Ttok, int d) {
-  const int vpt = d / 8;
+  const int vpt = d / 8 / NV;                       // threads per token
   const long long idx = (long long)blockIdx.x * 256 + threadIdx.x;
   if (idx >= (long long)Ttok * vpt) return;
   const int t = (int)(idx / vpt), v = (int)(idx - (long long)t * vpt);
-  float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+  float acc[NV][8];
+#pragma unroll
+  for (int u = 0; u < NV; ++u)
+#pragma unroll
+    for (int e = 0; e < 8; ++e) acc[u][e] = 0.f;
   const int beg = tok_ptr[t], end = tok_ptr[t + 1];
   for (int q = beg; q < end; ++q) {
     const int r = tok_row[q];
     const float g = gate ? gate[r] : 1.0f;
-    Vec8<T> o = Vec8<T>::load(O + (size_t)r * d + v * 8);
+    Vec8<T> o[NV];
 #pragma unroll
-    for (int e = 0; e < 8; ++e) acc[e] = fmaf(g, o.v[e], acc[e]);
+    for (int u = 0; u < NV; ++u) o[u] = Vec8<T>::load(O + (size_t)r * d + (size_t)(v + u * vpt) * 8);
+#pragma unroll
+    for (int u = 0; u < NV; ++u)
+#pragma unroll
+      for (int e = 0; e < 8; ++e) acc[u][e] = fmaf(g, o[u].v[e], acc[u][e]);
   }
-  Vec8<T>::store(Y + (size_t)t * d + v * 8, acc);
+#pragma unroll
+  for (int u = 0; u < NV; ++u) Vec8<T>::store(Y + (size_t)t * d + (size_t)(v + u * vpt) * 8, acc[u]);
 }
 
 // dO[r,:] = gate[r] dY[t(r),:], dgate[r] = <dY[t(r),:], O[r,:]>; pad rows zero.  Warp per row.
@@ -99,10 +109,17 @@ static etr_status permute_launch(int which, const etr_config* c, const etr_route
       break;
     case 1:
     case 3: {
-      const long long n = (long long)c->T * (c->d / 8);
+      const float* g = which == 1 ? rt->gate : nullptr;
       ETR_TIME_BEGIN("combine_kernel");
-      combine_kernel<T><<<(unsigned)((n + 255) / 256), 256, 0, st>>>(
-          (const T*)a, which == 1 ? rt->gate : nullptr, rt->tok_ptr, rt->tok_row, (T*)out, c->T, c->d);
+      if (c->d % 32 == 0) {
+        const long long n = (long long)c->T * (c->d / 32);
+        combine_kernel<T, 4><<<(unsigned)((n + 255) / 256), 256, 0, st>>>((const T*)a, g, rt->tok_ptr,
+                                                                         rt->tok_row, (T*)out, c->T, c->d);
+      } else {
+        const long long n = (long long)c->T * (c->d / 8);
+        combine_kernel<T, 1><<<(unsigned)((n + 255) / 256), 256, 0, st>>>((const T*)a, g, rt->tok_ptr,
+                                                                         rt->tok_row, (T*)out, c->T, c->d);
+      }
       break;
     }
     case 2:
