@@ -62,6 +62,7 @@ def algorithmic_work(w, rows, kernel, unrouted=0):
     T_routed = T - unrouted
     table = {
         "affinity_fwd_kernel": (T * d * b + T * E * 4 + T * m * 4 + T * 4, "bytes"),
+        "affinity_fwd_warp_kernel": (T * d * b + T * E * 4 + T * m * 4 + T * 4, "bytes"),
         "select_token_side_kernel": (2 * T * E * 4, "bytes"),
         "select_expert_side_kernel": (T * E * 4 + rows * 8, "bytes"),
         "csr_count_kernel": (T * E * 4, "bytes"),
@@ -83,6 +84,20 @@ def algorithmic_work(w, rows, kernel, unrouted=0):
         "tc_gemm_dw1": (4 * rows * d * h, "flops"),
     }
     return table.get(kernel, (0, "bytes"))
+
+
+def aggregate_over_ranks(values, world, device=None):
+    """Element-wise max of per-rank timings over all ranks (the slowest rank sets the pace)."""
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if world > 1:
+        import torch.distributed as dist
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t]
+
+
+def whole_job_tokens_per_sec(world, tokens_per_rank, ms_per_step):
+    """Replicas process world * tokens_per_rank tokens per step (weak scaling)."""
+    return world * tokens_per_rank / (ms_per_step * 1e-3)
 
 
 class ClockSampler:
@@ -181,6 +196,7 @@ def main():
     ap.add_argument("--gemm", default="auto", choices=["auto", "simt", "tcgen05"])
     ap.add_argument("--cpu-tokens", type=int, default=128, help="tokens in the CPU-oracle sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--set", default="", help="override workload fields, e.g. T=32768,h=512 (profiling cases)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -188,6 +204,10 @@ def main():
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
     w0 = gw.WORKLOADS[args.workload]
+    if args.set:
+        kv = dict(item.split("=") for item in args.set.split(","))
+        w0 = replace(w0, name=w0.name + "+" + args.set,
+                     **{k: type(getattr(w0, k))(v) for k, v in kv.items()})
     config = {"workload": f"{w0.name} (config {w0.config_id}): T={w0.T} d={w0.d} D={w0.D} E={w0.E} "
                           f"k={w0.k} h={w0.h} cf={w0.cf} {mode_name(w0)} adaptive={int(w0.adaptive)} "
                           f"x={w0.x_kind}",
@@ -284,10 +304,7 @@ def main():
     torch.cuda.synchronize()
     e2e_ms = (time.perf_counter() - t0) * 1e3 / e2e_steps
 
-    t = torch.tensor([ms_total, e2e_ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_total, e2e_ms = float(t[0]), float(t[1])
+    ms_total, e2e_ms = aggregate_over_ranks([ms_total, e2e_ms], world, dev)
     ms_step = ms_total / args.steps
 
     # per-kernel table and the roofline of the dominant kernel
@@ -332,12 +349,12 @@ def main():
                     "traffic": NCU_TRAFFIC_BYTES.get(top["kernel"]),
                     "peak_source": peaks["source"] + (" (sustained)" if top["bound"] == "tensor" else "")}
 
-    out = {"metric": METRIC, "value": world * w.T / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world,
+    out = {"metric": METRIC, "value": whole_job_tokens_per_sec(world, w.T, ms_step), "unit": UNIT, "n_gpus": world,
            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_step,
            "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
            "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic", "config": config,
            "clocks": clocks, "gpu_launches": int(launches),
-           "e2e": {"value": world * w.T / (e2e_ms * 1e-3), "unit": UNIT,
+           "e2e": {"value": whole_job_tokens_per_sec(world, w.T, e2e_ms), "unit": UNIT,
                    "h2d_bytes_per_step": int(2 * Xh.numel() * Xh.element_size()),
                    "d2h_bytes_per_step": int(2 * Xh.numel() * Xh.element_size()),
                    "ms_per_step": e2e_ms},
