@@ -123,6 +123,166 @@ __device__ inline void pool_token(const T* __restrict__ x, float* __restrict__ z
   sumsq = warp_sum(pool_token_partial<T>(x, zrow, d, D, m, lane));
 }
 
+// ---- forward, split form (the default when the caller keeps Z) -----------------------------------
+// Kernel 1 streams X once and leaves the pooled rows Z and ||x_t||: one warp per token, the
+// row dealt to the lanes as consecutive 16-byte pieces (each load instruction moves 512
+// contiguous bytes), 8 independent loads per lane in flight; a group of D elements is PPG
+// adjacent pieces whose partial sums meet through xor-shuffles.  Pure HBM streaming.
+template <class T, int PPG>
+__global__ void __launch_bounds__(256)
+grap_pool_kernel(const T* __restrict__ X, float* __restrict__ Z, float* __restrict__ xnorm, int Ttok,
+                 int d, int D, int m) {
+  constexpr int PE = Raw16<T>::ELEMS;
+  constexpr int BATCH = 8;
+  const int lane = threadIdx.x & 31;
+  const int t = blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (t >= Ttok) return;
+  const T* x = X + (size_t)t * d;
+  float* zrow = Z + (size_t)t * m;
+  float sq = 0.f;
+  if (PPG > 0) {
+    const float invD = 1.0f / (float)D;
+    const int npieces = m * PPG;
+    for (int p0 = 0; p0 < npieces; p0 += 32 * BATCH) {
+      Raw16<T> q[BATCH];
+#pragma unroll
+      for (int g = 0; g < BATCH; ++g) {
+        const int p = p0 + 32 * g + lane;
+        q[g].load(x + (size_t)(p < npieces ? p : lane) * PE);
+      }
+#pragma unroll
+      for (int g = 0; g < BATCH; ++g) {
+        const int p = p0 + 32 * g + lane;
+        float s = 0.f, q2 = 0.f;
+        q[g].reduce(s, q2);
+#pragma unroll
+        for (int o = 1; o < (PPG > 0 ? PPG : 1); o <<= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+        if (p < npieces) {
+          sq += q2;
+          if ((lane & ((PPG > 0 ? PPG : 1) - 1)) == 0) zrow[p / (PPG > 0 ? PPG : 1)] = s * invD;
+        }
+      }
+    }
+  } else {
+    sq = pool_token_partial<T>(x, zrow, d, D, m, lane);     // any group size
+  }
+  sq = warp_sum(sq);
+  if (lane == 0) xnorm[t] = sqrtf(sq);
+}
+
+// Kernel 2: s = Z R^T and the cosine.  R stays in shared memory; each warp copies the pooled
+// rows of TPG tokens into its slice (coalesced float4), then lane = expert, TPG x EPL
+// accumulators, float4 operands (R rows conflict-free, z rows broadcast).  Bound by the fp32
+// FMA rate (2 m E flop per token against 4 m bytes), not by HBM.
+template <int EPL, int TPG>
+__global__ void __launch_bounds__(512, 1)
+affinity_score_kernel(const float* __restrict__ Z, const float* __restrict__ xnorm,
+                      const float* __restrict__ R, float* __restrict__ delta,
+                      float* __restrict__ rnorm, etr_stats* stats, int Ttok, int D, int E, int m,
+                      int ldm) {
+  extern __shared__ __align__(16) float smem[];
+  constexpr int EROWS = 32 * EPL;
+  const int nw = blockDim.x >> 5;
+  float* Rs = smem;                               // [EROWS][ldm]
+  float* rn = Rs + (size_t)EROWS * ldm;           // [EROWS]
+  float* Zall = rn + EROWS;                       // [nw][TPG][ldm]
+  __shared__ uint32_t red[16];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+  for (int idx = tid; idx < EROWS * ldm; idx += blockDim.x) {
+    const int i = idx / ldm, j = idx - i * ldm;
+    Rs[idx] = (i < E && j < m) ? R[(size_t)i * m + j] : 0.f;
+  }
+  float* zs = Zall + (size_t)warp * TPG * ldm;
+  for (int idx = lane; idx < TPG * ldm; idx += 32) zs[idx] = 0.f;
+  __syncthreads();
+  for (int i = warp; i < EROWS; i += nw) {
+    float s = 0.f;
+    for (int j = lane; j < m; j += 32) s += Rs[i * ldm + j] * Rs[i * ldm + j];
+    s = warp_sum(s);
+    if (lane == 0) {
+      rn[i] = sqrtf(s);
+      if (blockIdx.x == 0 && i < E) rnorm[i] = rn[i];
+    }
+  }
+  __syncthreads();
+
+  const float sqD = sqrtf((float)D);
+  const int mr4 = (m + 3) / 4, rs4 = ldm / 4;
+  const bool vec_ok = (m & 3) == 0;
+  const int ngroups = (Ttok + TPG - 1) / TPG;
+  float best = -INFINITY;
+  for (int g = blockIdx.x * nw + warp; g < ngroups; g += gridDim.x * nw) {
+    const int t0 = g * TPG;
+    float xn[TPG];
+#pragma unroll
+    for (int u = 0; u < TPG; ++u) {
+      const int t = t0 + u;
+      xn[u] = t < Ttok ? xnorm[t] : 0.f;
+      float* zr = zs + (size_t)u * ldm;
+      if (t < Ttok) {
+        const float* src = Z + (size_t)t * m;
+        if (vec_ok) {
+          for (int j = lane; j < m / 4; j += 32)
+            reinterpret_cast<float4*>(zr)[j] = __ldg(reinterpret_cast<const float4*>(src) + j);
+        } else {
+          for (int j = lane; j < m; j += 32) zr[j] = src[j];
+        }
+      } else {
+        for (int j = lane; j < m; j += 32) zr[j] = 0.f;
+      }
+    }
+    __syncwarp();
+    float acc[TPG][EPL];
+#pragma unroll
+    for (int u = 0; u < TPG; ++u)
+#pragma unroll
+      for (int e = 0; e < EPL; ++e) acc[u][e] = 0.f;
+    const float4* r4 = reinterpret_cast<const float4*>(Rs) + (size_t)lane * rs4;
+    const float4* z4 = reinterpret_cast<const float4*>(zs);
+#pragma unroll 2
+    for (int j = 0; j < mr4; ++j) {
+      float4 r[EPL];
+#pragma unroll
+      for (int e = 0; e < EPL; ++e) r[e] = r4[(size_t)(32 * e) * rs4 + j];
+#pragma unroll
+      for (int u = 0; u < TPG; ++u) {
+        const float4 z = z4[(size_t)u * rs4 + j];
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) {
+          acc[u][e] = fmaf(z.x, r[e].x, acc[u][e]); acc[u][e] = fmaf(z.y, r[e].y, acc[u][e]);
+          acc[u][e] = fmaf(z.z, r[e].z, acc[u][e]); acc[u][e] = fmaf(z.w, r[e].w, acc[u][e]);
+        }
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < TPG; ++u) {
+      const int t = t0 + u;
+      if (t >= Ttok) continue;
+#pragma unroll
+      for (int e = 0; e < EPL; ++e) {
+        const int i = lane + 32 * e;
+        if (i < E) {
+          const float den = xn[u] * rn[i];
+          const float v = den == 0.f ? 0.f : sqD * acc[u][e] / den;
+          delta[(size_t)t * E + i] = v;
+          best = fmaxf(best, v);
+        }
+      }
+    }
+    __syncwarp();        // the slice is rewritten by the next group's copy
+  }
+  uint32_t key = best == -INFINITY ? 0u : ordered_key(best);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) key = max(key, __shfl_xor_sync(0xffffffffu, key, o));
+  if (lane == 0) red[warp] = key;
+  __syncthreads();
+  if (tid == 0) {
+    for (int w = 1; w < nw; ++w) key = max(key, red[w]);
+    if (key) atomicMax(&stats->delta_max_key, key);
+  }
+}
+
 // ---- forward, warp-autonomous persistent form (the default) ------------------------------------
 // R stays in shared memory for the life of the CTA; every warp owns a private slice for the
 // pooled rows of TPG tokens and loops on its own: pool TPG tokens (16-byte loads, one pass
@@ -512,11 +672,67 @@ static etr_status affinity_forward_warp(const etr_config* c, const void* X, cons
   return launch_affinity_warp<T, 8, 2>(c, X, R, delta, Z, xnorm, rnorm, stats, st, done);
 }
 
+template <class T>
+static etr_status launch_pool(const etr_config* c, const void* X, float* Z, float* xnorm, cudaStream_t st) {
+  constexpr int PE = Raw16<T>::ELEMS;
+  const int m = c->d / c->D, grid = ceil_div(c->T, 8), D = c->D;
+  ETR_TIME_BEGIN("grap_pool_kernel");
+  if (D == PE) grap_pool_kernel<T, 1><<<grid, 256, 0, st>>>((const T*)X, Z, xnorm, c->T, c->d, D, m);
+  else if (D == 2 * PE) grap_pool_kernel<T, 2><<<grid, 256, 0, st>>>((const T*)X, Z, xnorm, c->T, c->d, D, m);
+  else if (D == 4 * PE) grap_pool_kernel<T, 4><<<grid, 256, 0, st>>>((const T*)X, Z, xnorm, c->T, c->d, D, m);
+  else grap_pool_kernel<T, 0><<<grid, 256, 0, st>>>((const T*)X, Z, xnorm, c->T, c->d, D, m);
+  ETR_LAUNCH_CHECK();
+  return ETR_OK;
+}
+
+template <int EPL, int TPG>
+static etr_status launch_score(const etr_config* c, const float* Z, const float* xnorm, const float* R,
+                               float* delta, float* rnorm, etr_stats* stats, cudaStream_t st, bool* done) {
+  const int m = c->d / c->D, ldm = (m + 3) / 4 * 4 + 4;
+  *done = false;
+  for (int nw = 16; nw >= 4; nw /= 2) {
+    const size_t smem = ((size_t)(32 * EPL + nw * TPG) * ldm + 32 * EPL) * sizeof(float);
+    if (smem > 220 * 1024) continue;
+    auto k = affinity_score_kernel<EPL, TPG>;
+    if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+      return ETR_ERR_CUDA;
+    const int ngroups = ceil_div(c->T, TPG);
+    const int grid = std::min(device_sm_count(), ceil_div(ngroups, nw));
+    ETR_TIME_BEGIN("affinity_score_kernel");
+    k<<<grid, nw * 32, smem, st>>>(Z, xnorm, R, delta, rnorm, stats, c->T, c->D, c->E, m, ldm);
+    ETR_LAUNCH_CHECK();
+    *done = true;
+    return ETR_OK;
+  }
+  return ETR_OK;
+}
+
+// pool + score as two kernels; *done is false if the score kernel's shared memory does not fit
+static etr_status affinity_forward_split(const etr_config* c, const void* X, const float* R, float* delta,
+                                         float* Z, float* xnorm, float* rnorm, etr_stats* stats,
+                                         cudaStream_t st, bool* done) {
+  const int m = c->d / c->D, ldm = (m + 3) / 4 * 4 + 4;
+  const int EPL = c->E <= 32 ? 1 : c->E <= 64 ? 2 : c->E <= 128 ? 4 : 8;
+  const int TPG = EPL <= 2 ? 8 : EPL == 4 ? 4 : 2;
+  *done = false;
+  if (((size_t)(32 * EPL + 4 * TPG) * ldm + 32 * EPL) * sizeof(float) > 220 * 1024) return ETR_OK;
+  if (c->dtype == ETR_BF16) ETR_TRY(launch_pool<__nv_bfloat16>(c, X, Z, xnorm, st));
+  else ETR_TRY(launch_pool<float>(c, X, Z, xnorm, st));
+  if (EPL == 1) return launch_score<1, 8>(c, Z, xnorm, R, delta, rnorm, stats, st, done);
+  if (EPL == 2) return launch_score<2, 8>(c, Z, xnorm, R, delta, rnorm, stats, st, done);
+  if (EPL == 4) return launch_score<4, 4>(c, Z, xnorm, R, delta, rnorm, stats, st, done);
+  return launch_score<8, 2>(c, Z, xnorm, R, delta, rnorm, stats, st, done);
+}
+
 etr_status affinity_forward(const etr_config* c, const void* X, const float* R, float* delta,
                             float* Z, float* xnorm, float* rnorm, etr_stats* stats,
                             cudaStream_t st) {
   const int m = c->d / c->D;
   bool done = false;
+  if (Z != nullptr) {
+    ETR_TRY(affinity_forward_split(c, X, R, delta, Z, xnorm, rnorm, stats, st, &done));
+    if (done) return ETR_OK;
+  }
   if (c->dtype == ETR_BF16)
     ETR_TRY(affinity_forward_warp<__nv_bfloat16>(c, X, R, delta, Z, xnorm, rnorm, stats, st, &done));
   else
