@@ -1,0 +1,101 @@
+"""Edge cases of the CUDA path against the oracle: experts that receive no token, Top-1
+routing (the paper's efficiency runs), k = E, capacity 1, a handful of tokens, and group
+sizes that take the generic pooling path."""
+import numpy as np
+import pytest
+import torch
+
+from gen import workloads as gw
+from oracle import binding as ob
+from tests import harness as hz
+
+pytestmark = pytest.mark.gpu
+etr = hz.etr
+W = gw.WORKLOADS
+
+
+def layer_vs_oracle(w, inp, mode, impl=etr.GEMM_AUTO):
+    o = ob.Oracle("f32")
+    fw = o.forward(inp["X"], inp["R"], inp["W1g"], inp["W1u"], inp["W2"], D=w.D, k=w.k,
+                   capacity=w.capacity, mode=mode)
+    bw = o.backward(fw, inp["X"], inp["R"], inp["W1g"], inp["W1u"], inp["W2"], inp["dY"])
+    cfg = hz.make_cfg(w, mode=mode, gemm_impl=impl)
+    dev = hz.upload(w, inp)
+    buf = etr.LayerBuffers(cfg)
+    out = dict(Y=torch.empty_like(dev.X), dX=torch.empty_like(dev.X), dR=torch.empty_like(dev.R),
+               dW1g=torch.full_like(dev.W1g, float("nan")), dW1u=torch.full_like(dev.W1u, float("nan")),
+               dW2=torch.full_like(dev.W2, float("nan")))
+    etr.layer_forward(cfg, dev.X, dev.R, dev.W1g, dev.W1u, dev.W2, buf, out["Y"])
+    etr.layer_backward(cfg, dev.X, dev.R, dev.W1g, dev.W1u, dev.W2, dev.dY, buf, out["dX"], out["dR"],
+                       out["dW1g"], out["dW1u"], out["dW2"])
+    torch.cuda.synchronize()
+    assert buf.read_stats().error_word == 0
+    got = hz.route_from_buffers(buf, cfg)
+    hz.check_route_structure(hz.to_np(buf.delta), got, mode)
+    identical = hz.assert_routes_match(fw.delta, fw.route, got, mode)
+    assert identical, "these cases are built with clear margins"
+    tol = 2e-2 if w.dtype == "bf16" else 1e-4
+    for nm, ref, chain in (("Y", fw.Y, 4), ("dX", bw.dX, 6), ("dR", bw.dR, 1), ("dW1g", bw.dW1g, 6),
+                           ("dW1u", bw.dW1u, 6), ("dW2", bw.dW2, 4)):
+        hz.assert_close_rms(hz.to_np(out[nm]), ref, tol, nm, chain=chain)
+    return fw, got, out
+
+
+@pytest.mark.parametrize("dtype,impl", [("f32", etr.GEMM_AUTO), ("bf16", etr.GEMM_AUTO), ("bf16", etr.GEMM_SIMT)])
+def test_experts_without_tokens_get_zero_gradients(dtype, impl):
+    """Token choice with every token pushed away from experts 2 and 5: their buffers stay
+    empty, their weight gradients must be exactly zero, everything else must match."""
+    w = gw.scaled(W["small"], T=384, d=256, D=8, E=8, h=128, dtype=dtype)
+    inp = gw.make_inputs(w)
+    lean = np.repeat(inp["R"], w.D, axis=1)              # expert directions in R^d
+    X = inp["X"] - 0.5 * (lean[2] + lean[5])[None, :] * np.sqrt(w.d / w.D)
+    inp["X"] = gw.round_to_bf16(X) if dtype == "bf16" else X.astype(np.float32)
+    fw, got, out = layer_vs_oracle(w, inp, ob.MODE_TCR, impl)
+    assert got.counts[2] == 0 and got.counts[5] == 0 and got.counts.sum() > 0
+    for nm in ("dW1g", "dW1u", "dW2"):
+        g = out[nm]
+        assert bool((g[2] == 0).all()) and bool((g[5] == 0).all()), nm
+    assert bool((out["dR"][2] == 0).all())
+
+
+@pytest.mark.parametrize("k", [1, 8])
+def test_top1_and_top_all(k):
+    w = gw.scaled(W["small"], T=300, d=256, D=8, E=8, h=192, k=k, cf=0.8)
+    layer_vs_oracle(w, gw.make_inputs(w), ob.MODE_TCR)
+
+
+@pytest.mark.parametrize("mode", [ob.MODE_TCR, ob.MODE_ECR])
+def test_capacity_one_and_few_tokens(mode):
+    w = gw.scaled(W["small"], T=5, d=128, D=8, E=4, h=64, cf=0.2)
+    assert w.capacity == 1
+    layer_vs_oracle(w, gw.make_inputs(w), mode)
+
+
+@pytest.mark.parametrize("D,dtype", [(1, "f32"), (2, "bf16"), (4, "bf16"), (32, "bf16"), (24, "f32")])
+def test_group_sizes(D, dtype):
+    """D = 1 (plain cosine routing), sub-vector groups, wide groups and a group size that is
+    neither a divisor nor a multiple of 8."""
+    d = 768 if D == 24 else 512
+    w = gw.scaled(W["small"], T=200, d=d, D=D, E=8, h=64, dtype=dtype)
+    layer_vs_oracle(w, gw.make_inputs(w), ob.MODE_TCR)
+
+
+def test_sweep_modes_follow_the_step():
+    """ETR_MODE_AUTO picks token choice before switch_step and expert choice from it on."""
+    for step, want in ((999, etr.MODE_TCR), (1000, etr.MODE_ECR)):
+        w = gw.scaled(W["sweep"], T=256, d=256, D=16, E=8, h=64, n_clusters=8, step=step)
+        inp = gw.make_inputs(w)
+        cfg = etr.make_config(T=w.T, d=w.d, D=w.D, E=w.E, k=w.k, h=w.h, capacity=w.capacity,
+                              dtype=etr.BF16, mode=etr.MODE_AUTO, step=step, switch_step=w.switch_step,
+                              adaptive=True)
+        dev = hz.upload(w, inp)
+        buf = etr.LayerBuffers(cfg)
+        Y = torch.empty_like(dev.X)
+        etr.layer_forward(cfg, dev.X, dev.R, dev.W1g, dev.W1u, dev.W2, buf, Y)
+        st = buf.read_stats()
+        assert st.mode == want and 1 <= st.C <= w.capacity
+        o = ob.Oracle("f32")
+        delta, *_ = o.affinity(inp["X"], inp["R"], w.D)
+        assert st.C == ob.capacity_bound(w.d, w.E, w.capacity, 1, True, st.delta_max)
+        if want == etr.MODE_ECR:
+            assert np.all(hz.to_np(buf.counts) == min(st.C, w.T))
