@@ -420,6 +420,344 @@ tc_grouped_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_c
   }
 }
 
+// ---- two-CTA form ---------------------------------------------------------------------------------
+// The same pipeline on CTA pairs (thread-block cluster of 2, tcgen05 cta_group::2): one MMA covers
+// 256 x 256 x 16, each CTA holding its own 128 rows of A, half of the B tile (128 of the 256
+// columns) and the accumulator of its 128 rows.  Per CTA and K block only 32 KiB enter shared
+// memory instead of 48 KiB, and the tensor core reads half of B from the peer, which takes
+// pressure off the shared-memory port; six stages fit.  Only the leader CTA (cluster rank 0)
+// issues MMAs.  Both CTAs' TMA loads complete on the leader's "full" barrier; the leader's
+// commits are multicast to both CTAs' "empty" and "accumulator full" barriers; the epilogue
+// warps of both CTAs arrive on the leader's "accumulator empty" barrier.  No load is multicast.
+constexpr int TC2_STAGES = 6;
+constexpr uint32_t TC2_STAGE_BYTES = 4 * TC_BOX_BYTES;       // per CTA: 2 boxes of A, 2 of B
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ uint32_t cluster_id_x() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%clusterid.x;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ uint32_t cluster_count_x() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%nclusterid.x;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  if (mbar_try_wait_cluster(bar, parity)) return true;
+  const long long t0 = clock64();
+  for (uint32_t it = 1;; ++it) {
+    if (mbar_try_wait_cluster(bar, parity)) return true;
+    if ((it & 255u) == 0u) {
+      if (*abort_flag) return false;
+      if (clock64() - t0 > TC_WAIT_LIMIT_CYCLES) { *abort_flag = 1; return false; }
+    }
+  }
+}
+// TMA load into this CTA's shared memory whose completion is counted on a barrier of the pair
+// (cluster address); not a multicast.
+__device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap* map, uint32_t bar_cluster,
+                                                 int c0, int c1, int c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes"
+      " [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar_cluster), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {      // arrives on `bar` in both CTAs
+  const uint16_t mask = 3;
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"(mask) : "memory");
+}
+__device__ __forceinline__ void tc_mma_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                            uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+
+// Pair-tile index -> coordinates (256 rows per pair tile).
+__device__ __forceinline__ bool tile_coord_pair(const TcParams& p, const int* tile_prefix, int tile, int& e_cur,
+                                                int n_tile_cols, TileCoord& tc) {
+  if (tile >= tile_prefix[p.E]) return false;
+  while (tile >= tile_prefix[e_cur + 1]) ++e_cur;
+  const int local = tile - tile_prefix[e_cur];
+  const int n_e = p.counts[e_cur];
+  int mt_count;
+  if (p.dyn == TC_DYN_M) {
+    mt_count = (min(n_e, p.M) + 255) / 256;
+    tc.kblocks = (p.K + TC_BK - 1) / TC_BK;
+    tc.m_lim = (min(n_e, p.M) + TC_BM - 1) / TC_BM * TC_BM;
+  } else {
+    mt_count = (p.M + 255) / 256;
+    tc.kblocks = (n_e + TC_BK - 1) / TC_BK;
+    tc.m_lim = p.M;
+  }
+  tc.e = e_cur;
+  tc.m0 = (local % mt_count) * 256;
+  tc.n0 = (local / mt_count) * n_tile_cols;
+  return true;
+}
+
+template <int EPI>
+__global__ void __launch_bounds__(TC_THREADS, 1)
+tc_grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtensorMap mapA1,
+                            const __grid_constant__ CUtensorMap mapB0, const __grid_constant__ CUtensorMap mapB1,
+                            const TcParams p) {
+  constexpr int BN = 256;
+  constexpr int N_TILE_COLS = (EPI == TC_EPI_SWIGLU) ? BN / 2 : BN;
+  constexpr uint32_t TMEM_COLS = 512;
+
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t bars[2 * TC2_STAGES + 4];
+  __shared__ uint32_t tmem_base_slot;
+  __shared__ int abort_flag_s;
+  __shared__ int tile_prefix[257];
+
+  volatile int* abort_flag = &abort_flag_s;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const uint32_t rank = cluster_ctarank();
+  const int pair = (int)cluster_id_x(), npairs = (int)cluster_count_x();
+  const uint32_t tiles_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t full_bar = smem_u32(&bars[0]);                    // [TC2_STAGES]  used in the leader
+  const uint32_t empty_bar = smem_u32(&bars[TC2_STAGES]);          // [TC2_STAGES]  in each CTA
+  const uint32_t tfull_bar = smem_u32(&bars[2 * TC2_STAGES]);      // [2]           in each CTA
+  const uint32_t tempty_bar = smem_u32(&bars[2 * TC2_STAGES + 2]); // [2]           used in the leader
+
+  if (tid == 0) {
+    abort_flag_s = 0;
+    for (int s = 0; s < TC2_STAGES; ++s) { mbar_init(full_bar + 8 * s, 1); mbar_init(empty_bar + 8 * s, 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar + 8 * a, 1); mbar_init(tempty_bar + 8 * a, 16); }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    const int nt = (p.N + N_TILE_COLS - 1) / N_TILE_COLS;
+    int acc = 0;
+    for (int e = 0; e < p.E; ++e) {
+      tile_prefix[e] = acc;
+      const int n_e = p.counts[e];
+      const int mt = p.dyn == TC_DYN_M ? (min(n_e, p.M) + 255) / 256 : (p.M + 255) / 256;
+      acc += mt * nt;
+    }
+    tile_prefix[p.E] = acc;
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"(TMEM_COLS) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();                 // both CTAs' barriers exist before any remote arrive
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_slot;
+  const uint32_t leader_full = map_to_cta(full_bar, 0);
+  const uint32_t leader_tempty = map_to_cta(tempty_bar, 0);
+
+  if (warp == 0) {
+    // ---- TMA producer (both CTAs) ---------------------------------------------------------------
+    if (lane == 0) {
+      int e_cur = 0, stage = 0;
+      uint32_t phase = 0;
+      TileCoord tc;
+      bool ok = true;
+      for (int tile = pair; ok && tile_coord_pair(p, tile_prefix, tile, e_cur, N_TILE_COLS, tc); tile += npairs) {
+        const int m0c = tc.m0 + 128 * (int)rank;
+        for (int kb = 0; kb < tc.kblocks; ++kb) {
+          if (!mbar_wait_cluster(empty_bar + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
+          if (rank == 0) mbar_expect_tx(full_bar + 8 * stage, 2 * TC2_STAGE_BYTES);
+          const uint32_t fb = leader_full + 8 * stage;
+          const bool second = p.k1_blocks > 0 && kb >= p.k1_blocks;
+          const int k0 = (second ? kb - p.k1_blocks : kb) * TC_BK;
+          const CUtensorMap* ma = second ? &mapA1 : &mapA0;
+          const CUtensorMap* mb = p.dual_b ? (rank ? &mapB1 : &mapB0) : (second ? &mapB1 : &mapB0);
+          const int nb = p.dual_b ? tc.n0 : tc.n0 + 128 * (int)rank;
+          const uint32_t sa = tiles_base + stage * TC2_STAGE_BYTES;
+          const uint32_t sb = sa + 2 * TC_BOX_BYTES;
+#pragma unroll
+          for (int j = 0; j < 2; ++j) {
+            if (p.a_mn) tma_load_3d_pair(sa + j * TC_BOX_BYTES, ma, fb, m0c + 64 * j, k0, tc.e);
+            else        tma_load_3d_pair(sa + j * TC_BOX_BYTES, ma, fb, k0, m0c + 64 * j, tc.e);
+            if (p.b_mn) tma_load_3d_pair(sb + j * TC_BOX_BYTES, mb, fb, nb + 64 * j, k0, tc.e);
+            else        tma_load_3d_pair(sb + j * TC_BOX_BYTES, mb, fb, k0, nb + 64 * j, tc.e);
+          }
+          if (++stage == TC2_STAGES) { stage = 0; phase ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---- MMA issuer (leader CTA only) --------------------------------------------------------------
+    if (lane == 0 && rank == 0) {
+      int e_cur = 0, stage = 0, acc_stage = 0;
+      uint32_t phase = 0, acc_phase = 0;
+      TileCoord tc;
+      bool ok = true;
+      const uint32_t a_lbo = p.a_mn ? TC_BOX_BYTES : 16u, b_lbo = p.b_mn ? TC_BOX_BYTES : 16u;
+      const uint32_t a_kstep = p.a_mn ? 2048u : 32u, b_kstep = p.b_mn ? 2048u : 32u;
+      for (int tile = pair; ok && tile_coord_pair(p, tile_prefix, tile, e_cur, N_TILE_COLS, tc); tile += npairs) {
+        if (tc.kblocks == 0) continue;
+        if (!mbar_wait_cluster(tempty_bar + 8 * acc_stage, acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc_stage * 256);
+        for (int kb = 0; kb < tc.kblocks; ++kb) {
+          if (!mbar_wait_cluster(full_bar + 8 * stage, phase, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sa = tiles_base + stage * TC2_STAGE_BYTES;
+          const uint32_t sb = sa + 2 * TC_BOX_BYTES;
+#pragma unroll
+          for (int kk = 0; kk < TC_BK / 16; ++kk) {
+            const uint64_t ad = make_smem_desc(sa + kk * a_kstep, a_lbo, 1024u);
+            const uint64_t bd = make_smem_desc(sb + kk * b_kstep, b_lbo, 1024u);
+            tc_mma_pair(d_tmem, ad, bd, p.idesc, (kb > 0 || kk > 0) ? 1u : 0u);
+          }
+          tc_commit_pair(empty_bar + 8 * stage);      // frees the stage in both CTAs
+          if (++stage == TC2_STAGES) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        tc_commit_pair(tfull_bar + 8 * acc_stage);    // accumulators complete in both CTAs
+        if (++acc_stage == 2) { acc_stage = 0; acc_phase ^= 1u; }
+      }
+    }
+  } else {
+    // ---- epilogue warps (both CTAs, own 128 rows) -----------------------------------------------------
+    const int q = warp & 3;
+    const int half = (warp - 2) >> 2;
+    constexpr int NCH = N_TILE_COLS / 32 / 2;
+    const int row_in_tile = 128 * (int)rank + 32 * q + lane;
+    int e_cur = 0, acc_stage = 0;
+    uint32_t acc_phase = 0;
+    TileCoord tc;
+    bool ok = true;
+    for (int tile = pair; ok && tile_coord_pair(p, tile_prefix, tile, e_cur, N_TILE_COLS, tc); tile += npairs) {
+      const int grow = tc.m0 + row_in_tile;
+      const bool row_ok = grow < tc.m_lim;
+      const int c_beg = half * NCH;
+      const long long obase = (long long)tc.e * p.out_bs + (long long)grow * p.ld_out + tc.n0;
+      if (tc.kblocks == 0) {
+        if (row_ok) {
+          float z[32];
+#pragma unroll
+          for (int i = 0; i < 32; ++i) z[i] = 0.f;
+          for (int c = c_beg; c < c_beg + NCH && tc.n0 + 32 * c < p.N; ++c) store32(p.out0 + obase + 32 * c, z);
+        }
+        continue;
+      }
+      uint4 pg[4], pu[4];
+      if (EPI == TC_EPI_DSWIGLU && row_ok && tc.n0 + 32 * c_beg < p.N) {
+        const uint4* sg = reinterpret_cast<const uint4*>(p.in0 + obase + 32 * c_beg);
+        const uint4* su = reinterpret_cast<const uint4*>(p.in1 + obase + 32 * c_beg);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) { pg[i] = sg[i]; pu[i] = su[i]; }
+      }
+      if (!mbar_wait_cluster(tfull_bar + 8 * acc_stage, acc_phase, abort_flag)) { ok = false; break; }
+      tc_fence_after();
+      const uint32_t taddr = tmem_base + (uint32_t)(acc_stage * 256) + ((uint32_t)(32 * q) << 16);
+#pragma unroll 1
+      for (int c = c_beg; c < c_beg + NCH; ++c) {
+        if (tc.n0 + 32 * c >= p.N) break;
+        __syncwarp();
+        uint32_t r0[32];
+        float v[32];
+        tc_ld32(taddr + 32 * c, r0);
+        if (EPI == TC_EPI_SWIGLU) {
+          uint32_t r1[32];
+          tc_ld32(taddr + BN / 2 + 32 * c, r1);
+          tc_wait_ld();
+          if (row_ok) {
+            float hv[32];
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+              const float g = __uint_as_float(r0[i]), u = __uint_as_float(r1[i]);
+              hv[i] = g / (1.0f + __expf(-g)) * u;
+              v[i] = g;
+            }
+            store32(p.out0 + obase + 32 * c, v);
+            store32(p.out2 + obase + 32 * c, hv);
+#pragma unroll
+            for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r1[i]);
+            store32(p.out1 + obase + 32 * c, v);
+          }
+        } else if (EPI == TC_EPI_DSWIGLU) {
+          uint4 cg[4], cu[4];
+#pragma unroll
+          for (int i = 0; i < 4; ++i) { cg[i] = pg[i]; cu[i] = pu[i]; }
+          if (row_ok && c + 1 < c_beg + NCH && tc.n0 + 32 * (c + 1) < p.N) {
+            const uint4* sg = reinterpret_cast<const uint4*>(p.in0 + obase + 32 * (c + 1));
+            const uint4* su = reinterpret_cast<const uint4*>(p.in1 + obase + 32 * (c + 1));
+#pragma unroll
+            for (int i = 0; i < 4; ++i) { pg[i] = sg[i]; pu[i] = su[i]; }
+          }
+          tc_wait_ld();
+          if (row_ok) {
+            float dg[32];
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+              const uint32_t wg = reinterpret_cast<const uint32_t*>(cg)[i >> 1];
+              const uint32_t wu = reinterpret_cast<const uint32_t*>(cu)[i >> 1];
+              const float g = (i & 1) ? __uint_as_float(wg & 0xffff0000u) : __uint_as_float(wg << 16);
+              const float u = (i & 1) ? __uint_as_float(wu & 0xffff0000u) : __uint_as_float(wu << 16);
+              const float dh = __uint_as_float(r0[i]);
+              const float sgm = 1.0f / (1.0f + __expf(-g));
+              dg[i] = dh * u * sgm * (1.0f + g * (1.0f - sgm));
+              v[i] = dh * g * sgm;
+            }
+            store32(p.out0 + obase + 32 * c, dg);
+            store32(p.out1 + obase + 32 * c, v);
+          }
+        } else {
+          tc_wait_ld();
+          if (row_ok) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r0[i]);
+            store32(p.out0 + obase + 32 * c, v);
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(leader_tempty + 8 * acc_stage);
+      if (++acc_stage == 2) { acc_stage = 0; acc_phase ^= 1u; }
+    }
+  }
+
+  // ---- teardown: neither CTA leaves while the other may still touch its barriers or memory -------
+  __syncwarp();
+  if (*abort_flag) {
+    const long long t0 = clock64();
+    while (clock64() - t0 < 2000000ll) { }
+    if (tid == 0) atomicExch(&p.stats->error_word, 0x7c06);
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+  }
+}
+
 // ---- host side --------------------------------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
@@ -453,7 +791,7 @@ static etr_status make_map(CUtensorMap* m, const void* base, int cols, int rows,
   return r == CUDA_SUCCESS ? ETR_OK : ETR_ERR_CUDA;
 }
 
-static uint32_t make_idesc(int a_mn, int b_mn, int n) {
+static uint32_t make_idesc(int a_mn, int b_mn, int n, int m_instr = TC_BM) {
   uint32_t d = 0;
   d |= 1u << 4;                     // accumulator fp32
   d |= 1u << 7;                     // A bf16
@@ -461,7 +799,7 @@ static uint32_t make_idesc(int a_mn, int b_mn, int n) {
   d |= (uint32_t)(a_mn ? 1 : 0) << 15;
   d |= (uint32_t)(b_mn ? 1 : 0) << 16;
   d |= (uint32_t)(n >> 3) << 17;
-  d |= (uint32_t)(TC_BM >> 4) << 24;
+  d |= (uint32_t)(m_instr >> 4) << 24;
   return d;
 }
 
@@ -496,6 +834,46 @@ static etr_status tc_launch(const char* name, const CUtensorMap& a0, const CUten
   return ETR_OK;
 }
 
+template <int EPI>
+static etr_status tc_launch_pair(const char* name, const CUtensorMap& a0, const CUtensorMap& a1,
+                                 const CUtensorMap& b0, const CUtensorMap& b1, TcParams p, int max_tiles,
+                                 cudaStream_t st) {
+  constexpr size_t smem = (size_t)TC2_STAGES * TC2_STAGE_BYTES + 1024;
+  auto k = tc_grouped_gemm_pair_kernel<EPI>;
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+      return ETR_ERR_CUDA;
+    attr_set = true;
+  }
+  p.idesc = make_idesc(p.a_mn, p.b_mn, 256, 256);
+  const int pairs_max = sm_count() / 2;
+  const int pairs = max_tiles < pairs_max ? (max_tiles < 1 ? 1 : max_tiles) : pairs_max;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(2 * pairs);
+  cfg.blockDim = dim3(TC_THREADS);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  ETR_TIME_BEGIN(name);
+  if (cudaLaunchKernelEx(&cfg, k, a0, a1, b0, b1, p) != cudaSuccess) { timing_end(st); return ETR_ERR_CUDA; }
+  ETR_LAUNCH_CHECK();
+  return ETR_OK;
+}
+
+// 1-CTA or 2-CTA form of one contraction; max tiles are counted in 128-row tiles
+template <int EPI>
+static etr_status tc_run(bool pair, const char* name, const CUtensorMap& a0, const CUtensorMap& a1,
+                         const CUtensorMap& b0, const CUtensorMap& b1, const TcParams& p, int max_tiles,
+                         cudaStream_t st) {
+  if (pair) return tc_launch_pair<EPI>(name, a0, a1, b0, b1, p, (max_tiles + 1) / 2, st);
+  return tc_launch<256, EPI>(name, a0, a1, b0, b1, p, max_tiles, st);
+}
+
 size_t tc_workspace_bytes(const etr_config*) { return 0; }
 bool tc_available() { return true; }
 
@@ -503,6 +881,7 @@ etr_status tc_ffn_forward(const etr_config* c, const etr_route* rt, const void* 
                           const void* W1u, const void* W2, void* G, void* U, void* H, void* O,
                           etr_stats* stats, void*, cudaStream_t st) {
   const int d = c->d, h = c->h, Cs = c_stride_of(c), E = c->E;
+  const bool pair = c->gemm_impl == ETR_GEMM_TCGEN05_2CTA;
   CUtensorMap mXp, mW1g, mW1u, mW2, mH;
   ETR_TRY(make_map(&mXp, Xp, d, Cs, E));
   ETR_TRY(make_map(&mW1g, W1g, d, h, E));
@@ -515,14 +894,14 @@ etr_status tc_ffn_forward(const etr_config* c, const etr_route* rt, const void* 
     p.dual_b = 1; p.M = Cs; p.N = h; p.K = d; p.dyn = TC_DYN_M; p.E = E; p.counts = rt->counts;
     p.out0 = (__nv_bfloat16*)G; p.out1 = (__nv_bfloat16*)U; p.out2 = (__nv_bfloat16*)H;
     p.out_bs = (long long)Cs * h; p.ld_out = h; p.stats = stats;
-    ETR_TRY((tc_launch<256, TC_EPI_SWIGLU>("tc_gemm_swiglu", mXp, mXp, mW1g, mW1u, p,
+    ETR_TRY((tc_run<TC_EPI_SWIGLU>(pair, "tc_gemm_swiglu", mXp, mXp, mW1g, mW1u, p,
                                            E * mt * ceil_div(h, 128), st)));
   }
   {  // O = H W2^T
     TcParams p = {};
     p.M = Cs; p.N = d; p.K = h; p.dyn = TC_DYN_M; p.E = E; p.counts = rt->counts;
     p.out0 = (__nv_bfloat16*)O; p.out_bs = (long long)Cs * d; p.ld_out = d; p.stats = stats;
-    ETR_TRY((tc_launch<256, TC_EPI_STORE>("tc_gemm_down", mH, mH, mW2, mW2, p, E * mt * ceil_div(d, 256), st)));
+    ETR_TRY((tc_run<TC_EPI_STORE>(pair, "tc_gemm_down", mH, mH, mW2, mW2, p, E * mt * ceil_div(d, 256), st)));
   }
   return ETR_OK;
 }
@@ -532,6 +911,7 @@ etr_status tc_ffn_backward(const etr_config* c, const etr_route* rt, const void*
                            const void* W1u, const void* W2, void* dG, void* dU, void* dXp, void* dW1g,
                            void* dW1u, void* dW2, etr_stats* stats, void*, cudaStream_t st) {
   const int d = c->d, h = c->h, Cs = c_stride_of(c), E = c->E;
+  const bool pair = c->gemm_impl == ETR_GEMM_TCGEN05_2CTA;
   CUtensorMap mdO, mXp, mH, mdG, mdU, mW1g, mW1u, mW2;
   ETR_TRY(make_map(&mdO, dO, d, Cs, E));
   ETR_TRY(make_map(&mXp, Xp, d, Cs, E));
@@ -548,7 +928,7 @@ etr_status tc_ffn_backward(const etr_config* c, const etr_route* rt, const void*
     p.out0 = (__nv_bfloat16*)dG; p.out1 = (__nv_bfloat16*)dU;
     p.in0 = (const __nv_bfloat16*)G; p.in1 = (const __nv_bfloat16*)U;
     p.out_bs = (long long)Cs * h; p.ld_out = h; p.stats = stats;
-    ETR_TRY((tc_launch<256, TC_EPI_DSWIGLU>("tc_gemm_dswiglu", mdO, mdO, mW2, mW2, p,
+    ETR_TRY((tc_run<TC_EPI_DSWIGLU>(pair, "tc_gemm_dswiglu", mdO, mdO, mW2, mW2, p,
                                             E * mt * ceil_div(h, 256), st)));
   }
   {  // dXp = dG W1g + dU W1u: one contraction over 2h
@@ -556,14 +936,14 @@ etr_status tc_ffn_backward(const etr_config* c, const etr_route* rt, const void*
     p.b_mn = 1; p.k1_blocks = ceil_div(h, TC_BK); p.M = Cs; p.N = d; p.K = 2 * h; p.dyn = TC_DYN_M;
     p.E = E; p.counts = rt->counts;
     p.out0 = (__nv_bfloat16*)dXp; p.out_bs = (long long)Cs * d; p.ld_out = d; p.stats = stats;
-    ETR_TRY((tc_launch<256, TC_EPI_STORE>("tc_gemm_dxp", mdG, mdU, mW1g, mW1u, p,
+    ETR_TRY((tc_run<TC_EPI_STORE>(pair, "tc_gemm_dxp", mdG, mdU, mW1g, mW1u, p,
                                           E * mt * ceil_div(d, 256), st)));
   }
   {  // dW2 = dO^T H: contraction over the expert's rows, both operands MN-major
     TcParams p = {};
     p.a_mn = 1; p.b_mn = 1; p.M = d; p.N = h; p.dyn = TC_DYN_K; p.E = E; p.counts = rt->counts;
     p.out0 = (__nv_bfloat16*)dW2; p.out_bs = (long long)d * h; p.ld_out = h; p.stats = stats;
-    ETR_TRY((tc_launch<256, TC_EPI_STORE>("tc_gemm_dw2", mdO, mdO, mH, mH, p,
+    ETR_TRY((tc_run<TC_EPI_STORE>(pair, "tc_gemm_dw2", mdO, mdO, mH, mH, p,
                                           E * ceil_div(d, TC_BM) * ceil_div(h, 256), st)));
   }
   for (int which = 0; which < 2; ++which) {  // dW1g = dG^T Xp, dW1u = dU^T Xp
@@ -571,7 +951,7 @@ etr_status tc_ffn_backward(const etr_config* c, const etr_route* rt, const void*
     p.a_mn = 1; p.b_mn = 1; p.M = h; p.N = d; p.dyn = TC_DYN_K; p.E = E; p.counts = rt->counts;
     p.out0 = (__nv_bfloat16*)(which ? dW1u : dW1g); p.out_bs = (long long)h * d; p.ld_out = d; p.stats = stats;
     const CUtensorMap& ma = which ? mdU : mdG;
-    ETR_TRY((tc_launch<256, TC_EPI_STORE>("tc_gemm_dw1", ma, ma, mXp, mXp, p,
+    ETR_TRY((tc_run<TC_EPI_STORE>(pair, "tc_gemm_dw1", ma, ma, mXp, mXp, p,
                                           E * ceil_div(h, TC_BM) * ceil_div(d, 256), st)));
   }
   return ETR_OK;
