@@ -209,7 +209,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="large", choices=list(gw.WORKLOADS))
-    ap.add_argument("--gemm", default="auto", choices=["auto", "simt", "tcgen05"])
+    ap.add_argument("--gemm", default="auto", choices=["auto", "simt", "tcgen05", "tcgen05_2cta"])
     ap.add_argument("--cpu-tokens", type=int, default=128, help="tokens in the CPU-oracle sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--set", default="", help="override workload fields, e.g. T=32768,h=512 (profiling cases)")
@@ -266,7 +266,8 @@ def main():
     X, dY = Xh.to(dev), dYh.to(dev)
     R = torch.from_numpy(inp["R"]).to(dev)
     W1g, W1u, W2 = device_weights(w, dev, w.seed)
-    impl = {"auto": etr.GEMM_AUTO, "simt": etr.GEMM_SIMT, "tcgen05": etr.GEMM_TCGEN05}[args.gemm]
+    impl = {"auto": etr.GEMM_AUTO, "simt": etr.GEMM_SIMT, "tcgen05": etr.GEMM_TCGEN05,
+            "tcgen05_2cta": etr.GEMM_TCGEN05_2CTA}[args.gemm]
     cfg = etr.make_config(T=w.T, d=w.d, D=w.D, E=w.E, k=w.k, h=w.h, capacity=w.capacity,
                           dtype=etr.BF16 if w.dtype == "bf16" else etr.F32,
                           mode=etr.MODE_TCR if mode_name(w) == "tcr" else etr.MODE_ECR,
