@@ -69,7 +69,7 @@ typedef struct etr_config {
   int64_t step, switch_step;  /* ETR_MODE_AUTO: token choice while step < switch_step */
   int32_t mode;               /* etr_mode */
   int32_t dtype;              /* etr_dtype of activations and expert weights */
-  int32_t gemm_impl;          /* etr_gemm_impl; AUTO = tcgen05 for bf16, SIMT for fp32 */
+  int32_t gemm_impl;          /* etr_gemm_impl; AUTO = two-CTA tcgen05 for bf16, SIMT for fp32 */
   int32_t reserved;
 } etr_config;
 

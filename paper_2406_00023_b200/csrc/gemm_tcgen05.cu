@@ -881,7 +881,7 @@ etr_status tc_ffn_forward(const etr_config* c, const etr_route* rt, const void* 
                           const void* W1u, const void* W2, void* G, void* U, void* H, void* O,
                           etr_stats* stats, void*, cudaStream_t st) {
   const int d = c->d, h = c->h, Cs = c_stride_of(c), E = c->E;
-  const bool pair = c->gemm_impl == ETR_GEMM_TCGEN05_2CTA;
+  const bool pair = c->gemm_impl != ETR_GEMM_TCGEN05;      // default: CTA pairs
   CUtensorMap mXp, mW1g, mW1u, mW2, mH;
   ETR_TRY(make_map(&mXp, Xp, d, Cs, E));
   ETR_TRY(make_map(&mW1g, W1g, d, h, E));
@@ -911,7 +911,7 @@ etr_status tc_ffn_backward(const etr_config* c, const etr_route* rt, const void*
                            const void* W1u, const void* W2, void* dG, void* dU, void* dXp, void* dW1g,
                            void* dW1u, void* dW2, etr_stats* stats, void*, cudaStream_t st) {
   const int d = c->d, h = c->h, Cs = c_stride_of(c), E = c->E;
-  const bool pair = c->gemm_impl == ETR_GEMM_TCGEN05_2CTA;
+  const bool pair = c->gemm_impl != ETR_GEMM_TCGEN05;      // default: CTA pairs
   CUtensorMap mdO, mXp, mH, mdG, mdU, mW1g, mW1u, mW2;
   ETR_TRY(make_map(&mdO, dO, d, Cs, E));
   ETR_TRY(make_map(&mXp, Xp, d, Cs, E));
