@@ -586,15 +586,23 @@ affinity_bwd_dr_partial_kernel(const float* __restrict__ Z, const float* __restr
 #pragma unroll
   for (int u = 0; u < DR_MAXJ; ++u) acc[u] = 0.f;
   float sdd = 0.f;
-  for (int p = 0; p < np; ++p) {
-    const int t = s_t[p];
-    const float w = s_w[p];
-    sdd += s_dd[p];
+  // slots in batches of 8: the gathered Z values of a batch are all requested before the first
+  // is used; the accumulation order (ascending slot) is unchanged
+  for (int p0 = 0; p0 < np; p0 += 8) {
 #pragma unroll
     for (int u = 0; u < DR_MAXJ; ++u) {
       const int j = tid + u * 256;
-      if (j < m) acc[u] = fmaf(w, Z[(size_t)t * m + j], acc[u]);
+      if (j >= m) break;
+      float zv[8];
+#pragma unroll
+      for (int b = 0; b < 8; ++b) zv[b] = p0 + b < np ? Z[(size_t)s_t[p0 + b] * m + j] : 0.f;
+#pragma unroll
+      for (int b = 0; b < 8; ++b)
+        if (p0 + b < np) acc[u] = fmaf(s_w[p0 + b], zv[b], acc[u]);
     }
+#pragma unroll
+    for (int b = 0; b < 8; ++b)
+      if (p0 + b < np) sdd += s_dd[p0 + b];
   }
 #pragma unroll
   for (int u = 0; u < DR_MAXJ; ++u) {

@@ -156,6 +156,78 @@ __device__ __forceinline__ void load32(const __nv_bfloat16* src, float* v) {
 
 struct TileCoord { int e, m0, n0, kblocks, m_lim; };
 
+// The epilogue of one accumulator tile for one warp: `nch` chunks of 32 columns starting at
+// chunk c_beg, read from tensor memory at taddr and stored (or fused with SwiGLU / its
+// derivative) at row offset obase.  pg/pu hold the prefetched G and U of the first chunk.
+template <int EPI, int BN>
+__device__ __forceinline__ void epilogue_chunks(const TcParams& p, int n0, uint32_t taddr, long long obase,
+                                                bool row_ok, int c_beg, int nch, uint4 (&pg)[4],
+                                                uint4 (&pu)[4]) {
+#pragma unroll 1
+  for (int c = c_beg; c < c_beg + nch; ++c) {
+    if (n0 + 32 * c >= p.N) break;
+    __syncwarp();               // tcgen05.ld is warp-collective: reconverge after masked stores
+    uint32_t r0[32];
+    float v[32];
+    tc_ld32(taddr + 32 * c, r0);
+    if (EPI == TC_EPI_SWIGLU) {
+      uint32_t r1[32];
+      tc_ld32(taddr + BN / 2 + 32 * c, r1);
+      tc_wait_ld();
+      if (row_ok) {
+        float hv[32];
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          const float g = __uint_as_float(r0[i]), u = __uint_as_float(r1[i]);
+          hv[i] = __fdividef(g, 1.0f + __expf(-g)) * u;
+          v[i] = g;
+        }
+        store32(p.out0 + obase + 32 * c, v);
+        store32(p.out2 + obase + 32 * c, hv);
+#pragma unroll
+        for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r1[i]);
+        store32(p.out1 + obase + 32 * c, v);
+      }
+    } else if (EPI == TC_EPI_DSWIGLU) {
+      uint4 cg[4], cu[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) { cg[i] = pg[i]; cu[i] = pu[i]; }
+      if (row_ok && c + 1 < c_beg + nch && n0 + 32 * (c + 1) < p.N) {
+        const uint4* sg = reinterpret_cast<const uint4*>(p.in0 + obase + 32 * (c + 1));
+        const uint4* su = reinterpret_cast<const uint4*>(p.in1 + obase + 32 * (c + 1));
+#pragma unroll
+        for (int i = 0; i < 4; ++i) { pg[i] = sg[i]; pu[i] = su[i]; }
+      }
+      tc_wait_ld();
+      if (row_ok) {
+        float dg[32];
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          const uint32_t wg = reinterpret_cast<const uint32_t*>(cg)[i >> 1];
+          const uint32_t wu = reinterpret_cast<const uint32_t*>(cu)[i >> 1];
+          const float g = (i & 1) ? __uint_as_float(wg & 0xffff0000u) : __uint_as_float(wg << 16);
+          const float u = (i & 1) ? __uint_as_float(wu & 0xffff0000u) : __uint_as_float(wu << 16);
+          const float dh = __uint_as_float(r0[i]);
+          const float sgm = __fdividef(1.0f, 1.0f + __expf(-g));
+          dg[i] = dh * u * sgm * (1.0f + g * (1.0f - sgm));
+          v[i] = dh * g * sgm;
+        }
+        store32(p.out0 + obase + 32 * c, dg);
+        store32(p.out1 + obase + 32 * c, v);
+      }
+    } else {
+      tc_wait_ld();
+      if (row_ok) {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r0[i]);
+        store32(p.out0 + obase + 32 * c, v);
+      }
+    }
+  }
+}
+
+
+
 // Tile index -> coordinates.  tile_prefix[e] = first tile of expert e.
 __device__ __forceinline__ bool tile_coord(const TcParams& p, const int* tile_prefix, int tile, int& e_cur,
                                            int n_tile_cols, TileCoord& tc) {
@@ -336,67 +408,7 @@ tc_grouped_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_c
       if (!mbar_wait(tfull_bar + 8 * acc_stage, acc_phase, abort_flag)) { ok = false; break; }
       tc_fence_after();
       const uint32_t taddr = tmem_base + (uint32_t)(acc_stage * 256) + ((uint32_t)(32 * q) << 16);
-#pragma unroll 1
-      for (int c = c_beg; c < c_beg + NCH; ++c) {
-        if (tc.n0 + 32 * c >= p.N) break;
-        __syncwarp();               // tcgen05.ld is warp-collective: reconverge after masked stores
-        uint32_t r0[32];
-        float v[32];
-        tc_ld32(taddr + 32 * c, r0);
-        if (EPI == TC_EPI_SWIGLU) {
-          uint32_t r1[32];
-          tc_ld32(taddr + BN / 2 + 32 * c, r1);
-          tc_wait_ld();
-          if (row_ok) {
-            float hv[32];
-#pragma unroll
-            for (int i = 0; i < 32; ++i) {
-              const float g = __uint_as_float(r0[i]), u = __uint_as_float(r1[i]);
-              hv[i] = g / (1.0f + __expf(-g)) * u;
-              v[i] = g;
-            }
-            store32(p.out0 + obase + 32 * c, v);
-            store32(p.out2 + obase + 32 * c, hv);
-#pragma unroll
-            for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r1[i]);
-            store32(p.out1 + obase + 32 * c, v);
-          }
-        } else if (EPI == TC_EPI_DSWIGLU) {
-          uint4 cg[4], cu[4];
-#pragma unroll
-          for (int i = 0; i < 4; ++i) { cg[i] = pg[i]; cu[i] = pu[i]; }
-          if (row_ok && c + 1 < c_beg + NCH && tc.n0 + 32 * (c + 1) < p.N) {
-            const uint4* sg = reinterpret_cast<const uint4*>(p.in0 + obase + 32 * (c + 1));
-            const uint4* su = reinterpret_cast<const uint4*>(p.in1 + obase + 32 * (c + 1));
-#pragma unroll
-            for (int i = 0; i < 4; ++i) { pg[i] = sg[i]; pu[i] = su[i]; }
-          }
-          tc_wait_ld();
-          if (row_ok) {
-            float dg[32];
-#pragma unroll
-            for (int i = 0; i < 32; ++i) {
-              const uint32_t wg = reinterpret_cast<const uint32_t*>(cg)[i >> 1];
-              const uint32_t wu = reinterpret_cast<const uint32_t*>(cu)[i >> 1];
-              const float g = (i & 1) ? __uint_as_float(wg & 0xffff0000u) : __uint_as_float(wg << 16);
-              const float u = (i & 1) ? __uint_as_float(wu & 0xffff0000u) : __uint_as_float(wu << 16);
-              const float dh = __uint_as_float(r0[i]);
-              const float sgm = 1.0f / (1.0f + __expf(-g));
-              dg[i] = dh * u * sgm * (1.0f + g * (1.0f - sgm));
-              v[i] = dh * g * sgm;
-            }
-            store32(p.out0 + obase + 32 * c, dg);
-            store32(p.out1 + obase + 32 * c, v);
-          }
-        } else {
-          tc_wait_ld();
-          if (row_ok) {
-#pragma unroll
-            for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r0[i]);
-            store32(p.out0 + obase + 32 * c, v);
-          }
-        }
-      }
+      epilogue_chunks<EPI, BN>(p, tc.n0, taddr, obase, row_ok, c_beg, NCH, pg, pu);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(tempty_bar + 8 * acc_stage);
@@ -674,67 +686,7 @@ tc_grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap mapA0, const __g
       if (!mbar_wait_cluster(tfull_bar + 8 * acc_stage, acc_phase, abort_flag)) { ok = false; break; }
       tc_fence_after();
       const uint32_t taddr = tmem_base + (uint32_t)(acc_stage * 256) + ((uint32_t)(32 * q) << 16);
-#pragma unroll 1
-      for (int c = c_beg; c < c_beg + NCH; ++c) {
-        if (tc.n0 + 32 * c >= p.N) break;
-        __syncwarp();
-        uint32_t r0[32];
-        float v[32];
-        tc_ld32(taddr + 32 * c, r0);
-        if (EPI == TC_EPI_SWIGLU) {
-          uint32_t r1[32];
-          tc_ld32(taddr + BN / 2 + 32 * c, r1);
-          tc_wait_ld();
-          if (row_ok) {
-            float hv[32];
-#pragma unroll
-            for (int i = 0; i < 32; ++i) {
-              const float g = __uint_as_float(r0[i]), u = __uint_as_float(r1[i]);
-              hv[i] = g / (1.0f + __expf(-g)) * u;
-              v[i] = g;
-            }
-            store32(p.out0 + obase + 32 * c, v);
-            store32(p.out2 + obase + 32 * c, hv);
-#pragma unroll
-            for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r1[i]);
-            store32(p.out1 + obase + 32 * c, v);
-          }
-        } else if (EPI == TC_EPI_DSWIGLU) {
-          uint4 cg[4], cu[4];
-#pragma unroll
-          for (int i = 0; i < 4; ++i) { cg[i] = pg[i]; cu[i] = pu[i]; }
-          if (row_ok && c + 1 < c_beg + NCH && tc.n0 + 32 * (c + 1) < p.N) {
-            const uint4* sg = reinterpret_cast<const uint4*>(p.in0 + obase + 32 * (c + 1));
-            const uint4* su = reinterpret_cast<const uint4*>(p.in1 + obase + 32 * (c + 1));
-#pragma unroll
-            for (int i = 0; i < 4; ++i) { pg[i] = sg[i]; pu[i] = su[i]; }
-          }
-          tc_wait_ld();
-          if (row_ok) {
-            float dg[32];
-#pragma unroll
-            for (int i = 0; i < 32; ++i) {
-              const uint32_t wg = reinterpret_cast<const uint32_t*>(cg)[i >> 1];
-              const uint32_t wu = reinterpret_cast<const uint32_t*>(cu)[i >> 1];
-              const float g = (i & 1) ? __uint_as_float(wg & 0xffff0000u) : __uint_as_float(wg << 16);
-              const float u = (i & 1) ? __uint_as_float(wu & 0xffff0000u) : __uint_as_float(wu << 16);
-              const float dh = __uint_as_float(r0[i]);
-              const float sgm = 1.0f / (1.0f + __expf(-g));
-              dg[i] = dh * u * sgm * (1.0f + g * (1.0f - sgm));
-              v[i] = dh * g * sgm;
-            }
-            store32(p.out0 + obase + 32 * c, dg);
-            store32(p.out1 + obase + 32 * c, v);
-          }
-        } else {
-          tc_wait_ld();
-          if (row_ok) {
-#pragma unroll
-            for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r0[i]);
-            store32(p.out0 + obase + 32 * c, v);
-          }
-        }
-      }
+      epilogue_chunks<EPI, BN>(p, tc.n0, taddr, obase, row_ok, c_beg, NCH, pg, pu);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(leader_tempty + 8 * acc_stage);
