@@ -85,9 +85,10 @@ def algorithmic_work(w, rows, kernel, unrouted=0):
         "csr_scan_kernel": (T * 8, "bytes"),
         "csr_fill_kernel": (T * E * 4 + rows * 4, "bytes"),
         "dispatch_kernel": (2 * rows * d * b, "bytes"),
-        "combine_kernel": (2 * (rows * d * b + T * d * b), "bytes"),       # combine + dispatch_bwd
+        "combine_kernel": (rows * d * b + T * d * b, "bytes"),
         "combine_bwd_kernel": (3 * rows * d * b, "bytes"),
         "affinity_bwd_dx_kernel": (3 * T_routed * d * b, "bytes"),
+        "affinity_bwd_dx_fused_kernel": (T_routed * d * b + rows * d * b + T * d * b, "bytes"),
         "affinity_bwd_dr_partial_kernel": (rows * m * 4, "bytes"),
         "affinity_bwd_dr_final_kernel": (E * m * 8, "bytes"),
         "gemm_simt_kernel": (18 * rows * d * h, "flops"),

@@ -237,7 +237,8 @@ etr_status etr_layer_forward(const etr_config* cfg, const void* X, const float* 
                              const etr_buffers* buf, void* Y, void* stream);
 
 /* combine_bwd, expert_ffn_bwd, dispatch_bwd, affinity_bwd, in that order, on the buffers
- * a preceding etr_layer_forward filled. */
+ * a preceding etr_layer_forward filled.  The last two run as one fused kernel (dX is written
+ * once, with the row sum kept in fp32 until the router term has been added). */
 etr_status etr_layer_backward(const etr_config* cfg, const void* X, const float* R,
                               const void* W1g, const void* W1u, const void* W2,
                               const void* dY, const etr_buffers* buf,

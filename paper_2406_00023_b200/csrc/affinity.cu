@@ -509,13 +509,16 @@ affinity_fwd_kernel(const T* __restrict__ X, const float* __restrict__ R, float*
 // ---- backward -----------------------------------------------------------------------------
 // dX[t,:] += cz[q/D] - beta x[t,:]  with  cz = sum_r (dgate_r sqrt(D)/(a b_i D)) R_i,
 // beta = sum_r dgate_r delta_ti / a^2 over the rows r of token t.  One warp per token.
-template <class T>
+// FUSED: dX is not read; the FFN path's gradient is gathered here from dXp (the backward of the
+// token rearrangement, dX[t] = sum of the token's rows of dXp), so dX is written exactly once.
+template <class T, bool FUSED>
 __global__ void __launch_bounds__(256)
 affinity_bwd_dx_kernel(const T* __restrict__ X, const float* __restrict__ R,
                        const float* __restrict__ delta, const float* __restrict__ xnorm,
                        const float* __restrict__ rnorm, const int32_t* __restrict__ tok_ptr,
                        const int32_t* __restrict__ tok_row, const float* __restrict__ dgate,
-                       T* __restrict__ dX, int Ttok, int d, int D, int E, int m, int C_stride) {
+                       const T* __restrict__ dXp, T* __restrict__ dX, int Ttok, int d, int D, int E,
+                       int m, int C_stride) {
   extern __shared__ __align__(16) float smem[];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   float* cz = smem + (size_t)warp * m;
@@ -523,27 +526,48 @@ affinity_bwd_dx_kernel(const T* __restrict__ X, const float* __restrict__ R,
   if (t >= Ttok) return;
   const int beg = tok_ptr[t], end = tok_ptr[t + 1];
   const float a = xnorm[t];
-  if (beg == end || a == 0.f) return;
+  T* g = dX + (size_t)t * d;
+  if (beg == end) {
+    if (FUSED)
+      for (int v = lane; v < d * (int)sizeof(T) / 16; v += 32) reinterpret_cast<uint4*>(g)[v] = make_uint4(0, 0, 0, 0);
+    return;
+  }
+  if (!FUSED && a == 0.f) return;
   for (int j = lane; j < m; j += 32) cz[j] = 0.f;
   float beta = 0.f;
   const float sqD = sqrtf((float)D);
-  for (int q = beg; q < end; ++q) {
-    const int r = tok_row[q], i = r / C_stride;
-    const float b = rnorm[i], dg = dgate[r];
-    if (b == 0.f) continue;
-    const float w = dg * sqD / (a * b) / (float)D;
-    beta += dg * delta[(size_t)t * E + i];
-    for (int j = lane; j < m; j += 32) cz[j] = fmaf(w, R[(size_t)i * m + j], cz[j]);
+  if (a != 0.f) {
+    for (int q = beg; q < end; ++q) {
+      const int r = tok_row[q], i = r / C_stride;
+      const float b = rnorm[i], dg = dgate[r];
+      if (b == 0.f) continue;
+      const float w = dg * sqD / (a * b) / (float)D;
+      beta += dg * delta[(size_t)t * E + i];
+      for (int j = lane; j < m; j += 32) cz[j] = fmaf(w, R[(size_t)i * m + j], cz[j]);
+    }
+    beta /= (a * a);
   }
-  beta /= (a * a);
   __syncwarp();
   const T* x = X + (size_t)t * d;
-  T* g = dX + (size_t)t * d;
   for (int v = lane; v < d / 8; v += 32) {
-    Vec8<T> xv = Vec8<T>::load(x + v * 8), gv = Vec8<T>::load(g + v * 8);
+    Vec8<T> xv = Vec8<T>::load(x + v * 8);
+    float base[8];
+    if (FUSED) {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) base[e] = 0.f;
+      for (int q = beg; q < end; ++q) {
+        Vec8<T> rv = Vec8<T>::load(dXp + (size_t)tok_row[q] * d + v * 8);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) base[e] += rv.v[e];
+      }
+    } else {
+      Vec8<T> gv = Vec8<T>::load(g + v * 8);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) base[e] = gv.v[e];
+    }
     float out[8];
 #pragma unroll
-    for (int e = 0; e < 8; ++e) out[e] = gv.v[e] + (cz[(v * 8 + e) / D] - beta * xv.v[e]);
+    for (int e = 0; e < 8; ++e) out[e] = base[e] + (cz[(v * 8 + e) / D] - beta * xv.v[e]);
     Vec8<T>::store(g + v * 8, out);
   }
 }
@@ -774,31 +798,44 @@ size_t affinity_bwd_workspace_bytes(const etr_config* c) {
   return (size_t)c->E * nch * (m + 1) * sizeof(float);
 }
 
+template <class T>
+static etr_status launch_bwd_dx(const etr_config* c, const void* X, const float* R, const float* delta,
+                                const float* xnorm, const float* rnorm, const etr_route* rt,
+                                const float* dgate, const void* dXp_fused, void* dX, size_t smem,
+                                cudaStream_t st) {
+  const int m = c->d / c->D, Cs = c_stride_of(c), grid = ceil_div(c->T, 8);
+  if (dXp_fused) {
+    auto k = affinity_bwd_dx_kernel<T, true>;
+    if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+      return ETR_ERR_CUDA;
+    ETR_TIME_BEGIN("affinity_bwd_dx_fused_kernel");
+    k<<<grid, 256, smem, st>>>((const T*)X, R, delta, xnorm, rnorm, rt->tok_ptr, rt->tok_row, dgate,
+                               (const T*)dXp_fused, (T*)dX, c->T, c->d, c->D, c->E, m, Cs);
+  } else {
+    auto k = affinity_bwd_dx_kernel<T, false>;
+    if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+      return ETR_ERR_CUDA;
+    ETR_TIME_BEGIN("affinity_bwd_dx_kernel");
+    k<<<grid, 256, smem, st>>>((const T*)X, R, delta, xnorm, rnorm, rt->tok_ptr, rt->tok_row, dgate,
+                               (const T*)nullptr, (T*)dX, c->T, c->d, c->D, c->E, m, Cs);
+  }
+  ETR_LAUNCH_CHECK();
+  return ETR_OK;
+}
+
+// dXp_fused != nullptr: dX is produced here in one pass (dispatch backward + router gradient)
 etr_status affinity_backward(const etr_config* c, const void* X, const float* R, const float* delta,
                              const float* Z, const float* xnorm, const float* rnorm,
-                             const etr_route* rt, const float* dgate, void* dX, float* dR,
-                             void* ws, cudaStream_t st) {
+                             const etr_route* rt, const float* dgate, const void* dXp_fused, void* dX,
+                             float* dR, void* ws, cudaStream_t st) {
   const int m = c->d / c->D, Cs = c_stride_of(c), nch = Cs / DR_CHUNK;
   if (m > 256 * DR_MAXJ) return ETR_ERR_UNSUPPORTED;
   const size_t smem = (size_t)8 * m * sizeof(float);
   if (smem > 200 * 1024) return ETR_ERR_UNSUPPORTED;
   const int grid = ceil_div(c->T, 8);
-  if (c->dtype == ETR_BF16) {
-    auto k = affinity_bwd_dx_kernel<__nv_bfloat16>;
-    if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-      return ETR_ERR_CUDA;
-    ETR_TIME_BEGIN("affinity_bwd_dx_kernel");
-    k<<<grid, 256, smem, st>>>((const __nv_bfloat16*)X, R, delta, xnorm, rnorm, rt->tok_ptr,
-                               rt->tok_row, dgate, (__nv_bfloat16*)dX, c->T, c->d, c->D, c->E, m, Cs);
-  } else {
-    auto k = affinity_bwd_dx_kernel<float>;
-    if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-      return ETR_ERR_CUDA;
-    ETR_TIME_BEGIN("affinity_bwd_dx_kernel");
-    k<<<grid, 256, smem, st>>>((const float*)X, R, delta, xnorm, rnorm, rt->tok_ptr, rt->tok_row,
-                               dgate, (float*)dX, c->T, c->d, c->D, c->E, m, Cs);
-  }
-  ETR_LAUNCH_CHECK();
+  ETR_TRY((c->dtype == ETR_BF16
+               ? launch_bwd_dx<__nv_bfloat16>(c, X, R, delta, xnorm, rnorm, rt, dgate, dXp_fused, dX, smem, st)
+               : launch_bwd_dx<float>(c, X, R, delta, xnorm, rnorm, rt, dgate, dXp_fused, dX, smem, st)));
   float* part = (float*)ws;
   ETR_TIME_BEGIN("affinity_bwd_dr_partial_kernel");
   affinity_bwd_dr_partial_kernel<<<dim3(c->E, nch), 256, 0, st>>>(

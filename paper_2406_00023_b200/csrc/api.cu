@@ -268,7 +268,7 @@ etr_status etr_affinity_bwd(const etr_config* c, const void* X, const float* R, 
   ETR_TRY(etr_validate(c));
   ETR_TRY(check_ptrs({X, R, delta, Z, xnorm, rnorm, dgate, dX, dR, ws}));
   ETR_TRY(check_route(route));
-  return affinity_backward(c, X, R, delta, Z, xnorm, rnorm, route, dgate, dX, dR, ws,
+  return affinity_backward(c, X, R, delta, Z, xnorm, rnorm, route, dgate, nullptr, dX, dR, ws,
                            (cudaStream_t)stream);
 }
 
@@ -295,10 +295,11 @@ etr_status etr_layer_backward(const etr_config* c, const void* X, const float* R
   ETR_TRY(etr_combine_bwd(c, &b->route, dY, b->O, b->dO, b->dgate, stream));
   ETR_TRY(etr_expert_ffn_bwd(c, &b->route, b->dO, b->Xp, b->G, b->U, b->H, W1g, W1u, W2, b->dG, b->dU,
                              b->dXp, dW1g, dW1u, dW2, b->stats, b->ws, stream));
-  ETR_TRY(etr_dispatch_bwd(c, &b->route, b->dXp, dX, stream));
+  // dispatch backward and the router gradient in one pass over dX
   ETR_TRY(etr_select_bwd(c, &b->route, b->dgate));
-  return etr_affinity_bwd(c, X, R, b->delta, b->Z, b->xnorm, b->rnorm, &b->route, b->dgate, dX, dR,
-                          b->ws, stream);
+  ETR_TRY(check_ptrs({X, R, dX, dR, b->dXp, b->ws}));
+  return affinity_backward(c, X, R, b->delta, b->Z, b->xnorm, b->rnorm, &b->route, b->dgate, b->dXp, dX,
+                           dR, b->ws, (cudaStream_t)stream);
 }
 
 // Side streams and events for the host-buffer step (host-side objects, created once per device).

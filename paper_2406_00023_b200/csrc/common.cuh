@@ -112,8 +112,8 @@ etr_status affinity_forward(const etr_config* c, const void* X, const float* R, 
 size_t affinity_bwd_workspace_bytes(const etr_config* c);
 etr_status affinity_backward(const etr_config* c, const void* X, const float* R, const float* delta,
                              const float* Z, const float* xnorm, const float* rnorm,
-                             const etr_route* rt, const float* dgate, void* dX, float* dR, void* ws,
-                             cudaStream_t st);
+                             const etr_route* rt, const float* dgate, const void* dXp_fused, void* dX,
+                             float* dR, void* ws, cudaStream_t st);
 size_t select_workspace_bytes(const etr_config* c);
 int resolve_mode(const etr_config* c);
 etr_status select_forward(const etr_config* c, const float* delta, etr_stats* stats,

@@ -299,6 +299,41 @@ def test_layer_is_deterministic_and_host_step_matches():
         assert torch.equal(a[k].cpu(), c[k].cpu()), k
 
 
+@pytest.mark.parametrize("name", ["tiny", "small_s", "mid_s"])
+def test_stage_calls_compose_to_the_layer_calls(name):
+    """The ten stage entry points called one by one give what etr_layer_forward/backward give.
+    Only dX may differ, by one rounding: the layer call fuses the dispatch backward into the
+    router-gradient kernel and keeps the row sum in fp32, the stage path stores it first."""
+    w, inp, o, fw, bw = case(name)
+    cfg = hz.make_cfg(w)
+    dev = hz.upload(w, inp)
+    _, ref = run_layer(w, inp, cfg)
+    buf = etr.LayerBuffers(cfg)
+    ws = torch.empty(etr.workspace_bytes(cfg), dtype=torch.uint8, device="cuda")
+    out = {k: torch.empty_like(v) for k, v in ref.items()}
+    buf.stats.zero_()
+    etr.affinity(cfg, dev.X, dev.R, buf.delta, buf.Z, buf.xnorm, buf.rnorm, buf.c.stats)
+    etr.select(cfg, buf.delta, buf.c.stats, buf.route, ws)
+    etr.dispatch(cfg, dev.X, buf.route, buf.Xp)
+    etr.expert_ffn(cfg, buf.route, buf.Xp, dev.W1g, dev.W1u, dev.W2, buf.G, buf.U, buf.H, buf.O, buf.c.stats, ws)
+    etr.combine(cfg, buf.route, buf.O, out["Y"])
+    etr.combine_bwd(cfg, buf.route, dev.dY, buf.O, buf.dO, buf.dgate)
+    etr.expert_ffn_bwd(cfg, buf.route, buf.dO, buf.Xp, buf.G, buf.U, buf.H, dev.W1g, dev.W1u, dev.W2,
+                       buf.dG, buf.dU, buf.dXp, out["dW1g"], out["dW1u"], out["dW2"], buf.c.stats, ws)
+    etr.dispatch_bwd(cfg, buf.route, buf.dXp, out["dX"])
+    etr.select_bwd(cfg, buf.route, buf.dgate)
+    etr.affinity_bwd(cfg, dev.X, dev.R, buf.delta, buf.Z, buf.xnorm, buf.rnorm, buf.route, buf.dgate,
+                     out["dX"], out["dR"], ws)
+    torch.cuda.synchronize()
+    for k in ("Y", "dR", "dW1g", "dW1u", "dW2"):
+        assert torch.equal(out[k], ref[k]), k
+    a, b = hz.to_np(out["dX"]), hz.to_np(ref["dX"])
+    if w.dtype == "bf16":      # one extra bf16 rounding of a sum that may cancel
+        hz.assert_close_rms(a, b, 1e-2, "dX (stage path vs fused)", chain=2)
+    else:
+        assert np.allclose(a, b, rtol=1e-6, atol=1e-7)
+
+
 def test_argument_errors_are_reported_without_launching():
     import ctypes as C
     w = CASES["tiny"]
