@@ -156,13 +156,39 @@ __device__ __forceinline__ void load32(const __nv_bfloat16* src, float* v) {
 
 struct TileCoord { int e, m0, n0, kblocks, m_lim; };
 
+// Warp-cooperative store of a 32-row x 32-column bf16 block whose row `lane` is held by lane
+// `lane` as 32 floats.  Written directly, every store instruction would touch 32 rows with 16
+// bytes each (half a sector per row).  Instead the block is turned in a per-warp shared-memory
+// scratch (32 rows x 80 bytes: the 16-byte pad makes both phases bank-conflict free) so that an
+// instruction writes 8 rows x 64 contiguous bytes: whole sectors, half as many of them.
+constexpr int TC_SCRATCH_ROW_BYTES = 80;
+constexpr int TC_SCRATCH_BYTES = 32 * TC_SCRATCH_ROW_BYTES;      // per epilogue warp
+__device__ __forceinline__ void store32_warp(uint8_t* scratch, int lane, int nvalid, __nv_bfloat16* dst,
+                                             int ld_out, const float* v) {
+  uint4* mine = reinterpret_cast<uint4*>(scratch + lane * TC_SCRATCH_ROW_BYTES);
+#pragma unroll
+  for (int q = 0; q < 4; ++q)
+    mine[q] = make_uint4(pack_bf16(v[8 * q], v[8 * q + 1]), pack_bf16(v[8 * q + 2], v[8 * q + 3]),
+                         pack_bf16(v[8 * q + 4], v[8 * q + 5]), pack_bf16(v[8 * q + 6], v[8 * q + 7]));
+  __syncwarp();
+  const int sub = lane & 3;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int row = (lane >> 2) + 8 * i;
+    const uint4 w = *reinterpret_cast<const uint4*>(scratch + row * TC_SCRATCH_ROW_BYTES + sub * 16);
+    if (row < nvalid) *reinterpret_cast<uint4*>(dst + (long long)row * ld_out + sub * 8) = w;
+  }
+  __syncwarp();
+}
+
 // The epilogue of one accumulator tile for one warp: `nch` chunks of 32 columns starting at
 // chunk c_beg, read from tensor memory at taddr and stored (or fused with SwiGLU / its
 // derivative) at row offset obase.  pg/pu hold the prefetched G and U of the first chunk.
 template <int EPI, int BN>
 __device__ __forceinline__ void epilogue_chunks(const TcParams& p, int n0, uint32_t taddr, long long obase,
                                                 bool row_ok, int c_beg, int nch, uint4 (&pg)[4],
-                                                uint4 (&pu)[4]) {
+                                                uint4 (&pu)[4], uint8_t* scratch, int lane, int nvalid) {
+  const long long wbase = obase - (long long)lane * p.ld_out;     // row 0 of this warp's 32 rows
 #pragma unroll 1
   for (int c = c_beg; c < c_beg + nch; ++c) {
     if (n0 + 32 * c >= p.N) break;
@@ -174,20 +200,18 @@ __device__ __forceinline__ void epilogue_chunks(const TcParams& p, int n0, uint3
       uint32_t r1[32];
       tc_ld32(taddr + BN / 2 + 32 * c, r1);
       tc_wait_ld();
-      if (row_ok) {
-        float hv[32];
+      float hv[32];
 #pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          const float g = __uint_as_float(r0[i]), u = __uint_as_float(r1[i]);
-          hv[i] = __fdividef(g, 1.0f + __expf(-g)) * u;
-          v[i] = g;
-        }
-        store32(p.out0 + obase + 32 * c, v);
-        store32(p.out2 + obase + 32 * c, hv);
-#pragma unroll
-        for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r1[i]);
-        store32(p.out1 + obase + 32 * c, v);
+      for (int i = 0; i < 32; ++i) {
+        const float g = __uint_as_float(r0[i]), u = __uint_as_float(r1[i]);
+        hv[i] = __fdividef(g, 1.0f + __expf(-g)) * u;
+        v[i] = g;
       }
+      store32_warp(scratch, lane, nvalid, p.out0 + wbase + 32 * c, p.ld_out, v);
+      store32_warp(scratch, lane, nvalid, p.out2 + wbase + 32 * c, p.ld_out, hv);
+#pragma unroll
+      for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r1[i]);
+      store32_warp(scratch, lane, nvalid, p.out1 + wbase + 32 * c, p.ld_out, v);
     } else if (EPI == TC_EPI_DSWIGLU) {
       uint4 cg[4], cu[4];
 #pragma unroll
@@ -199,7 +223,11 @@ __device__ __forceinline__ void epilogue_chunks(const TcParams& p, int n0, uint3
         for (int i = 0; i < 4; ++i) { pg[i] = sg[i]; pu[i] = su[i]; }
       }
       tc_wait_ld();
-      if (row_ok) {
+      if (!row_ok) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) { cg[i] = make_uint4(0, 0, 0, 0); cu[i] = make_uint4(0, 0, 0, 0); }
+      }
+      {
         float dg[32];
 #pragma unroll
         for (int i = 0; i < 32; ++i) {
@@ -212,16 +240,14 @@ __device__ __forceinline__ void epilogue_chunks(const TcParams& p, int n0, uint3
           dg[i] = dh * u * sgm * (1.0f + g * (1.0f - sgm));
           v[i] = dh * g * sgm;
         }
-        store32(p.out0 + obase + 32 * c, dg);
-        store32(p.out1 + obase + 32 * c, v);
+        store32_warp(scratch, lane, nvalid, p.out0 + wbase + 32 * c, p.ld_out, dg);
+        store32_warp(scratch, lane, nvalid, p.out1 + wbase + 32 * c, p.ld_out, v);
       }
     } else {
       tc_wait_ld();
-      if (row_ok) {
 #pragma unroll
-        for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r0[i]);
-        store32(p.out0 + obase + 32 * c, v);
-      }
+      for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r0[i]);
+      store32_warp(scratch, lane, nvalid, p.out0 + wbase + 32 * c, p.ld_out, v);
     }
   }
 }
@@ -375,6 +401,7 @@ tc_grouped_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_c
   } else {
     // ---- epilogue warps ---------------------------------------------------------------------------
     const int q = warp & 3;                        // quarter of tensor memory this warp may read
+    uint8_t* scratch = smem_raw + (tiles_base - smem_u32(smem_raw)) + TC_STAGES * STAGE_BYTES + (warp - 2) * TC_SCRATCH_BYTES;
     const int half = (warp - 2) >> 2;              // which half of the tile's columns it handles
     constexpr int NCH = N_TILE_COLS / 32 / 2;      // 32-column chunks per warp
     const int row_in_tile = 32 * q + lane;
@@ -408,7 +435,8 @@ tc_grouped_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_c
       if (!mbar_wait(tfull_bar + 8 * acc_stage, acc_phase, abort_flag)) { ok = false; break; }
       tc_fence_after();
       const uint32_t taddr = tmem_base + (uint32_t)(acc_stage * 256) + ((uint32_t)(32 * q) << 16);
-      epilogue_chunks<EPI, BN>(p, tc.n0, taddr, obase, row_ok, c_beg, NCH, pg, pu);
+      epilogue_chunks<EPI, BN>(p, tc.n0, taddr, obase, row_ok, c_beg, NCH, pg, pu, scratch, lane,
+                               min(32, max(0, tc.m_lim - (grow - lane))));
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(tempty_bar + 8 * acc_stage);
@@ -655,6 +683,7 @@ tc_grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap mapA0, const __g
   } else {
     // ---- epilogue warps (both CTAs, own 128 rows) -----------------------------------------------------
     const int q = warp & 3;
+    uint8_t* scratch = smem_raw + (tiles_base - smem_u32(smem_raw)) + TC2_STAGES * TC2_STAGE_BYTES + (warp - 2) * TC_SCRATCH_BYTES;
     const int half = (warp - 2) >> 2;
     constexpr int NCH = N_TILE_COLS / 32 / 2;
     const int row_in_tile = 128 * (int)rank + 32 * q + lane;
@@ -686,7 +715,8 @@ tc_grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap mapA0, const __g
       if (!mbar_wait_cluster(tfull_bar + 8 * acc_stage, acc_phase, abort_flag)) { ok = false; break; }
       tc_fence_after();
       const uint32_t taddr = tmem_base + (uint32_t)(acc_stage * 256) + ((uint32_t)(32 * q) << 16);
-      epilogue_chunks<EPI, BN>(p, tc.n0, taddr, obase, row_ok, c_beg, NCH, pg, pu);
+      epilogue_chunks<EPI, BN>(p, tc.n0, taddr, obase, row_ok, c_beg, NCH, pg, pu, scratch, lane,
+                               min(32, max(0, tc.m_lim - (grow - lane))));
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(leader_tempty + 8 * acc_stage);
@@ -770,7 +800,7 @@ template <int BN, int EPI>
 static etr_status tc_launch(const char* name, const CUtensorMap& a0, const CUtensorMap& a1,
                             const CUtensorMap& b0, const CUtensorMap& b1, TcParams p, int max_tiles,
                             cudaStream_t st) {
-  constexpr size_t smem = (size_t)TC_STAGES * (2 + BN / 64) * TC_BOX_BYTES + 1024;
+  constexpr size_t smem = (size_t)TC_STAGES * (2 + BN / 64) * TC_BOX_BYTES + 1024 + 8 * TC_SCRATCH_BYTES;
   auto k = tc_grouped_gemm_kernel<BN, EPI>;
   static bool attr_set = false;
   if (!attr_set) {
@@ -790,7 +820,7 @@ template <int EPI>
 static etr_status tc_launch_pair(const char* name, const CUtensorMap& a0, const CUtensorMap& a1,
                                  const CUtensorMap& b0, const CUtensorMap& b1, TcParams p, int max_tiles,
                                  cudaStream_t st) {
-  constexpr size_t smem = (size_t)TC2_STAGES * TC2_STAGE_BYTES + 1024;
+  constexpr size_t smem = (size_t)TC2_STAGES * TC2_STAGE_BYTES + 1024 + 8 * TC_SCRATCH_BYTES;
   auto k = tc_grouped_gemm_pair_kernel<EPI>;
   static bool attr_set = false;
   if (!attr_set) {

@@ -12,7 +12,7 @@ import os
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libetr.so")
+LIB_PATH = os.environ.get("ETR_LIB_PATH") or os.path.join(_HERE, "libetr.so")   # override: another build of the library
 
 OK, ERR_ARG, ERR_SHAPE, ERR_ALIGN, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_UNSUPPORTED = range(8)
 F32, BF16 = 0, 1
