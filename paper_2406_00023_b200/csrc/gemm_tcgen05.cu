@@ -181,6 +181,31 @@ __device__ __forceinline__ void store32_warp(uint8_t* scratch, int lane, int nva
   __syncwarp();
 }
 
+// The reverse turn for the saved activations the SwiGLU derivative reads: fetched as 8 rows x
+// 64 contiguous bytes per instruction (regs `t`), later handed to the lane that owns the row.
+__device__ __forceinline__ void load32_warp_issue(const __nv_bfloat16* src, int ld, int lane, int nvalid,
+                                                  uint4 (&t)[4]) {
+  const int sub = lane & 3;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int row = (lane >> 2) + 8 * i;
+    t[i] = row < nvalid ? *reinterpret_cast<const uint4*>(src + (long long)row * ld + sub * 8)
+                        : make_uint4(0, 0, 0, 0);
+  }
+}
+__device__ __forceinline__ void load32_warp_turn(uint8_t* scratch, int lane, const uint4 (&t)[4],
+                                                 uint4 (&mine)[4]) {
+  const int sub = lane & 3;
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+    *reinterpret_cast<uint4*>(scratch + ((lane >> 2) + 8 * i) * TC_SCRATCH_ROW_BYTES + sub * 16) = t[i];
+  __syncwarp();
+#pragma unroll
+  for (int q = 0; q < 4; ++q)
+    mine[q] = *reinterpret_cast<const uint4*>(scratch + lane * TC_SCRATCH_ROW_BYTES + q * 16);
+  __syncwarp();
+}
+
 // The epilogue of one accumulator tile for one warp: `nch` chunks of 32 columns starting at
 // chunk c_beg, read from tensor memory at taddr and stored (or fused with SwiGLU / its
 // derivative) at row offset obase.  pg/pu hold the prefetched G and U of the first chunk.
@@ -214,19 +239,13 @@ __device__ __forceinline__ void epilogue_chunks(const TcParams& p, int n0, uint3
       store32_warp(scratch, lane, nvalid, p.out1 + wbase + 32 * c, p.ld_out, v);
     } else if (EPI == TC_EPI_DSWIGLU) {
       uint4 cg[4], cu[4];
-#pragma unroll
-      for (int i = 0; i < 4; ++i) { cg[i] = pg[i]; cu[i] = pu[i]; }
-      if (row_ok && c + 1 < c_beg + nch && n0 + 32 * (c + 1) < p.N) {
-        const uint4* sg = reinterpret_cast<const uint4*>(p.in0 + obase + 32 * (c + 1));
-        const uint4* su = reinterpret_cast<const uint4*>(p.in1 + obase + 32 * (c + 1));
-#pragma unroll
-        for (int i = 0; i < 4; ++i) { pg[i] = sg[i]; pu[i] = su[i]; }
+      load32_warp_turn(scratch, lane, pg, cg);
+      load32_warp_turn(scratch, lane, pu, cu);
+      if (c + 1 < c_beg + nch && n0 + 32 * (c + 1) < p.N) {
+        load32_warp_issue(p.in0 + wbase + 32 * (c + 1), p.ld_out, lane, nvalid, pg);
+        load32_warp_issue(p.in1 + wbase + 32 * (c + 1), p.ld_out, lane, nvalid, pu);
       }
       tc_wait_ld();
-      if (!row_ok) {
-#pragma unroll
-        for (int i = 0; i < 4; ++i) { cg[i] = make_uint4(0, 0, 0, 0); cu[i] = make_uint4(0, 0, 0, 0); }
-      }
       {
         float dg[32];
 #pragma unroll
@@ -426,17 +445,16 @@ tc_grouped_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_c
       // SwiGLU derivative: the saved G and U of the first chunk are fetched before the
       // accumulator is ready, those of chunk c+1 while chunk c is processed
       uint4 pg[4], pu[4];
-      if (EPI == TC_EPI_DSWIGLU && row_ok && tc.n0 + 32 * c_beg < p.N) {
-        const uint4* sg = reinterpret_cast<const uint4*>(p.in0 + obase + 32 * c_beg);
-        const uint4* su = reinterpret_cast<const uint4*>(p.in1 + obase + 32 * c_beg);
-#pragma unroll
-        for (int i = 0; i < 4; ++i) { pg[i] = sg[i]; pu[i] = su[i]; }
+      const int nvalid = min(32, max(0, tc.m_lim - (grow - lane)));
+      if (EPI == TC_EPI_DSWIGLU && tc.n0 + 32 * c_beg < p.N) {
+        const long long wb = obase - (long long)lane * p.ld_out + 32 * c_beg;
+        load32_warp_issue(p.in0 + wb, p.ld_out, lane, nvalid, pg);
+        load32_warp_issue(p.in1 + wb, p.ld_out, lane, nvalid, pu);
       }
       if (!mbar_wait(tfull_bar + 8 * acc_stage, acc_phase, abort_flag)) { ok = false; break; }
       tc_fence_after();
       const uint32_t taddr = tmem_base + (uint32_t)(acc_stage * 256) + ((uint32_t)(32 * q) << 16);
-      epilogue_chunks<EPI, BN>(p, tc.n0, taddr, obase, row_ok, c_beg, NCH, pg, pu, scratch, lane,
-                               min(32, max(0, tc.m_lim - (grow - lane))));
+      epilogue_chunks<EPI, BN>(p, tc.n0, taddr, obase, row_ok, c_beg, NCH, pg, pu, scratch, lane, nvalid);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(tempty_bar + 8 * acc_stage);
@@ -706,17 +724,16 @@ tc_grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap mapA0, const __g
         continue;
       }
       uint4 pg[4], pu[4];
-      if (EPI == TC_EPI_DSWIGLU && row_ok && tc.n0 + 32 * c_beg < p.N) {
-        const uint4* sg = reinterpret_cast<const uint4*>(p.in0 + obase + 32 * c_beg);
-        const uint4* su = reinterpret_cast<const uint4*>(p.in1 + obase + 32 * c_beg);
-#pragma unroll
-        for (int i = 0; i < 4; ++i) { pg[i] = sg[i]; pu[i] = su[i]; }
+      const int nvalid = min(32, max(0, tc.m_lim - (grow - lane)));
+      if (EPI == TC_EPI_DSWIGLU && tc.n0 + 32 * c_beg < p.N) {
+        const long long wb = obase - (long long)lane * p.ld_out + 32 * c_beg;
+        load32_warp_issue(p.in0 + wb, p.ld_out, lane, nvalid, pg);
+        load32_warp_issue(p.in1 + wb, p.ld_out, lane, nvalid, pu);
       }
       if (!mbar_wait_cluster(tfull_bar + 8 * acc_stage, acc_phase, abort_flag)) { ok = false; break; }
       tc_fence_after();
       const uint32_t taddr = tmem_base + (uint32_t)(acc_stage * 256) + ((uint32_t)(32 * q) << 16);
-      epilogue_chunks<EPI, BN>(p, tc.n0, taddr, obase, row_ok, c_beg, NCH, pg, pu, scratch, lane,
-                               min(32, max(0, tc.m_lim - (grow - lane))));
+      epilogue_chunks<EPI, BN>(p, tc.n0, taddr, obase, row_ok, c_beg, NCH, pg, pu, scratch, lane, nvalid);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(leader_tempty + 8 * acc_stage);
