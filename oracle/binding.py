@@ -137,6 +137,14 @@ class Oracle:
                               _p(W2), _p(G), _p(U), _p(H), _p(O))
         return G, U, H, O
 
+    def expert_ffn_down(self, H, route, W2):
+        """O = H W2_i^T alone (the second half of the FFN on a given hidden activation)."""
+        H, W2 = self.arr(H), self.arr(W2)
+        E, d, h = W2.shape
+        O = np.empty((E * route.C_stride, d), self.np)
+        self._f("expert_ffn_down")(E, route.C_stride, d, h, _p(route.counts), _p(H), _p(W2), _p(O))
+        return O
+
     def combine(self, O, route, gate=None):
         O = self.arr(O)
         gate = self.arr(route.gate if gate is None else gate)

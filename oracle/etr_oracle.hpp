@@ -195,6 +195,29 @@ void ffn_row(int d, int h, const S* x, const S* W1g, const S* W1u, const S* W2,
   }
 }
 
+// Second half of ffn_row on its own: o = W2 hh for a given hidden activation (used to model a
+// pipeline that stores hh in a narrower type between the two halves).
+template <class S>
+void ffn_down_row(int d, int h, const S* hh, const S* W2, S* o) {
+  for (int a = 0; a < d; ++a) {
+    double acc = 0.0;
+    const S* w = W2 + (size_t)a * h;
+    for (int b = 0; b < h; ++b) acc += (double)w[b] * (double)hh[b];
+    o[a] = (S)acc;
+  }
+}
+
+template <class S>
+void expert_ffn_down(int E, int C_stride, int d, int h, const int32_t* counts, const S* H, const S* W2, S* O) {
+#pragma omp parallel for schedule(dynamic, 8)
+  for (long r = 0; r < (long)E * C_stride; ++r) {
+    const int i = (int)(r / C_stride), p = (int)(r % C_stride);
+    S* o = O + (size_t)r * d;
+    if (p < counts[i]) ffn_down_row(d, h, H + (size_t)r * h, W2 + (size_t)i * d * h, o);
+    else std::fill(o, o + d, (S)0);
+  }
+}
+
 // All experts: rows p < counts[i] of expert i; other rows of G,U,H,O are set to zero.
 template <class S>
 void expert_ffn(int E, int C_stride, int d, int h, const int32_t* counts, const S* Xp,

@@ -33,6 +33,11 @@ using namespace etr_oracle;
                                               const S* W1u, const S* W2, S* G, S* U, S* H, S* O) {   \
     expert_ffn<S>(E, C_stride, d, h, counts, Xp, W1g, W1u, W2, G, U, H, O);                          \
   }                                                                                                  \
+  extern "C" void etr_oracle_expert_ffn_down_##SUF(int E, int C_stride, int d, int h,                \
+                                                   const int32_t* counts, const S* H, const S* W2,   \
+                                                   S* O) {                                           \
+    expert_ffn_down<S>(E, C_stride, d, h, counts, H, W2, O);                                         \
+  }                                                                                                  \
   extern "C" void etr_oracle_combine_##SUF(int T, int d, const int32_t* tok_ptr,                     \
                                            const int32_t* tok_row, const S* gate, const S* O,        \
                                            S* Y) {                                                   \

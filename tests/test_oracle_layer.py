@@ -162,6 +162,16 @@ def test_router_gradient_orthogonality(o64):
     assert np.allclose((bw.dR * p["R"]).sum(1), 0, atol=1e-12)
 
 
+def test_ffn_down_is_the_second_half_of_the_ffn(o64):
+    p = problem(8)
+    fw = o64.forward(p["X"], p["R"], p["W1g"], p["W1u"], p["W2"], D=2, k=2, capacity=6, mode=ob.MODE_TCR)
+    assert np.array_equal(o64.expert_ffn_down(fw.H, fw.route, p["W2"]), fw.O)
+    t = torch.from_numpy
+    r = int(np.nonzero(fw.route.slot_token >= 0)[0][3])
+    e = r // fw.route.C_stride
+    assert np.allclose(fw.O[r], (t(p["W2"][e]) @ t(fw.H[r])).numpy(), rtol=1e-13, atol=1e-14)
+
+
 def test_f32_layer_close_to_f64(o32, o64):
     w = gw.scaled(gw.WORKLOADS["tiny"], T=128, h=64)
     inp = gw.make_inputs(w)
