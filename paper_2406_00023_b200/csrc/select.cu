@@ -99,15 +99,49 @@ select_token_side_kernel(const float* __restrict__ delta, int32_t* __restrict__ 
   }
 }
 
-// Histogram add with warp aggregation: lanes holding the same digit elect one leader that
-// adds their number.  Affinity keys share their top bits, so the unaggregated form would
-// serialise on a handful of bins.
-__device__ __forceinline__ void hist_add(uint32_t* hist, uint32_t digit, bool active) {
-  const uint32_t amask = __ballot_sync(0xffffffffu, active);
-  if (active) {
-    const uint32_t peers = __match_any_sync(amask, digit);
-    if ((threadIdx.x & 31) == (uint32_t)(__ffs(peers) - 1)) atomicAdd(&hist[digit], (uint32_t)__popc(peers));
+// Histogram add.  In the first pass (top byte) affinity keys share their top bits and plain
+// atomics would serialise on a handful of bins, so lanes holding the same digit elect one
+// leader that adds their number.
+__device__ __forceinline__ void hist_add(uint32_t* hist, uint32_t digit, bool active, bool aggregate) {
+  if (aggregate) {
+    const uint32_t amask = __ballot_sync(0xffffffffu, active);
+    if (active) {
+      const uint32_t peers = __match_any_sync(amask, digit);
+      if ((threadIdx.x & 31) == (uint32_t)(__ffs(peers) - 1)) atomicAdd(&hist[digit], (uint32_t)__popc(peers));
+    }
+  } else if (active) {
+    atomicAdd(&hist[digit], 1u);      // later passes: few keys match the prefix and their digits spread
   }
+}
+
+// Radix step by one warp: walking the 256 bins from the top, the first bin whose count reaches
+// `rem` (bin 0 takes whatever is left); rem is reduced by the counts of the bins above it.
+// Lane l owns bins 255-8l .. 248-8l.  The result is returned in every lane.
+__device__ __forceinline__ void pick_bin(const uint32_t* hist, uint32_t rem, int lane, uint32_t& bin,
+                                         uint32_t& rem_out) {
+  uint32_t c[8], mine = 0;
+#pragma unroll
+  for (int u = 0; u < 8; ++u) { c[u] = hist[255 - 8 * lane - u]; mine += c[u]; }
+  uint32_t inc = mine;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const uint32_t y = __shfl_up_sync(0xffffffffu, inc, o);
+    if (lane >= o) inc += y;
+  }
+  const uint32_t hit = __ballot_sync(0xffffffffu, inc >= rem || lane == 31);
+  const int owner = __ffs(hit) - 1;
+  uint32_t b = 0, r = rem - (inc - mine);
+  if (lane == owner) {
+    int u = 0;
+    for (; u < 8; ++u) {
+      const int idx = 255 - 8 * lane - u;
+      if (idx == 0 || c[u] >= r) break;
+      r -= c[u];
+    }
+    b = (uint32_t)(255 - 8 * lane - u);
+  }
+  bin = __shfl_sync(0xffffffffu, b, owner);
+  rem_out = __shfl_sync(0xffffffffu, r, owner);
 }
 
 // One CTA (1024 threads) per expert; every thread owns 4 consecutive tokens per sweep.
@@ -152,7 +186,7 @@ select_expert_side_kernel(uint32_t* __restrict__ keyT, const etr_stats* __restri
         const uint32_t kx = cur[u];
         const bool in_range = c0 + tid * SEL_KPT + u < T;
         nc += (in_range && kx != 0u);
-        hist_add(hist, (kx >> shift) & 0xffu, in_range && (kx & pmask) == prefix);
+        hist_add(hist, (kx >> shift) & 0xffu, in_range && (kx & pmask) == prefix, pass == 0);
       }
 #pragma unroll
       for (int u = 0; u < SEL_KPT; ++u) cur[u] = nxt[u];
@@ -164,15 +198,13 @@ select_expert_side_kernel(uint32_t* __restrict__ keyT, const etr_stats* __restri
     __syncthreads();
     if (pass == 0) n_keep = min((uint32_t)C, s_ncand);
     if (n_keep == 0) break;                       // uniform across the CTA
-    if (tid == 0) {
-      uint32_t rem = pass == 0 ? n_keep : s_remaining;
-      int b = 255;
-      for (; b > 0; --b) {
-        if (hist[b] >= rem) break;
-        rem -= hist[b];
+    if (warp == 0) {
+      uint32_t b, rem;
+      pick_bin(hist, pass == 0 ? n_keep : s_remaining, lane, b, rem);
+      if (lane == 0) {
+        s_prefix = prefix | (b << shift);
+        s_remaining = rem;      // after the last pass: how many keys == tau are admitted
       }
-      s_prefix = prefix | ((uint32_t)b << shift);
-      s_remaining = rem;        // after the last pass: how many keys == tau are admitted
     }
     __syncthreads();
   }
@@ -249,6 +281,203 @@ select_expert_side_kernel(uint32_t* __restrict__ keyT, const etr_stats* __restri
   }
   for (int p = (int)n_keep + tid; p < C_stride; p += 1024) { my_slot[p] = -1; my_gate[p] = 0.f; }
   if (tid == 0) counts[i] = (int)n_keep;
+}
+
+// The same selection with an expert's row of keys split over a thread-block cluster of CL CTAs
+// (large T: one CTA per expert leaves most SMs idle and walks 64 Ki keys five times).  Each CTA
+// histograms its own quarter of the tokens; the CL histograms are added through distributed
+// shared memory after a hardware cluster barrier, so every CTA takes the same radix decision;
+// the slot positions of a CTA start after the kept tokens of the lower-ranked CTAs.
+__device__ __forceinline__ uint32_t sel_cluster_rank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void sel_cluster_sync() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t sel_peer_load(const uint32_t* local, uint32_t rank) {
+  uint32_t a = (uint32_t)__cvta_generic_to_shared(local), ra, v;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"(a), "r"(rank));
+  asm volatile("ld.shared::cluster.u32 %0, [%1];" : "=r"(v) : "r"(ra) : "memory");
+  return v;
+}
+
+template <int CL>
+__global__ void __launch_bounds__(1024)
+select_expert_side_cluster_kernel(uint32_t* __restrict__ keyT, const etr_stats* __restrict__ stats,
+                                  int32_t* __restrict__ counts, int32_t* __restrict__ slot_token,
+                                  float* __restrict__ gate, int T, int C_stride) {
+  __shared__ uint32_t hist[256], tot[256];
+  __shared__ uint32_t s_prefix, s_remaining, s_ncand_local, s_ncand;
+  __shared__ uint32_t s_cnt_gt, s_cnt_eq;
+  __shared__ uint32_t warp_tot[32], warp_pre[32];
+  __shared__ uint32_t base_sel, base_eq;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const uint32_t rank = sel_cluster_rank();
+  const int i = blockIdx.x / CL;
+  const int span = ((T + CL - 1) / CL + SEL_KPT - 1) / SEL_KPT * SEL_KPT;
+  const int t_beg = min(T, (int)rank * span), t_end = min(T, t_beg + span);
+  uint32_t* row = keyT + (size_t)i * T;
+  int32_t* my_slot = slot_token + (size_t)i * C_stride;
+  float* my_gate = gate + (size_t)i * C_stride;
+  const int C = stats->C;
+
+  // this CTA's keys are read from global memory once and stay in shared memory for every pass
+  extern __shared__ uint32_t sk[];
+  for (int t = t_beg + tid; t < t_end; t += 1024) sk[t - t_beg] = row[t];
+  const uint32_t* rowl = sk - t_beg;              // rowl[t] for t in [t_beg, t_end)
+
+  uint32_t tau = 0, quota = 0, n_keep = 0;
+  if (tid == 0) { s_prefix = 0; s_ncand_local = 0; s_cnt_gt = 0; s_cnt_eq = 0; }
+  for (int pass = 0; pass < 4; ++pass) {
+    const int shift = 24 - 8 * pass;
+    if (tid < 256) hist[tid] = 0;
+    __syncthreads();
+    const uint32_t prefix = s_prefix;
+    const uint32_t pmask = pass == 0 ? 0u : (0xffffffffu << (shift + 8));
+    uint32_t nc = 0;
+    uint32_t cur[SEL_KPT], nxt[SEL_KPT];
+    load_keys(rowl, t_beg + tid * SEL_KPT, t_end, cur);
+    for (int c0 = t_beg; c0 < t_end; c0 += SEL_SWEEP) {
+      if (c0 + SEL_SWEEP < t_end) load_keys(rowl, c0 + SEL_SWEEP + tid * SEL_KPT, t_end, nxt);
+#pragma unroll
+      for (int u = 0; u < SEL_KPT; ++u) {
+        const uint32_t kx = cur[u];
+        const bool in_range = c0 + tid * SEL_KPT + u < t_end;
+        nc += (in_range && kx != 0u);
+        hist_add(hist, (kx >> shift) & 0xffu, in_range && (kx & pmask) == prefix, pass == 0);
+      }
+#pragma unroll
+      for (int u = 0; u < SEL_KPT; ++u) cur[u] = nxt[u];
+    }
+    if (pass == 0) {
+      for (int o = 16; o > 0; o >>= 1) nc += __shfl_xor_sync(0xffffffffu, nc, o);
+      if (lane == 0 && nc) atomicAdd(&s_ncand_local, nc);
+    }
+    __syncthreads();
+    sel_cluster_sync();                           // every CTA's histogram of this pass is complete
+    if (tid < 256) {
+      uint32_t sum = 0;
+#pragma unroll
+      for (int r = 0; r < CL; ++r) sum += sel_peer_load(&hist[tid], r);
+      tot[tid] = sum;
+    }
+    if (pass == 0 && tid == 256) {
+      uint32_t sum = 0;
+      for (int r = 0; r < CL; ++r) sum += sel_peer_load(&s_ncand_local, r);
+      s_ncand = sum;
+    }
+    __syncthreads();
+    if (pass == 0) n_keep = min((uint32_t)C, s_ncand);
+    if (n_keep > 0 && warp == 0) {
+      uint32_t b, rem;
+      pick_bin(tot, pass == 0 ? n_keep : s_remaining, lane, b, rem);
+      if (lane == 0) {
+        s_prefix = prefix | (b << shift);
+        s_remaining = rem;
+      }
+    }
+    __syncthreads();
+    sel_cluster_sync();                           // peers have read this CTA's histogram
+    if (n_keep == 0) break;                       // same decision in every CTA of the cluster
+  }
+  __syncthreads();
+  if (n_keep > 0) { tau = s_prefix; quota = s_remaining; }
+
+  // kept tokens of the lower-ranked CTAs: count own keys above / equal to tau, exchange
+  {
+    uint32_t ngt = 0, neq = 0;
+    for (int t = t_beg + tid; t < t_end; t += 1024) {
+      const uint32_t kx = rowl[t];
+      ngt += (n_keep > 0 && kx != 0u && kx > tau);
+      neq += (n_keep > 0 && kx != 0u && kx == tau);
+    }
+    for (int o = 16; o > 0; o >>= 1) {
+      ngt += __shfl_xor_sync(0xffffffffu, ngt, o);
+      neq += __shfl_xor_sync(0xffffffffu, neq, o);
+    }
+    if (lane == 0) { if (ngt) atomicAdd(&s_cnt_gt, ngt); if (neq) atomicAdd(&s_cnt_eq, neq); }
+    __syncthreads();
+    sel_cluster_sync();
+    if (tid == 0) {
+      uint32_t gt_before = 0, eq_before = 0;
+      for (uint32_t r = 0; r < rank; ++r) { gt_before += sel_peer_load(&s_cnt_gt, r); eq_before += sel_peer_load(&s_cnt_eq, r); }
+      base_eq = eq_before;
+      base_sel = gt_before + min(eq_before, quota);
+    }
+    __syncthreads();
+  }
+
+  // slot assignment over this CTA's tokens, ascending token order
+  uint32_t cur[SEL_KPT], nxt[SEL_KPT];
+  load_keys(rowl, t_beg + tid * SEL_KPT, t_end, cur);
+  for (int c0 = t_beg; c0 < t_end; c0 += SEL_SWEEP) {
+    if (c0 + SEL_SWEEP < t_end) load_keys(rowl, c0 + SEL_SWEEP + tid * SEL_KPT, t_end, nxt);
+    const int tb = c0 + tid * SEL_KPT;
+    uint32_t ngt = 0, neq = 0;
+#pragma unroll
+    for (int u = 0; u < SEL_KPT; ++u) {
+      const bool live = n_keep > 0 && tb + u < t_end && cur[u] != 0u;
+      ngt += live && cur[u] > tau;
+      neq += live && cur[u] == tau;
+    }
+    const uint32_t mine = ngt | (neq << 16);
+    uint32_t inc = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const uint32_t y = __shfl_up_sync(0xffffffffu, inc, o);
+      if (lane >= o) inc += y;
+    }
+    if (lane == 31) warp_tot[warp] = inc;
+    __syncthreads();
+    if (warp == 0) {
+      const uint32_t wt = warp_tot[lane];
+      uint32_t winc = wt;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t y = __shfl_up_sync(0xffffffffu, winc, o);
+        if (lane >= o) winc += y;
+      }
+      warp_pre[lane] = winc - wt;
+      if (lane == 31) warp_tot[0] = winc;
+    }
+    __syncthreads();
+    const uint32_t excl = warp_pre[warp] + inc - mine;
+    const uint32_t totals = warp_tot[0];
+    uint32_t gt_before = excl & 0xffffu, eq_rank = base_eq + (excl >> 16);
+    const uint32_t eq_before_sweep = min(base_eq, quota);
+    const uint32_t bs = base_sel;
+#pragma unroll
+    for (int u = 0; u < SEL_KPT; ++u) {
+      const int t = tb + u;
+      const uint32_t kx = cur[u];
+      const bool live = n_keep > 0 && t < t_end && kx != 0u;
+      const bool gt = live && kx > tau, eq = live && kx == tau;
+      int pos = -1;
+      if (gt || (eq && eq_rank < quota)) {
+        pos = (int)(bs + gt_before + (min(eq_rank, quota) - eq_before_sweep));
+        my_slot[pos] = t;
+        my_gate[pos] = key_to_float(kx);
+      }
+      if (t < t_end) row[t] = (uint32_t)pos;
+      gt_before += gt;
+      eq_rank += eq;
+    }
+    __syncthreads();
+    if (tid == 0) {
+      const uint32_t tot_gt = totals & 0xffffu, tot_eq = totals >> 16;
+      const uint32_t eq_after = min(base_eq + tot_eq, quota);
+      base_sel += tot_gt + (eq_after - eq_before_sweep);
+      base_eq += tot_eq;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int u = 0; u < SEL_KPT; ++u) cur[u] = nxt[u];
+  }
+  for (int p = (int)n_keep + (int)rank * 1024 + tid; p < C_stride; p += CL * 1024) { my_slot[p] = -1; my_gate[p] = 0.f; }
+  if (tid == 0 && rank == 0) counts[i] = (int)n_keep;
+  sel_cluster_sync();                             // no CTA leaves while a peer may still read its counters
 }
 
 // Token-major CSR in three small kernels without a long serial scan:
@@ -361,8 +590,35 @@ etr_status select_forward(const etr_config* c, const float* delta, etr_stats* st
   select_token_side_kernel<<<ceil_div(c->T, SEL_TB), 256, 0, st>>>(delta, rt->topk_idx, keyT, stats, p);
   ETR_LAUNCH_CHECK();
   ETR_TIME_BEGIN("select_expert_side_kernel");
-  select_expert_side_kernel<<<c->E, 1024, 0, st>>>(keyT, stats, rt->counts, rt->slot_token, rt->gate,
-                                                   c->T, p.C_stride);
+  if (c->T >= 8192 && c->T <= 4 * 49152) {     // split each expert's row over a cluster of 4 CTAs
+    constexpr int CL = 4;
+    const size_t key_bytes = (size_t)((ceil_div(c->T, CL) + SEL_KPT - 1) / SEL_KPT * SEL_KPT) * sizeof(uint32_t);
+    static bool attr_set = false;
+    if (!attr_set) {
+      if (cudaFuncSetAttribute(select_expert_side_cluster_kernel<CL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               196608) != cudaSuccess)
+        return ETR_ERR_CUDA;
+      attr_set = true;
+    }
+    cudaLaunchConfig_t lc = {};
+    lc.gridDim = dim3(c->E * CL);
+    lc.blockDim = dim3(1024);
+    lc.dynamicSmemBytes = key_bytes;
+    lc.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = CL; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    lc.attrs = attr;
+    lc.numAttrs = 1;
+    if (cudaLaunchKernelEx(&lc, select_expert_side_cluster_kernel<CL>, keyT, (const etr_stats*)stats,
+                           rt->counts, rt->slot_token, rt->gate, c->T, p.C_stride) != cudaSuccess) {
+      timing_end(st);
+      return ETR_ERR_CUDA;
+    }
+  } else {
+    select_expert_side_kernel<<<c->E, 1024, 0, st>>>(keyT, stats, rt->counts, rt->slot_token, rt->gate,
+                                                     c->T, p.C_stride);
+  }
   ETR_LAUNCH_CHECK();
   ETR_TIME_BEGIN("csr_count_kernel");
   int32_t* block_total = reinterpret_cast<int32_t*>(reinterpret_cast<char*>(ws) + select_keys_bytes(c));
