@@ -304,7 +304,7 @@ __device__ __forceinline__ uint32_t sel_peer_load(const uint32_t* local, uint32_
 }
 
 template <int CL>
-__global__ void __launch_bounds__(1024)
+__global__ void __launch_bounds__(1024, 2)
 select_expert_side_cluster_kernel(uint32_t* __restrict__ keyT, const etr_stats* __restrict__ stats,
                                   int32_t* __restrict__ counts, int32_t* __restrict__ slot_token,
                                   float* __restrict__ gate, int T, int C_stride) {
