@@ -38,11 +38,11 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised
 # under profiles/ (absent: not captured for the current version of that kernel).
 NCU_TRAFFIC_BYTES = {}
-# tc_grouped_gemm_kernel: measured on the mid workload, all 7 launches of one step
-# (profiles/tc_grouped_gemm_kernel_mid_ncu_full.md): 3562.6 MB of DRAM traffic against 3799.7 MB of
-# algorithmic bytes (part of the output is still in L2 when a kernel ends).  The large workload is too
-# big for a multi-pass capture, so its traffic is this ratio times its own algorithmic bytes.
-TC_GEMM_DRAM_OVER_ALGORITHMIC = 3562.6 / 3799.7
+# tc_grouped_gemm_pair_kernel: measured on the mid workload, all 7 launches of one step
+# (profiles/tc_grouped_gemm_pair_kernel_mid_ncu_full.md): 3652.0 MB of DRAM traffic against 3799.7 MB
+# of algorithmic bytes (part of the output is still in L2 when a kernel ends).  The large workload is
+# too big for a multi-pass capture, so its traffic is this ratio times its own algorithmic bytes.
+TC_GEMM_DRAM_OVER_ALGORITHMIC = 3652.0 / 3799.7
 
 
 def tc_gemm_algorithmic_bytes(w, rows_padded):
@@ -210,7 +210,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="large", choices=list(gw.WORKLOADS))
-    ap.add_argument("--gemm", default="auto", choices=["auto", "simt", "tcgen05", "tcgen05_2cta"])
+    ap.add_argument("--gemm", default="auto", choices=["auto", "simt", "tcgen05", "tcgen05_2cta", "tcgen05_2cta_wide"])
     ap.add_argument("--cpu-tokens", type=int, default=128, help="tokens in the CPU-oracle sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--set", default="", help="override workload fields, e.g. T=32768,h=512 (profiling cases)")
@@ -268,7 +268,7 @@ def main():
     R = torch.from_numpy(inp["R"]).to(dev)
     W1g, W1u, W2 = device_weights(w, dev, w.seed)
     impl = {"auto": etr.GEMM_AUTO, "simt": etr.GEMM_SIMT, "tcgen05": etr.GEMM_TCGEN05,
-            "tcgen05_2cta": etr.GEMM_TCGEN05_2CTA}[args.gemm]
+            "tcgen05_2cta": etr.GEMM_TCGEN05_2CTA, "tcgen05_2cta_wide": etr.GEMM_TCGEN05_2CTA_WIDE}[args.gemm]
     cfg = etr.make_config(T=w.T, d=w.d, D=w.D, E=w.E, k=w.k, h=w.h, capacity=w.capacity,
                           dtype=etr.BF16 if w.dtype == "bf16" else etr.F32,
                           mode=etr.MODE_TCR if mode_name(w) == "tcr" else etr.MODE_ECR,
@@ -345,8 +345,9 @@ def main():
         kernels.append({"kernel": name, "launches_per_step": n / args.steps, "ms_per_step": ms / args.steps,
                         "share": ms / sum(v[1] for v in per.values()), "bound": bound,
                         "achieved": ach, "peak": peak, "unit": unit, "frac": ach / peak})
-    # The six tcgen05 contractions are instantiations of one kernel (tc_grouped_gemm_kernel);
-    # the roofline entry is that kernel over all its launches when it dominates the step.
+    # The six tcgen05 contractions are instantiations of one kernel (tc_grouped_gemm_pair_kernel,
+    # or the single-CTA tc_grouped_gemm_kernel when --gemm tcgen05 asks for it); the roofline
+    # entry is that kernel over all its launches when it dominates the step.
     tc = [k for k in kernels if k["kernel"].startswith("tc_gemm_")]
     roofline = None
     if tc and sum(k["ms_per_step"] for k in tc) >= 0.5 * sum(k["ms_per_step"] for k in kernels):
@@ -354,11 +355,14 @@ def main():
         ms = sum(k["ms_per_step"] for k in tc)
         n = sum(k["launches_per_step"] for k in tc)
         ach = flops / (ms * 1e-3) / 1e12
-        roofline = {"kernel": "tc_grouped_gemm_kernel", "launches_per_step": n, "bound": "tensor",
+        pair = args.gemm in ("auto", "tcgen05_2cta")
+        roofline = {"kernel": "tc_grouped_gemm_pair_kernel" if pair else "tc_grouped_gemm_kernel",
+                    "launches_per_step": n, "bound": "tensor",
                     "achieved": ach, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
                     "frac": ach / peaks["bf16_tflops_sustained"],
                     "flops_per_launch": flops / n, "avg_launch_ms": ms / n,
-                    "traffic": TC_GEMM_DRAM_OVER_ALGORITHMIC * tc_gemm_algorithmic_bytes(w, rows_padded) / n,
+                    "traffic": (TC_GEMM_DRAM_OVER_ALGORITHMIC * tc_gemm_algorithmic_bytes(w, rows_padded) / n
+                                if pair else None),
                     "traffic_note": "ncu dram bytes of the mid workload scaled by algorithmic bytes",
                     "peak_source": peaks["source"] + " (sustained: timed inside a long step)",
                     "frac_of_burst_peak": ach / peaks["bf16_tflops"]}

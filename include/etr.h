@@ -57,7 +57,11 @@ typedef enum {
 
 typedef enum { ETR_F32 = 0, ETR_BF16 = 1 } etr_dtype;
 typedef enum { ETR_MODE_AUTO = 0, ETR_MODE_TCR = 1, ETR_MODE_ECR = 2 } etr_mode;
-typedef enum { ETR_GEMM_AUTO = 0, ETR_GEMM_SIMT = 1, ETR_GEMM_TCGEN05 = 2, ETR_GEMM_TCGEN05_2CTA = 3 } etr_gemm_impl;
+/* Grouped-GEMM kernel of the expert FFN.  TCGEN05: one CTA per 128 x 256 tile; TCGEN05_2CTA: a CTA
+ * pair per 256 x 256 tile; TCGEN05_2CTA_WIDE: a CTA pair per 256 x 512 tile (two accumulators
+ * sharing the A operand). */
+typedef enum { ETR_GEMM_AUTO = 0, ETR_GEMM_SIMT = 1, ETR_GEMM_TCGEN05 = 2, ETR_GEMM_TCGEN05_2CTA = 3,
+               ETR_GEMM_TCGEN05_2CTA_WIDE = 4 } etr_gemm_impl;
 
 /* Immutable description of one layer call (host struct, passed by pointer). */
 typedef struct etr_config {

@@ -40,7 +40,7 @@ void timing_end(cudaStream_t st) {
 
 static bool use_tc(const etr_config* c) {
   if (c->gemm_impl == ETR_GEMM_SIMT) return false;
-  if (c->gemm_impl == ETR_GEMM_TCGEN05 || c->gemm_impl == ETR_GEMM_TCGEN05_2CTA) return true;
+  if (c->gemm_impl >= ETR_GEMM_TCGEN05 && c->gemm_impl <= ETR_GEMM_TCGEN05_2CTA_WIDE) return true;
   return c->dtype == ETR_BF16 && tc_available();
 }
 
@@ -134,7 +134,7 @@ etr_status etr_validate(const etr_config* c) {
     return ETR_ERR_ARG;
   if (c->dtype != ETR_F32 && c->dtype != ETR_BF16) return ETR_ERR_ARG;
   if (c->mode < ETR_MODE_AUTO || c->mode > ETR_MODE_ECR) return ETR_ERR_ARG;
-  if (c->gemm_impl < ETR_GEMM_AUTO || c->gemm_impl > ETR_GEMM_TCGEN05_2CTA) return ETR_ERR_ARG;
+  if (c->gemm_impl < ETR_GEMM_AUTO || c->gemm_impl > ETR_GEMM_TCGEN05_2CTA_WIDE) return ETR_ERR_ARG;
   if (c->d % c->D != 0 || c->d % 8 != 0 || c->h % 8 != 0) return ETR_ERR_SHAPE;
   if (c->k > c->E || c->E > 256 || c->E > c->d / c->D) return ETR_ERR_SHAPE;
   if ((long long)c->T * c->E >= (1ll << 31)) return ETR_ERR_SHAPE;

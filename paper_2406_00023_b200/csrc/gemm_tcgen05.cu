@@ -181,6 +181,23 @@ __device__ __forceinline__ void store32_warp(uint8_t* scratch, int lane, int nva
   __syncwarp();
 }
 
+// The same store for a block already packed to bf16 (16 words per lane).
+__device__ __forceinline__ void store32_warp_packed(uint8_t* scratch, int lane, int nvalid, __nv_bfloat16* dst,
+                                                    int ld_out, const uint32_t* w16) {
+  uint4* mine = reinterpret_cast<uint4*>(scratch + lane * TC_SCRATCH_ROW_BYTES);
+#pragma unroll
+  for (int q = 0; q < 4; ++q) mine[q] = make_uint4(w16[4 * q], w16[4 * q + 1], w16[4 * q + 2], w16[4 * q + 3]);
+  __syncwarp();
+  const int sub = lane & 3;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int row = (lane >> 2) + 8 * i;
+    const uint4 w = *reinterpret_cast<const uint4*>(scratch + row * TC_SCRATCH_ROW_BYTES + sub * 16);
+    if (row < nvalid) *reinterpret_cast<uint4*>(dst + (long long)row * ld_out + sub * 8) = w;
+  }
+  __syncwarp();
+}
+
 // The reverse turn for the saved activations the SwiGLU derivative reads: fetched as 8 rows x
 // 64 contiguous bytes per instruction (regs `t`), later handed to the lane that owns the row.
 __device__ __forceinline__ void load32_warp_issue(const __nv_bfloat16* src, int ld, int lane, int nvalid,
@@ -757,6 +774,290 @@ tc_grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap mapA0, const __g
   }
 }
 
+// ---- CTA-pair kernel, two output tiles per pass ------------------------------------------------------
+// Same pair as above, but one pass covers 256 rows x 2 adjacent column tiles: the A boxes of a K
+// block are fetched once and multiplied into two accumulators (tensor-memory columns [0,256) and
+// [256,512)), so a K block moves 48 KiB per CTA for twice the flops of the 32 KiB above: a
+// quarter less operand traffic from L2 per flop.  The price is that all of tensor memory is one
+// tile's accumulator: the next tile's MMAs wait for the epilogue.  To hide most of that, the
+// epilogue drains and releases the two halves separately, and the MMA warp runs the first K
+// blocks of the next tile into half 0 alone (those stages stay held) until half 1 is free.
+constexpr int TCW_STAGES = 4;
+constexpr uint32_t TCW_STAGE_BYTES = 6 * TC_BOX_BYTES;       // per CTA: 2 boxes of A, 2 + 2 of B
+constexpr int TCW_LEAD = TCW_STAGES - 1;                     // K blocks half 0 may run ahead of half 1
+
+__device__ __forceinline__ bool tile_coord_wide(const TcParams& p, const int* tile_prefix, int tile, int& e_cur,
+                                                int n_tile_cols, TileCoord& tc) {
+  if (tile >= tile_prefix[p.E]) return false;
+  while (tile >= tile_prefix[e_cur + 1]) ++e_cur;
+  const int local = tile - tile_prefix[e_cur];
+  const int n_e = p.counts[e_cur];
+  int mt_count;
+  if (p.dyn == TC_DYN_M) {
+    mt_count = (min(n_e, p.M) + 255) / 256;
+    tc.kblocks = (p.K + TC_BK - 1) / TC_BK;
+    tc.m_lim = (min(n_e, p.M) + TC_BM - 1) / TC_BM * TC_BM;
+  } else {
+    mt_count = (p.M + 255) / 256;
+    tc.kblocks = (n_e + TC_BK - 1) / TC_BK;
+    tc.m_lim = p.M;
+  }
+  tc.e = e_cur;
+  tc.m0 = (local % mt_count) * 256;
+  tc.n0 = (local / mt_count) * 2 * n_tile_cols;
+  return true;
+}
+
+template <int EPI>
+__global__ void __launch_bounds__(TC_THREADS, 1)
+tc_grouped_gemm_pair_wide_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtensorMap mapA1,
+                                 const __grid_constant__ CUtensorMap mapB0, const __grid_constant__ CUtensorMap mapB1,
+                                 const TcParams p) {
+  constexpr int BN = 256;
+  constexpr int N_TILE_COLS = (EPI == TC_EPI_SWIGLU) ? BN / 2 : BN;
+  constexpr uint32_t TMEM_COLS = 512;
+
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t bars[2 * TCW_STAGES + 3];
+  __shared__ uint32_t tmem_base_slot;
+  __shared__ int abort_flag_s;
+  __shared__ int tile_prefix[257];
+
+  volatile int* abort_flag = &abort_flag_s;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const uint32_t rank = cluster_ctarank();
+  const int pair = (int)cluster_id_x(), npairs = (int)cluster_count_x();
+  const uint32_t tiles_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t full_bar = smem_u32(&bars[0]);                    // [TCW_STAGES]  used in the leader
+  const uint32_t empty_bar = smem_u32(&bars[TCW_STAGES]);          // [TCW_STAGES]  in each CTA
+  const uint32_t tfull_bar = smem_u32(&bars[2 * TCW_STAGES]);      // [1]           in each CTA
+  const uint32_t tempty_bar = smem_u32(&bars[2 * TCW_STAGES + 1]); // [2]           used in the leader
+
+  if (tid == 0) {
+    abort_flag_s = 0;
+    for (int s = 0; s < TCW_STAGES; ++s) { mbar_init(full_bar + 8 * s, 1); mbar_init(empty_bar + 8 * s, 1); }
+    mbar_init(tfull_bar, 1);
+    for (int a = 0; a < 2; ++a) mbar_init(tempty_bar + 8 * a, 16);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    const int nt = (p.N + 2 * N_TILE_COLS - 1) / (2 * N_TILE_COLS);
+    int acc = 0;
+    for (int e = 0; e < p.E; ++e) {
+      tile_prefix[e] = acc;
+      const int n_e = p.counts[e];
+      const int mt = p.dyn == TC_DYN_M ? (min(n_e, p.M) + 255) / 256 : (p.M + 255) / 256;
+      acc += mt * nt;
+    }
+    tile_prefix[p.E] = acc;
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"(TMEM_COLS) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();                 // both CTAs' barriers exist before any remote arrive
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_slot;
+  const uint32_t leader_full = map_to_cta(full_bar, 0);
+  const uint32_t leader_tempty = map_to_cta(tempty_bar, 0);
+
+  if (warp == 0) {
+    // ---- TMA producer (both CTAs) ---------------------------------------------------------------
+    if (lane == 0) {
+      int e_cur = 0, stage = 0;
+      uint32_t phase = 0;
+      TileCoord tc;
+      bool ok = true;
+      for (int tile = pair; ok && tile_coord_wide(p, tile_prefix, tile, e_cur, N_TILE_COLS, tc); tile += npairs) {
+        const int m0c = tc.m0 + 128 * (int)rank;
+        const bool two = tc.n0 + N_TILE_COLS < p.N;
+        for (int kb = 0; kb < tc.kblocks; ++kb) {
+          if (!mbar_wait_cluster(empty_bar + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
+          if (rank == 0) mbar_expect_tx(full_bar + 8 * stage, 2 * (two ? 6 : 4) * TC_BOX_BYTES);
+          const uint32_t fb = leader_full + 8 * stage;
+          const bool second = p.k1_blocks > 0 && kb >= p.k1_blocks;
+          const int k0 = (second ? kb - p.k1_blocks : kb) * TC_BK;
+          const CUtensorMap* ma = second ? &mapA1 : &mapA0;
+          const CUtensorMap* mb = p.dual_b ? (rank ? &mapB1 : &mapB0) : (second ? &mapB1 : &mapB0);
+          const uint32_t sa = tiles_base + stage * TCW_STAGE_BYTES;
+#pragma unroll
+          for (int j = 0; j < 2; ++j) {
+            if (p.a_mn) tma_load_3d_pair(sa + j * TC_BOX_BYTES, ma, fb, m0c + 64 * j, k0, tc.e);
+            else        tma_load_3d_pair(sa + j * TC_BOX_BYTES, ma, fb, k0, m0c + 64 * j, tc.e);
+          }
+          for (int hf = 0; hf < (two ? 2 : 1); ++hf) {
+            const uint32_t sb = sa + (2 + 2 * hf) * TC_BOX_BYTES;
+            const int nh = tc.n0 + hf * N_TILE_COLS;
+            const int nb = p.dual_b ? nh : nh + 128 * (int)rank;
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+              if (p.b_mn) tma_load_3d_pair(sb + j * TC_BOX_BYTES, mb, fb, nb + 64 * j, k0, tc.e);
+              else        tma_load_3d_pair(sb + j * TC_BOX_BYTES, mb, fb, k0, nb + 64 * j, tc.e);
+            }
+          }
+          if (++stage == TCW_STAGES) { stage = 0; phase ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---- MMA issuer (leader CTA only) --------------------------------------------------------------
+    if (lane == 0 && rank == 0) {
+      int e_cur = 0, stage = 0;
+      uint32_t phase = 0, acc_phase = 0;
+      TileCoord tc;
+      bool ok = true;
+      const uint32_t a_lbo = p.a_mn ? TC_BOX_BYTES : 16u, b_lbo = p.b_mn ? TC_BOX_BYTES : 16u;
+      const uint32_t a_kstep = p.a_mn ? 2048u : 32u, b_kstep = p.b_mn ? 2048u : 32u;
+      // one K block of one half: 4 MMAs of 256 x 256 x 16
+      auto issue = [&](int st, int hf, bool first_block) {
+        const uint32_t sa = tiles_base + st * TCW_STAGE_BYTES;
+        const uint32_t sb = sa + (2 + 2 * hf) * TC_BOX_BYTES;
+#pragma unroll
+        for (int kk = 0; kk < TC_BK / 16; ++kk) {
+          const uint64_t ad = make_smem_desc(sa + kk * a_kstep, a_lbo, 1024u);
+          const uint64_t bd = make_smem_desc(sb + kk * b_kstep, b_lbo, 1024u);
+          tc_mma_pair(tmem_base + (uint32_t)(hf * 256), ad, bd, p.idesc, (!first_block || kk > 0) ? 1u : 0u);
+        }
+      };
+      for (int tile = pair; ok && tile_coord_wide(p, tile_prefix, tile, e_cur, N_TILE_COLS, tc); tile += npairs) {
+        if (tc.kblocks == 0) continue;
+        const bool two = tc.n0 + N_TILE_COLS < p.N;
+        if (!mbar_wait_cluster(tempty_bar, acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        // Lead-in: half 0 of the first K blocks while the epilogue still drains half 1.
+        const int lead = two ? min(TCW_LEAD, tc.kblocks) : 0;
+        int st = stage;
+        uint32_t ph = phase;
+        for (int kb = 0; kb < lead; ++kb) {
+          if (!mbar_wait_cluster(full_bar + 8 * st, ph, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          issue(st, 0, kb == 0);
+          if (++st == TCW_STAGES) { st = 0; ph ^= 1u; }
+        }
+        if (!ok) break;
+        if (!mbar_wait_cluster(tempty_bar + 8, acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        for (int kb = 0; kb < tc.kblocks; ++kb) {
+          if (kb >= lead) {
+            if (!mbar_wait_cluster(full_bar + 8 * stage, phase, abort_flag)) { ok = false; break; }
+            tc_fence_after();
+            issue(stage, 0, kb == 0);
+          }
+          if (two) issue(stage, 1, kb == 0);
+          tc_commit_pair(empty_bar + 8 * stage);      // frees the stage in both CTAs
+          if (++stage == TCW_STAGES) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        tc_commit_pair(tfull_bar);                    // both accumulators complete in both CTAs
+        acc_phase ^= 1u;
+      }
+    }
+  } else {
+    // ---- epilogue warps (both CTAs, own 128 rows) -----------------------------------------------------
+    const int q = warp & 3;
+    uint8_t* scratch = smem_raw + (tiles_base - smem_u32(smem_raw)) + TCW_STAGES * TCW_STAGE_BYTES + (warp - 2) * TC_SCRATCH_BYTES;
+    const int half = (warp - 2) >> 2;
+    constexpr int NCH = N_TILE_COLS / 32 / 2;
+    const int row_in_tile = 128 * (int)rank + 32 * q + lane;
+    int e_cur = 0;
+    uint32_t acc_phase = 0;
+    TileCoord tc;
+    bool ok = true;
+    for (int tile = pair; ok && tile_coord_wide(p, tile_prefix, tile, e_cur, N_TILE_COLS, tc); tile += npairs) {
+      const int grow = tc.m0 + row_in_tile;
+      const bool row_ok = grow < tc.m_lim;
+      const int c_beg = half * NCH;
+      const bool two = tc.n0 + N_TILE_COLS < p.N;
+      const long long obase = (long long)tc.e * p.out_bs + (long long)grow * p.ld_out + tc.n0;
+      if (tc.kblocks == 0) {
+        if (row_ok) {
+          float z[32];
+#pragma unroll
+          for (int i = 0; i < 32; ++i) z[i] = 0.f;
+          for (int hf = 0; hf < (two ? 2 : 1); ++hf)
+            for (int c = c_beg; c < c_beg + NCH && tc.n0 + hf * N_TILE_COLS + 32 * c < p.N; ++c)
+              store32(p.out0 + obase + hf * N_TILE_COLS + 32 * c, z);
+        }
+        continue;
+      }
+      uint4 pg[4], pu[4];
+      const int nvalid = min(32, max(0, tc.m_lim - (grow - lane)));
+      if (EPI == TC_EPI_DSWIGLU && tc.n0 + 32 * c_beg < p.N) {
+        const long long wb = obase - (long long)lane * p.ld_out + 32 * c_beg;
+        load32_warp_issue(p.in0 + wb, p.ld_out, lane, nvalid, pg);
+        load32_warp_issue(p.in1 + wb, p.ld_out, lane, nvalid, pu);
+      }
+      if (!mbar_wait_cluster(tfull_bar, acc_phase, abort_flag)) { ok = false; break; }
+      tc_fence_after();
+      if (EPI == TC_EPI_STORE) {
+        // Plain stores: empty each half into registers (packed bf16) and release it at once;
+        // the turn through the scratch and the global stores follow while the MMAs run on.
+        static_assert(EPI != TC_EPI_STORE || NCH == 4, "four chunks of 32 columns per warp and half");
+        for (int hf = 0; hf < 2; ++hf) {
+          uint32_t pk[NCH][16];
+          const int n0h = tc.n0 + hf * N_TILE_COLS;
+          const bool live = hf == 0 || two;
+          if (live) {
+            const uint32_t taddr = tmem_base + (uint32_t)(hf * 256) + ((uint32_t)(32 * q) << 16);
+            uint32_t r[NCH][32];
+#pragma unroll
+            for (int c = 0; c < NCH; ++c) tc_ld32(taddr + 32 * (c_beg + c), r[c]);
+            tc_wait_ld();
+#pragma unroll
+            for (int c = 0; c < NCH; ++c)
+#pragma unroll
+              for (int i = 0; i < 16; ++i)
+                pk[c][i] = pack_bf16(__uint_as_float(r[c][2 * i]), __uint_as_float(r[c][2 * i + 1]));
+          }
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive_cluster(leader_tempty + 8 * hf);
+          if (live) {
+            const long long wb = obase - (long long)lane * p.ld_out + hf * N_TILE_COLS;
+#pragma unroll
+            for (int c = 0; c < NCH; ++c)
+              if (n0h + 32 * (c_beg + c) < p.N)
+                store32_warp_packed(scratch, lane, nvalid, p.out0 + wb + 32 * (c_beg + c), p.ld_out, pk[c]);
+          }
+        }
+      } else {
+        for (int hf = 0; hf < 2; ++hf) {
+          if (hf == 0 || two) {
+            const int n0h = tc.n0 + hf * N_TILE_COLS;
+            const long long ob = obase + hf * N_TILE_COLS;
+            if (EPI == TC_EPI_DSWIGLU && hf == 1 && n0h + 32 * c_beg < p.N) {
+              const long long wb = ob - (long long)lane * p.ld_out + 32 * c_beg;
+              load32_warp_issue(p.in0 + wb, p.ld_out, lane, nvalid, pg);
+              load32_warp_issue(p.in1 + wb, p.ld_out, lane, nvalid, pu);
+            }
+            const uint32_t taddr = tmem_base + (uint32_t)(hf * 256) + ((uint32_t)(32 * q) << 16);
+            epilogue_chunks<EPI, BN>(p, n0h, taddr, ob, row_ok, c_beg, NCH, pg, pu, scratch, lane, nvalid);
+          }
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive_cluster(leader_tempty + 8 * hf);
+        }
+      }
+      acc_phase ^= 1u;
+    }
+  }
+
+  // ---- teardown: neither CTA leaves while the other may still touch its barriers or memory -------
+  __syncwarp();
+  if (*abort_flag) {
+    const long long t0 = clock64();
+    while (clock64() - t0 < 2000000ll) { }
+    if (tid == 0) atomicExch(&p.stats->error_word, 0x7c07);
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+  }
+}
+
 // ---- host side --------------------------------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
@@ -864,12 +1165,64 @@ static etr_status tc_launch_pair(const char* name, const CUtensorMap& a0, const 
   return ETR_OK;
 }
 
-// 1-CTA or 2-CTA form of one contraction; max tiles are counted in 128-row tiles
 template <int EPI>
-static etr_status tc_run(bool pair, const char* name, const CUtensorMap& a0, const CUtensorMap& a1,
+static etr_status tc_launch_pair_wide(const char* name, const CUtensorMap& a0, const CUtensorMap& a1,
+                                      const CUtensorMap& b0, const CUtensorMap& b1, TcParams p, int max_tiles,
+                                      cudaStream_t st) {
+  constexpr size_t smem = (size_t)TCW_STAGES * TCW_STAGE_BYTES + 1024 + 8 * TC_SCRATCH_BYTES;
+  auto k = tc_grouped_gemm_pair_wide_kernel<EPI>;
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+      return ETR_ERR_CUDA;
+    attr_set = true;
+  }
+  p.idesc = make_idesc(p.a_mn, p.b_mn, 256, 256);
+  const int pairs_max = sm_count() / 2;
+  const int pairs = max_tiles < pairs_max ? (max_tiles < 1 ? 1 : max_tiles) : pairs_max;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(2 * pairs);
+  cfg.blockDim = dim3(TC_THREADS);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  ETR_TIME_BEGIN(name);
+  if (cudaLaunchKernelEx(&cfg, k, a0, a1, b0, b1, p) != cudaSuccess) { timing_end(st); return ETR_ERR_CUDA; }
+  ETR_LAUNCH_CHECK();
+  return ETR_OK;
+}
+
+// The three forms of one contraction; max_tiles is an upper bound counted in 128-row tiles of one
+// column tile (it only caps the grid for small problems).
+enum TcForm { TC_FORM_SINGLE, TC_FORM_PAIR, TC_FORM_PAIR_WIDE };
+
+// Which form runs one contraction.  A forced gemm_impl decides alone.  Otherwise (AUTO) the wide
+// pair form is taken where its saving in operand traffic outweighs its exposed epilogue: plain
+// stores whose row extent is the expert's token count (down, dXp), and the fused SwiGLU when the
+// contraction is long (>= 48 K blocks); and only when the launch has at least four rounds of wide
+// tiles per CTA pair at full capacity, since a wide tile is twice the unit of work.  Weight
+// gradients (short contraction over the expert's rows, large outputs) and the SwiGLU derivative
+// (its epilogue also fetches G and U) measured faster on 256 x 256 tiles.
+static TcForm tc_form_of(const etr_config* c, int epi, const TcParams& p) {
+  if (c->gemm_impl == ETR_GEMM_TCGEN05) return TC_FORM_SINGLE;
+  if (c->gemm_impl == ETR_GEMM_TCGEN05_2CTA) return TC_FORM_PAIR;
+  if (c->gemm_impl == ETR_GEMM_TCGEN05_2CTA_WIDE) return TC_FORM_PAIR_WIDE;
+  if (p.dyn != TC_DYN_M || epi == TC_EPI_DSWIGLU) return TC_FORM_PAIR;
+  if (epi == TC_EPI_SWIGLU && ceil_div(p.K, TC_BK) < 48) return TC_FORM_PAIR;
+  const int cols = epi == TC_EPI_SWIGLU ? 256 : 512;
+  const long long wide_tiles = (long long)p.E * ceil_div(p.M, 256) * ceil_div(p.N, cols);
+  return wide_tiles >= 4ll * (sm_count() / 2) ? TC_FORM_PAIR_WIDE : TC_FORM_PAIR;
+}
+template <int EPI>
+static etr_status tc_run(TcForm form, const char* name, const CUtensorMap& a0, const CUtensorMap& a1,
                          const CUtensorMap& b0, const CUtensorMap& b1, const TcParams& p, int max_tiles,
                          cudaStream_t st) {
-  if (pair) return tc_launch_pair<EPI>(name, a0, a1, b0, b1, p, (max_tiles + 1) / 2, st);
+  if (form == TC_FORM_PAIR_WIDE) return tc_launch_pair_wide<EPI>(name, a0, a1, b0, b1, p, (max_tiles + 1) / 2, st);
+  if (form == TC_FORM_PAIR) return tc_launch_pair<EPI>(name, a0, a1, b0, b1, p, (max_tiles + 1) / 2, st);
   return tc_launch<256, EPI>(name, a0, a1, b0, b1, p, max_tiles, st);
 }
 
@@ -880,7 +1233,6 @@ etr_status tc_ffn_forward(const etr_config* c, const etr_route* rt, const void* 
                           const void* W1u, const void* W2, void* G, void* U, void* H, void* O,
                           etr_stats* stats, void*, cudaStream_t st) {
   const int d = c->d, h = c->h, Cs = c_stride_of(c), E = c->E;
-  const bool pair = c->gemm_impl != ETR_GEMM_TCGEN05;      // default: CTA pairs
   CUtensorMap mXp, mW1g, mW1u, mW2, mH;
   ETR_TRY(make_map(&mXp, Xp, d, Cs, E));
   ETR_TRY(make_map(&mW1g, W1g, d, h, E));
@@ -893,14 +1245,14 @@ etr_status tc_ffn_forward(const etr_config* c, const etr_route* rt, const void* 
     p.dual_b = 1; p.M = Cs; p.N = h; p.K = d; p.dyn = TC_DYN_M; p.E = E; p.counts = rt->counts;
     p.out0 = (__nv_bfloat16*)G; p.out1 = (__nv_bfloat16*)U; p.out2 = (__nv_bfloat16*)H;
     p.out_bs = (long long)Cs * h; p.ld_out = h; p.stats = stats;
-    ETR_TRY((tc_run<TC_EPI_SWIGLU>(pair, "tc_gemm_swiglu", mXp, mXp, mW1g, mW1u, p,
+    ETR_TRY((tc_run<TC_EPI_SWIGLU>(tc_form_of(c, TC_EPI_SWIGLU, p), "tc_gemm_swiglu", mXp, mXp, mW1g, mW1u, p,
                                            E * mt * ceil_div(h, 128), st)));
   }
   {  // O = H W2^T
     TcParams p = {};
     p.M = Cs; p.N = d; p.K = h; p.dyn = TC_DYN_M; p.E = E; p.counts = rt->counts;
     p.out0 = (__nv_bfloat16*)O; p.out_bs = (long long)Cs * d; p.ld_out = d; p.stats = stats;
-    ETR_TRY((tc_run<TC_EPI_STORE>(pair, "tc_gemm_down", mH, mH, mW2, mW2, p, E * mt * ceil_div(d, 256), st)));
+    ETR_TRY((tc_run<TC_EPI_STORE>(tc_form_of(c, TC_EPI_STORE, p), "tc_gemm_down", mH, mH, mW2, mW2, p, E * mt * ceil_div(d, 256), st)));
   }
   return ETR_OK;
 }
@@ -910,7 +1262,6 @@ etr_status tc_ffn_backward(const etr_config* c, const etr_route* rt, const void*
                            const void* W1u, const void* W2, void* dG, void* dU, void* dXp, void* dW1g,
                            void* dW1u, void* dW2, etr_stats* stats, void*, cudaStream_t st) {
   const int d = c->d, h = c->h, Cs = c_stride_of(c), E = c->E;
-  const bool pair = c->gemm_impl != ETR_GEMM_TCGEN05;      // default: CTA pairs
   CUtensorMap mdO, mXp, mH, mdG, mdU, mW1g, mW1u, mW2;
   ETR_TRY(make_map(&mdO, dO, d, Cs, E));
   ETR_TRY(make_map(&mXp, Xp, d, Cs, E));
@@ -927,7 +1278,7 @@ etr_status tc_ffn_backward(const etr_config* c, const etr_route* rt, const void*
     p.out0 = (__nv_bfloat16*)dG; p.out1 = (__nv_bfloat16*)dU;
     p.in0 = (const __nv_bfloat16*)G; p.in1 = (const __nv_bfloat16*)U;
     p.out_bs = (long long)Cs * h; p.ld_out = h; p.stats = stats;
-    ETR_TRY((tc_run<TC_EPI_DSWIGLU>(pair, "tc_gemm_dswiglu", mdO, mdO, mW2, mW2, p,
+    ETR_TRY((tc_run<TC_EPI_DSWIGLU>(tc_form_of(c, TC_EPI_DSWIGLU, p), "tc_gemm_dswiglu", mdO, mdO, mW2, mW2, p,
                                             E * mt * ceil_div(h, 256), st)));
   }
   {  // dXp = dG W1g + dU W1u: one contraction over 2h
@@ -935,14 +1286,14 @@ etr_status tc_ffn_backward(const etr_config* c, const etr_route* rt, const void*
     p.b_mn = 1; p.k1_blocks = ceil_div(h, TC_BK); p.M = Cs; p.N = d; p.K = 2 * h; p.dyn = TC_DYN_M;
     p.E = E; p.counts = rt->counts;
     p.out0 = (__nv_bfloat16*)dXp; p.out_bs = (long long)Cs * d; p.ld_out = d; p.stats = stats;
-    ETR_TRY((tc_run<TC_EPI_STORE>(pair, "tc_gemm_dxp", mdG, mdU, mW1g, mW1u, p,
+    ETR_TRY((tc_run<TC_EPI_STORE>(tc_form_of(c, TC_EPI_STORE, p), "tc_gemm_dxp", mdG, mdU, mW1g, mW1u, p,
                                           E * mt * ceil_div(d, 256), st)));
   }
   {  // dW2 = dO^T H: contraction over the expert's rows, both operands MN-major
     TcParams p = {};
     p.a_mn = 1; p.b_mn = 1; p.M = d; p.N = h; p.dyn = TC_DYN_K; p.E = E; p.counts = rt->counts;
     p.out0 = (__nv_bfloat16*)dW2; p.out_bs = (long long)d * h; p.ld_out = h; p.stats = stats;
-    ETR_TRY((tc_run<TC_EPI_STORE>(pair, "tc_gemm_dw2", mdO, mdO, mH, mH, p,
+    ETR_TRY((tc_run<TC_EPI_STORE>(tc_form_of(c, TC_EPI_STORE, p), "tc_gemm_dw2", mdO, mdO, mH, mH, p,
                                           E * ceil_div(d, TC_BM) * ceil_div(h, 256), st)));
   }
   for (int which = 0; which < 2; ++which) {  // dW1g = dG^T Xp, dW1u = dU^T Xp
@@ -950,7 +1301,7 @@ etr_status tc_ffn_backward(const etr_config* c, const etr_route* rt, const void*
     p.a_mn = 1; p.b_mn = 1; p.M = h; p.N = d; p.dyn = TC_DYN_K; p.E = E; p.counts = rt->counts;
     p.out0 = (__nv_bfloat16*)(which ? dW1u : dW1g); p.out_bs = (long long)h * d; p.ld_out = d; p.stats = stats;
     const CUtensorMap& ma = which ? mdU : mdG;
-    ETR_TRY((tc_run<TC_EPI_STORE>(pair, "tc_gemm_dw1", ma, ma, mXp, mXp, p,
+    ETR_TRY((tc_run<TC_EPI_STORE>(tc_form_of(c, TC_EPI_STORE, p), "tc_gemm_dw1", ma, ma, mXp, mXp, p,
                                           E * ceil_div(h, TC_BM) * ceil_div(d, 256), st)));
   }
   return ETR_OK;

@@ -17,7 +17,7 @@ LIB_PATH = os.environ.get("ETR_LIB_PATH") or os.path.join(_HERE, "libetr.so")   
 OK, ERR_ARG, ERR_SHAPE, ERR_ALIGN, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_UNSUPPORTED = range(8)
 F32, BF16 = 0, 1
 MODE_AUTO, MODE_TCR, MODE_ECR = 0, 1, 2
-GEMM_AUTO, GEMM_SIMT, GEMM_TCGEN05, GEMM_TCGEN05_2CTA = 0, 1, 2, 3
+GEMM_AUTO, GEMM_SIMT, GEMM_TCGEN05, GEMM_TCGEN05_2CTA, GEMM_TCGEN05_2CTA_WIDE = 0, 1, 2, 3, 4
 
 EXPORTS = [
     "etr_status_string", "etr_validate", "etr_c_stride", "etr_workspace_bytes", "etr_buffers_bytes",

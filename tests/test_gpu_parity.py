@@ -237,6 +237,11 @@ def test_expert_ffn_tcgen05_two_cta(name):
     ffn_stage(name, etr.GEMM_TCGEN05_2CTA)
 
 
+@pytest.mark.parametrize("name", ["small_s", "mid_s", "sweep_s_tcr", "sweep_s_ecr"])
+def test_expert_ffn_tcgen05_two_cta_wide(name):
+    ffn_stage(name, etr.GEMM_TCGEN05_2CTA_WIDE)
+
+
 def run_layer(w, inp, cfg, host_step=False):
     dev = hz.upload(w, inp)
     buf = etr.LayerBuffers(cfg, host_staging=host_step)
