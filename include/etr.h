@@ -260,6 +260,30 @@ etr_status etr_layer_step_host(const etr_config* cfg, const void* X_host, const 
                                const etr_buffers* buf, void* Y_host, void* dX_host,
                                float* dR, void* dW1g, void* dW1u, void* dW2, void* stream);
 
+/* Device staging of one host step in flight: four caller-owned device buffers of T*d elements of
+ * `dtype` each (16-byte aligned). */
+typedef struct etr_host_slot { void* X_dev; void* dY_dev; void* Y_dev; void* dX_dev; } etr_host_slot;
+#define ETR_HOST_SLOTS 4
+
+/* Pipelined form of etr_layer_step_host for a loop of steps: enqueues the same work and returns
+ * without waiting, so the next step's host-to-device copies run under this step's kernels and this
+ * step's device-to-host copies under the next step's.  Steps in flight at the same time use
+ * different `slot`s (index 0 .. ETR_HOST_SLOTS-1, each with its own staging); two slots already keep
+ * both copy directions busy.  The layer's internal buffers `buf` are shared: the kernels of
+ * successive steps run in call order on `stream`, only the copies overlap them.  Re-using a slot
+ * index orders the new step after the previous use of that slot on the device; the HOST buffers of
+ * a step (all four) belong to the library until etr_layer_step_host_wait(slot) has returned.
+ * dR and the weight gradients are those of the most recent step once `stream` is idle. */
+etr_status etr_layer_step_host_begin(const etr_config* cfg, const void* X_host, const void* dY_host,
+                                     const float* R, const void* W1g, const void* W1u, const void* W2,
+                                     const etr_buffers* buf, const etr_host_slot* staging, int32_t slot,
+                                     void* Y_host, void* dX_host, float* dR,
+                                     void* dW1g, void* dW1u, void* dW2, void* stream);
+
+/* Blocks the calling thread until the last step begun on `slot` has delivered Y_host and dX_host
+ * (ETR_OK at once if nothing was begun on it). */
+etr_status etr_layer_step_host_wait(int32_t slot);
+
 /* Copies the device stats to the host and synchronises the stream.  Returns
  * ETR_ERR_TIMEOUT if a kernel recorded an expired wait. */
 etr_status etr_read_stats(const etr_stats* stats_dev, etr_stats* stats_host, void* stream);

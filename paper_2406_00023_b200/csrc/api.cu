@@ -303,7 +303,12 @@ etr_status etr_layer_backward(const etr_config* c, const void* X, const float* R
 }
 
 // Side streams and events for the host-buffer step (host-side objects, created once per device).
-struct HostStepCtx { cudaStream_t up = nullptr, down = nullptr; cudaEvent_t dy_ready = nullptr, fwd_done = nullptr, y_done = nullptr, start = nullptr; };
+struct HostSlotEvents { cudaEvent_t x_ready, dy_ready, fwd_done, bwd_done, y_down, dx_down; bool used; };
+struct HostStepCtx {
+  cudaStream_t up = nullptr, down = nullptr;
+  cudaEvent_t dy_ready = nullptr, fwd_done = nullptr, y_done = nullptr, start = nullptr;
+  HostSlotEvents slot[ETR_HOST_SLOTS] = {};
+};
 static std::mutex g_ctx_mu;
 static HostStepCtx g_ctx[64];
 
@@ -320,6 +325,12 @@ static etr_status host_step_ctx(HostStepCtx** out) {
         cudaEventCreateWithFlags(&c.y_done, cudaEventDisableTiming) != cudaSuccess ||
         cudaEventCreateWithFlags(&c.start, cudaEventDisableTiming) != cudaSuccess)
       return ETR_ERR_CUDA;
+    for (auto& sl : c.slot) {
+      cudaEvent_t* ev[6] = {&sl.x_ready, &sl.dy_ready, &sl.fwd_done, &sl.bwd_done, &sl.y_down, &sl.dx_down};
+      for (cudaEvent_t* e : ev)
+        if (cudaEventCreateWithFlags(e, cudaEventDisableTiming) != cudaSuccess) return ETR_ERR_CUDA;
+      sl.used = false;
+    }
   }
   *out = &c;
   return ETR_OK;
@@ -357,6 +368,59 @@ etr_status etr_layer_step_host(const etr_config* c, const void* X_host, const vo
   ETR_CUDA(cudaMemcpyAsync(dX_host, b->dX_dev, bytes, cudaMemcpyDeviceToHost, st));
   ETR_CUDA(cudaStreamWaitEvent(st, hc->y_done, 0));
   ETR_CUDA(cudaStreamSynchronize(st));
+  return ETR_OK;
+}
+
+etr_status etr_layer_step_host_begin(const etr_config* c, const void* X_host, const void* dY_host,
+                                     const float* R, const void* W1g, const void* W1u, const void* W2,
+                                     const etr_buffers* b, const etr_host_slot* sg, int32_t slot,
+                                     void* Y_host, void* dX_host, float* dR, void* dW1g, void* dW1u,
+                                     void* dW2, void* stream) {
+  if (b == nullptr || sg == nullptr || X_host == nullptr || dY_host == nullptr || Y_host == nullptr ||
+      dX_host == nullptr || slot < 0 || slot >= ETR_HOST_SLOTS)
+    return ETR_ERR_ARG;
+  ETR_TRY(etr_validate(c));
+  ETR_TRY(check_ptrs({sg->X_dev, sg->dY_dev, sg->Y_dev, sg->dX_dev}));
+  cudaStream_t st = (cudaStream_t)stream;
+  HostStepCtx* hc = nullptr;
+  ETR_TRY(host_step_ctx(&hc));
+  HostSlotEvents& ev = hc->slot[slot];
+  const size_t bytes = (size_t)c->T * c->d * elem_bytes(c->dtype);
+  // Upload stream: both inputs, X first.  The staging was last read by the backward pass of the
+  // previous step on this slot (a wait on an event never recorded is a no-op).
+  ETR_CUDA(cudaStreamWaitEvent(hc->up, ev.bwd_done, 0));
+  ETR_CUDA(cudaMemcpyAsync(sg->X_dev, X_host, bytes, cudaMemcpyHostToDevice, hc->up));
+  ETR_CUDA(cudaEventRecord(ev.x_ready, hc->up));
+  ETR_CUDA(cudaMemcpyAsync(sg->dY_dev, dY_host, bytes, cudaMemcpyHostToDevice, hc->up));
+  ETR_CUDA(cudaEventRecord(ev.dy_ready, hc->up));
+  // Compute stream: forward once X is up and the slot's previous Y has left; backward once dY is
+  // up and the slot's previous dX has left.
+  ETR_CUDA(cudaStreamWaitEvent(st, ev.x_ready, 0));
+  ETR_CUDA(cudaStreamWaitEvent(st, ev.y_down, 0));
+  ETR_TRY(etr_layer_forward(c, sg->X_dev, R, W1g, W1u, W2, b, sg->Y_dev, stream));
+  ETR_CUDA(cudaEventRecord(ev.fwd_done, st));
+  ETR_CUDA(cudaStreamWaitEvent(st, ev.dy_ready, 0));
+  ETR_CUDA(cudaStreamWaitEvent(st, ev.dx_down, 0));
+  ETR_TRY(etr_layer_backward(c, sg->X_dev, R, W1g, W1u, W2, sg->dY_dev, b, sg->dX_dev, dR, dW1g, dW1u,
+                             dW2, stream));
+  ETR_CUDA(cudaEventRecord(ev.bwd_done, st));
+  // Download stream: each result as soon as its pass is done.
+  ETR_CUDA(cudaStreamWaitEvent(hc->down, ev.fwd_done, 0));
+  ETR_CUDA(cudaMemcpyAsync(Y_host, sg->Y_dev, bytes, cudaMemcpyDeviceToHost, hc->down));
+  ETR_CUDA(cudaEventRecord(ev.y_down, hc->down));
+  ETR_CUDA(cudaStreamWaitEvent(hc->down, ev.bwd_done, 0));
+  ETR_CUDA(cudaMemcpyAsync(dX_host, sg->dX_dev, bytes, cudaMemcpyDeviceToHost, hc->down));
+  ETR_CUDA(cudaEventRecord(ev.dx_down, hc->down));
+  ev.used = true;
+  return ETR_OK;
+}
+
+etr_status etr_layer_step_host_wait(int32_t slot) {
+  if (slot < 0 || slot >= ETR_HOST_SLOTS) return ETR_ERR_ARG;
+  HostStepCtx* hc = nullptr;
+  ETR_TRY(host_step_ctx(&hc));
+  if (!hc->slot[slot].used) return ETR_OK;
+  ETR_CUDA(cudaEventSynchronize(hc->slot[slot].dx_down));      // recorded after y_down on the same stream
   return ETR_OK;
 }
 

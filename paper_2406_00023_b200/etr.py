@@ -23,7 +23,8 @@ EXPORTS = [
     "etr_status_string", "etr_validate", "etr_c_stride", "etr_workspace_bytes", "etr_buffers_bytes",
     "etr_buffers_bind", "etr_affinity", "etr_select", "etr_select_static", "etr_dispatch", "etr_expert_ffn", "etr_combine",
     "etr_combine_bwd", "etr_expert_ffn_bwd", "etr_dispatch_bwd", "etr_select_bwd", "etr_affinity_bwd",
-    "etr_layer_forward", "etr_layer_backward", "etr_layer_step_host", "etr_read_stats",
+    "etr_layer_forward", "etr_layer_backward", "etr_layer_step_host", "etr_layer_step_host_begin",
+    "etr_layer_step_host_wait", "etr_read_stats",
     "etr_launch_count", "etr_timing_enable", "etr_timing_collect",
 ]
 
@@ -277,6 +278,35 @@ def layer_backward(cfg, X, R, W1g, W1u, W2, dY, buf: LayerBuffers, dX, dR, dW1g,
     _check(lib().etr_layer_backward(C.byref(cfg), _p(X), _p(R), _p(W1g), _p(W1u), _p(W2), _p(dY),
                                     C.byref(buf.c), _p(dX), _p(dR), _p(dW1g), _p(dW1u), _p(dW2),
                                     _stream()), "etr_layer_backward")
+
+
+class HostSlotC(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("X_dev", "dY_dev", "Y_dev", "dX_dev")]
+
+
+HOST_SLOTS = 4
+
+
+class HostSlot:
+    """Device staging of one host step in flight (four [T, d] tensors of the activation dtype)."""
+
+    def __init__(self, cfg: Config, index: int, device="cuda"):
+        self.index = index
+        self.tensors = [torch.empty(cfg.T, cfg.d, dtype=torch_dtype(cfg), device=device) for _ in range(4)]
+        self.c = HostSlotC(*[C.c_void_p(t.data_ptr()) for t in self.tensors])
+
+
+def layer_step_host_begin(cfg, X_host, dY_host, R, W1g, W1u, W2, buf: "LayerBuffers", slot: HostSlot,
+                          Y_host, dX_host, dR, dW1g, dW1u, dW2):
+    """Enqueues one step from host tensors on `slot` and returns without waiting."""
+    _check(lib().etr_layer_step_host_begin(C.byref(cfg), _p(X_host), _p(dY_host), _p(R), _p(W1g), _p(W1u),
+                                           _p(W2), C.byref(buf.c), C.byref(slot.c), C.c_int32(slot.index),
+                                           _p(Y_host), _p(dX_host), _p(dR), _p(dW1g), _p(dW1u), _p(dW2),
+                                           _stream()), "etr_layer_step_host_begin")
+
+
+def layer_step_host_wait(slot: HostSlot):
+    _check(lib().etr_layer_step_host_wait(C.c_int32(slot.index)), "etr_layer_step_host_wait")
 
 
 def layer_step_host(cfg, X_host, dY_host, R, W1g, W1u, W2, buf: LayerBuffers, Y_host, dX_host, dR,

@@ -304,6 +304,43 @@ def test_layer_is_deterministic_and_host_step_matches():
         assert torch.equal(a[k].cpu(), c[k].cpu()), k
 
 
+def test_pipelined_host_steps_match_the_layer_calls():
+    """Six steps through etr_layer_step_host_begin on two slots, alternating between two different
+    batches, with no wait between them: every step must deliver exactly what the layer calls give
+    for its own batch (slots do not leak into each other, re-use of a slot is ordered)."""
+    w, inp, o, fw, bw = case("small_s")
+    cfg = hz.make_cfg(w)
+    inp2 = dict(inp)
+    inp2["X"] = np.ascontiguousarray(inp["X"][::-1])          # another batch: the tokens reversed
+    inp2["dY"] = np.ascontiguousarray(inp["dY"][::-1] * 0.5)
+    refs = [run_layer(w, q, cfg)[1] for q in (inp, inp2)]
+    dev = hz.upload(w, inp)
+    buf = etr.LayerBuffers(cfg)
+    slots = [etr.HostSlot(cfg, i) for i in range(2)]
+    host = []
+    for q in (inp, inp2):
+        d = hz.upload(w, q)
+        host.append((d.X.cpu().pin_memory(), d.dY.cpu().pin_memory()))
+    outs = [(torch.empty_like(host[0][0]).pin_memory(), torch.empty_like(host[0][0]).pin_memory())
+            for _ in range(6)]
+    g = dict(dR=torch.empty_like(dev.R), dW1g=torch.empty_like(dev.W1g), dW1u=torch.empty_like(dev.W1u),
+             dW2=torch.empty_like(dev.W2))
+    for i in range(6):
+        Xh, dYh = host[i % 2]
+        etr.layer_step_host_begin(cfg, Xh, dYh, dev.R, dev.W1g, dev.W1u, dev.W2, buf, slots[i % 2],
+                                  outs[i][0], outs[i][1], g["dR"], g["dW1g"], g["dW1u"], g["dW2"])
+    for sl in slots:
+        etr.layer_step_host_wait(sl)
+    torch.cuda.synchronize()
+    for i in range(6):
+        assert torch.equal(outs[i][0], refs[i % 2]["Y"].cpu()), ("Y", i)
+        assert torch.equal(outs[i][1], refs[i % 2]["dX"].cpu()), ("dX", i)
+    for k in g:                                               # the last step used the second batch
+        assert torch.equal(g[k], refs[1][k]), k
+    with pytest.raises(etr.EtrError):
+        etr.layer_step_host_wait(etr.HostSlot(cfg, etr.HOST_SLOTS))
+
+
 @pytest.mark.parametrize("name", ["tiny", "small_s", "mid_s"])
 def test_stage_calls_compose_to_the_layer_calls(name):
     """The ten stage entry points called one by one give what etr_layer_forward/backward give.
