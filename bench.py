@@ -38,11 +38,11 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised
 # under profiles/ (absent: not captured for the current version of that kernel).
 NCU_TRAFFIC_BYTES = {}
-# tc_grouped_gemm_pair_kernel: measured on the mid workload, all 7 launches of one step
-# (profiles/tc_grouped_gemm_pair_kernel_mid_ncu_full.md): 3652.0 MB of DRAM traffic against 3799.7 MB
+# tc_grouped_gemm_pair_kernel and its wide form: measured on the mid workload, all 7 launches of one step
+# (profiles/tc_grouped_gemm_pair_kernels_mid_ncu_full.md): 3676.4 MB of DRAM traffic against 3799.7 MB
 # of algorithmic bytes (part of the output is still in L2 when a kernel ends).  The large workload is
 # too big for a multi-pass capture, so its traffic is this ratio times its own algorithmic bytes.
-TC_GEMM_DRAM_OVER_ALGORITHMIC = 3652.0 / 3799.7
+TC_GEMM_DRAM_OVER_ALGORITHMIC = 3676.4 / 3799.7
 
 
 def tc_gemm_algorithmic_bytes(w, rows_padded):
@@ -371,9 +371,9 @@ def main():
         kernels.append({"kernel": name, "launches_per_step": n / args.steps, "ms_per_step": ms / args.steps,
                         "share": ms / sum(v[1] for v in per.values()), "bound": bound,
                         "achieved": ach, "peak": peak, "unit": unit, "frac": ach / peak})
-    # The six tcgen05 contractions are instantiations of one kernel (tc_grouped_gemm_pair_kernel,
-    # or the single-CTA tc_grouped_gemm_kernel when --gemm tcgen05 asks for it); the roofline
-    # entry is that kernel over all its launches when it dominates the step.
+    # The six tcgen05 contractions run on one persistent grouped-GEMM design in two tile forms
+    # (tc_grouped_gemm_pair_kernel and its wide form; --gemm can force one, or the single-CTA
+    # tc_grouped_gemm_kernel); the roofline entry covers all their launches when they dominate.
     tc = [k for k in kernels if k["kernel"].startswith("tc_gemm_")]
     roofline = None
     if tc and sum(k["ms_per_step"] for k in tc) >= 0.5 * sum(k["ms_per_step"] for k in kernels):
@@ -381,8 +381,11 @@ def main():
         ms = sum(k["ms_per_step"] for k in tc)
         n = sum(k["launches_per_step"] for k in tc)
         ach = flops / (ms * 1e-3) / 1e12
-        pair = args.gemm in ("auto", "tcgen05_2cta")
-        roofline = {"kernel": "tc_grouped_gemm_pair_kernel" if pair else "tc_grouped_gemm_kernel",
+        pair = args.gemm == "auto"          # the ncu traffic ratio was taken with the library's own choice
+        kname = {"auto": "tc_grouped_gemm_pair_kernel + tc_grouped_gemm_pair_wide_kernel (chosen per contraction)",
+                 "tcgen05_2cta": "tc_grouped_gemm_pair_kernel", "tcgen05_2cta_wide": "tc_grouped_gemm_pair_wide_kernel",
+                 "tcgen05": "tc_grouped_gemm_kernel"}.get(args.gemm, "tc_grouped_gemm")
+        roofline = {"kernel": kname,
                     "launches_per_step": n, "bound": "tensor",
                     "achieved": ach, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
                     "frac": ach / peaks["bf16_tflops_sustained"],
