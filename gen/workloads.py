@@ -78,6 +78,10 @@ WORKLOADS = {
                       mode="auto", adaptive=True, x_kind="skew", n_clusters=32, step=0),
     "large": Workload("large", 5, T=65536, d=4096, D=16, E=64, k=2, h=2048, cf=1.0, dtype="bf16",
                       mode="ecr", adaptive=True, x_kind="mix", n_clusters=64, step=5000),
+    # The expert shape of the paper's own model (Mixtral 8x7B: 8 experts, d=4096, h=14336) at its
+    # sequence length, with Top-1 routing as in its efficiency runs; early training (TCR).
+    "mixtral_top1": Workload("mixtral_top1", 6, T=32768, d=4096, D=16, E=8, k=1, h=14336, cf=1.0,
+                             dtype="bf16", mode="tcr", adaptive=True, x_kind="mix", n_clusters=64, step=10),
 }
 
 # Training steps of the adaptive-switch sweep (five before the switch, three after)

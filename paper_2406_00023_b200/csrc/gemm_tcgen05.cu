@@ -1204,7 +1204,8 @@ enum TcForm { TC_FORM_SINGLE, TC_FORM_PAIR, TC_FORM_PAIR_WIDE };
 // pair form is taken where its saving in operand traffic outweighs its exposed epilogue: plain
 // stores whose row extent is the expert's token count (down, dXp), and the fused SwiGLU when the
 // contraction is long (>= 48 K blocks); and only when the launch has at least four rounds of wide
-// tiles per CTA pair at full capacity, since a wide tile is twice the unit of work.  Weight
+// tiles per CTA pair at full capacity, since a wide tile is twice the unit of work (small layers
+// fall back to the single-CTA form for those stores, see below).  Weight
 // gradients (short contraction over the expert's rows, large outputs) and the SwiGLU derivative
 // (its epilogue also fetches G and U) measured faster on 256 x 256 tiles.
 static TcForm tc_form_of(const etr_config* c, int epi, const TcParams& p) {
@@ -1214,8 +1215,13 @@ static TcForm tc_form_of(const etr_config* c, int epi, const TcParams& p) {
   if (p.dyn != TC_DYN_M || epi == TC_EPI_DSWIGLU) return TC_FORM_PAIR;
   if (epi == TC_EPI_SWIGLU && ceil_div(p.K, TC_BK) < 48) return TC_FORM_PAIR;
   const int cols = epi == TC_EPI_SWIGLU ? 256 : 512;
+  const long long rounds = 4ll * (sm_count() / 2);
   const long long wide_tiles = (long long)p.E * ceil_div(p.M, 256) * ceil_div(p.N, cols);
-  return wide_tiles >= 4ll * (sm_count() / 2) ? TC_FORM_PAIR_WIDE : TC_FORM_PAIR;
+  if (wide_tiles >= rounds) return TC_FORM_PAIR_WIDE;
+  // Few tiles (small layers): for the plain stores, 128-row tiles on single CTAs balance better and
+  // pad the expert's rows to 128 instead of 256.
+  const long long pair_tiles = (long long)p.E * ceil_div(p.M, 256) * ceil_div(p.N, 256);
+  return (epi == TC_EPI_STORE && pair_tiles < rounds) ? TC_FORM_SINGLE : TC_FORM_PAIR;
 }
 template <int EPI>
 static etr_status tc_run(TcForm form, const char* name, const CUtensorMap& a0, const CUtensorMap& a1,

@@ -1,4 +1,4 @@
-"""Parity at the full sizes of the five workloads, in the launch configuration the benchmark
+"""Parity at the full sizes of the five workloads (and of the Mixtral-shaped Top-1 workload), in the launch configuration the benchmark
 times (etr_layer_forward + etr_layer_backward, default GEMM path).
 
 The routing half is compared in full: the oracle computes every affinity and the complete
@@ -25,16 +25,20 @@ from tests import harness as hz
 pytestmark = pytest.mark.gpu
 etr = hz.etr
 
+# workload, delta_max given to both sides (None: the measured one), rows of the chosen expert that are
+# checked (None: all of them, and with them the expert's whole weight gradients)
 FULL = {
-    "small": (gw.WORKLOADS["small"], -1.0),
-    "mid": (gw.WORKLOADS["mid"], -1.0),
-    "sweep_step600": (gw.sweep_point(2), gw.SWEEP_DELTA_MAX[2]),
-    "sweep_step1500": (gw.sweep_point(6), gw.SWEEP_DELTA_MAX[6]),
-    "sweep_step0_measured": (gw.sweep_point(0), None),
-    "large": (gw.WORKLOADS["large"], None),
+    "small": (gw.WORKLOADS["small"], -1.0, None),
+    "mid": (gw.WORKLOADS["mid"], -1.0, None),
+    "sweep_step600": (gw.sweep_point(2), gw.SWEEP_DELTA_MAX[2], None),
+    "sweep_step1500": (gw.sweep_point(6), gw.SWEEP_DELTA_MAX[6], None),
+    "sweep_step0_measured": (gw.sweep_point(0), None, None),
+    "large": (gw.WORKLOADS["large"], None, None),
+    "mixtral_top1": (gw.WORKLOADS["mixtral_top1"], None, 24),     # 1 GFLOP per row on the CPU
 }
 if os.environ.get("ETR_SKIP_LARGE"):
     FULL.pop("large")
+    FULL.pop("mixtral_top1")
 
 
 def sub_route(E, Cs, n, T):
@@ -48,7 +52,7 @@ def sub_route(E, Cs, n, T):
 
 @pytest.mark.parametrize("name", list(FULL))
 def test_full_size(name):
-    w, dm = FULL[name]
+    w, dm, expert_rows = FULL[name]
     mode = hz.mode_of(w)
     o = ob.Oracle("f32")
     inp = gw.make_inputs(w)
@@ -109,7 +113,8 @@ def test_full_size(name):
     # ---- one whole expert -------------------------------------------------------------------------------
     ragged = [i for i in range(E) if counts[i] % 128 != 0 and counts[i] > 0]
     i = ragged[len(ragged) // 2] if ragged else E - 1
-    n = int(counts[i])
+    n_all = int(counts[i])
+    n = n_all if expert_rows is None else min(n_all, expert_rows)      # rows are independent of each other
     r0 = i * Cs
     toks = got.slot_token[r0:r0 + n]
     gate = got.gate[r0:r0 + n]
@@ -133,21 +138,23 @@ def test_full_size(name):
     hz.assert_close_rms(hz.to_np(buf.dG[rows]), dG[:n], tol, "dG", chain=3)
     hz.assert_close_rms(hz.to_np(buf.dU[rows]), dU[:n], tol, "dU", chain=3)
     hz.assert_close_rms(hz.to_np(buf.dXp[rows]), dXp[:n], tol, "dXp", chain=5)
-    hz.assert_close_rms(hz.to_np(out["dW1g"][i]), dW1g_i[0], tol, "dW1g[i]", chain=6)
-    hz.assert_close_rms(hz.to_np(out["dW1u"][i]), dW1u_i[0], tol, "dW1u[i]", chain=6)
-    hz.assert_close_rms(hz.to_np(out["dW2"][i]), dW2_i[0], tol, "dW2[i]", chain=4)
-    # dR[i] from this expert's tokens only
-    dd = np.zeros((n, E), np.float32)
-    dd[:, i] = dgate
-    _, dR_sub = o.affinity_bwd(X[toks], R, D, delta[toks], xnorm[toks], rnorm, dd, np.zeros((n, d), np.float32))
-    hz.assert_close_rms(hz.to_np(out["dR"][i]), dR_sub[i], tol, "dR[i]")
+    if n == n_all:          # sums over all the expert's rows
+        hz.assert_close_rms(hz.to_np(out["dW1g"][i]), dW1g_i[0], tol, "dW1g[i]", chain=6)
+        hz.assert_close_rms(hz.to_np(out["dW1u"][i]), dW1u_i[0], tol, "dW1u[i]", chain=6)
+        hz.assert_close_rms(hz.to_np(out["dW2"][i]), dW2_i[0], tol, "dW2[i]", chain=4)
+        # dR[i] from this expert's tokens only
+        dd = np.zeros((n, E), np.float32)
+        dd[:, i] = dgate
+        _, dR_sub = o.affinity_bwd(X[toks], R, D, delta[toks], xnorm[toks], rnorm, dd, np.zeros((n, d), np.float32))
+        hz.assert_close_rms(hz.to_np(out["dR"][i]), dR_sub[i], tol, "dR[i]")
 
     # ---- sampled tokens: Y[t] and dX[t] through every row of the token ------------------------------------------
     rng = np.random.default_rng(w.seed)
     nrows_t = np.diff(got.tok_ptr)
     routed = np.nonzero(nrows_t > 0)[0]
     multi = np.nonzero(nrows_t > 1)[0]
-    pick = list(rng.choice(routed, 6, replace=False)) + list(rng.choice(multi, min(4, len(multi)), replace=False))
+    n_tok = 6 if expert_rows is None else 3
+    pick = list(rng.choice(routed, n_tok, replace=False)) + (list(rng.choice(multi, min(4, len(multi)), replace=False)) if len(multi) else [])
     # RMS of the whole tensors over the routed tokens (unrouted rows are exact zeros)
     scale = np.sqrt(T / max(1, len(routed)))
     y_rms = float(out["Y"].float().pow(2).mean().sqrt()) * scale
