@@ -41,7 +41,11 @@ def layer_vs_oracle(w, inp, mode, impl=etr.GEMM_AUTO):
     return fw, got, out
 
 
-@pytest.mark.parametrize("dtype,impl", [("f32", etr.GEMM_AUTO), ("bf16", etr.GEMM_AUTO), ("bf16", etr.GEMM_SIMT)])
+TC_FORMS = [etr.GEMM_TCGEN05, etr.GEMM_TCGEN05_2CTA, etr.GEMM_TCGEN05_2CTA_WIDE]
+
+
+@pytest.mark.parametrize("dtype,impl", [("f32", etr.GEMM_AUTO), ("bf16", etr.GEMM_AUTO), ("bf16", etr.GEMM_SIMT)]
+                         + [("bf16", f) for f in TC_FORMS])
 def test_experts_without_tokens_get_zero_gradients(dtype, impl):
     """Token choice with every token pushed away from experts 2 and 5: their buffers stay
     empty, their weight gradients must be exactly zero, everything else must match."""
@@ -58,17 +62,28 @@ def test_experts_without_tokens_get_zero_gradients(dtype, impl):
     assert bool((out["dR"][2] == 0).all())
 
 
+@pytest.mark.parametrize("impl", [etr.GEMM_AUTO] + TC_FORMS)
 @pytest.mark.parametrize("k", [1, 8])
-def test_top1_and_top_all(k):
+def test_top1_and_top_all(k, impl):
+    """h = 192 and d = 256 leave ragged column tiles in every tile form."""
     w = gw.scaled(W["small"], T=300, d=256, D=8, E=8, h=192, k=k, cf=0.8)
-    layer_vs_oracle(w, gw.make_inputs(w), ob.MODE_TCR)
+    layer_vs_oracle(w, gw.make_inputs(w), ob.MODE_TCR, impl)
 
 
+@pytest.mark.parametrize("impl", [etr.GEMM_AUTO] + TC_FORMS)
 @pytest.mark.parametrize("mode", [ob.MODE_TCR, ob.MODE_ECR])
-def test_capacity_one_and_few_tokens(mode):
+def test_capacity_one_and_few_tokens(mode, impl):
     w = gw.scaled(W["small"], T=5, d=128, D=8, E=4, h=64, cf=0.2)
     assert w.capacity == 1
-    layer_vs_oracle(w, gw.make_inputs(w), mode)
+    layer_vs_oracle(w, gw.make_inputs(w), mode, impl)
+
+
+@pytest.mark.parametrize("impl", TC_FORMS)
+def test_wide_columns_with_a_ragged_second_half(impl):
+    """d = 640 and h = 320: the 512-column tiles of the wide form end in a partial second half
+    (640 = 512 + 128) or have none at all (320), with 700 tokens per expert at most (ragged rows)."""
+    w = gw.scaled(W["small"], T=1400, d=640, D=8, E=4, h=320, cf=1.0)
+    layer_vs_oracle(w, gw.make_inputs(w), ob.MODE_ECR, impl)
 
 
 @pytest.mark.parametrize("D,dtype", [(1, "f32"), (2, "bf16"), (4, "bf16"), (32, "bf16"), (24, "f32")])
