@@ -211,6 +211,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="large", choices=list(gw.WORKLOADS))
     ap.add_argument("--gemm", default="auto", choices=["auto", "simt", "tcgen05", "tcgen05_2cta", "tcgen05_2cta_wide"])
+    ap.add_argument("--fuse", default="auto", choices=["auto", "off", "on"],
+                    help="token rearrangement fused into the GEMM operand fetch (TMA row gathers)")
     ap.add_argument("--cpu-tokens", type=int, default=128, help="tokens in the CPU-oracle sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--set", default="", help="override workload fields, e.g. T=32768,h=512 (profiling cases)")
@@ -272,7 +274,8 @@ def main():
     cfg = etr.make_config(T=w.T, d=w.d, D=w.D, E=w.E, k=w.k, h=w.h, capacity=w.capacity,
                           dtype=etr.BF16 if w.dtype == "bf16" else etr.F32,
                           mode=etr.MODE_TCR if mode_name(w) == "tcr" else etr.MODE_ECR,
-                          step=w.step, switch_step=w.switch_step, adaptive=w.adaptive, gemm_impl=impl)
+                          step=w.step, switch_step=w.switch_step, adaptive=w.adaptive, gemm_impl=impl,
+                          fuse_dispatch={"auto": etr.FUSE_AUTO, "off": etr.FUSE_OFF, "on": etr.FUSE_ON}[args.fuse])
     buf = etr.LayerBuffers(cfg, host_staging=True, device=dev)
     Y, dX = torch.empty_like(X), torch.empty_like(X)
     dR = torch.empty_like(R)

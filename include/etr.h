@@ -63,6 +63,12 @@ typedef enum { ETR_MODE_AUTO = 0, ETR_MODE_TCR = 1, ETR_MODE_ECR = 2 } etr_mode;
 typedef enum { ETR_GEMM_AUTO = 0, ETR_GEMM_SIMT = 1, ETR_GEMM_TCGEN05 = 2, ETR_GEMM_TCGEN05_2CTA = 3,
                ETR_GEMM_TCGEN05_2CTA_WIDE = 4 } etr_gemm_impl;
 
+/* etr_layer_forward/backward on the tensor-core path can skip the token rearrangement: the first
+ * FFN GEMM and the W1 weight-gradient GEMMs then fetch their token rows straight from X with TMA
+ * row gathers (four rows per request, named by slot_token), and buf->Xp is neither written nor
+ * read.  The stage calls are unaffected.  ETR_FUSE_AUTO lets the library choose. */
+typedef enum { ETR_FUSE_AUTO = 0, ETR_FUSE_OFF = 1, ETR_FUSE_ON = 2 } etr_fuse;
+
 /* Immutable description of one layer call (host struct, passed by pointer). */
 typedef struct etr_config {
   int32_t T, d, D, E, k, h;
@@ -73,8 +79,8 @@ typedef struct etr_config {
   int64_t step, switch_step;  /* ETR_MODE_AUTO: token choice while step < switch_step */
   int32_t mode;               /* etr_mode */
   int32_t dtype;              /* etr_dtype of activations and expert weights */
-  int32_t gemm_impl;          /* etr_gemm_impl; AUTO = two-CTA tcgen05 for bf16, SIMT for fp32 */
-  int32_t reserved;
+  int32_t gemm_impl;          /* etr_gemm_impl; AUTO = CTA-pair tcgen05 for bf16, SIMT for fp32 */
+  int32_t fuse_dispatch;      /* etr_fuse: token rearrangement fused into the GEMM operand fetch */
 } etr_config;
 
 /* Per-call scalars produced and consumed on the device (device struct, 64 bytes). */

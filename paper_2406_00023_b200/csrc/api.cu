@@ -44,6 +44,11 @@ static bool use_tc(const etr_config* c) {
   return c->dtype == ETR_BF16 && tc_available();
 }
 
+// Token rearrangement fused into the GEMM operand fetch (layer calls, tensor-core path only).
+static bool fuse_dispatch(const etr_config* c) {
+  return use_tc(c) && c->fuse_dispatch == ETR_FUSE_ON;
+}
+
 static etr_status check_ptrs(std::initializer_list<const void*> ps) {
   for (const void* p : ps) {
     if (p == nullptr) return ETR_ERR_ARG;
@@ -135,6 +140,7 @@ etr_status etr_validate(const etr_config* c) {
   if (c->dtype != ETR_F32 && c->dtype != ETR_BF16) return ETR_ERR_ARG;
   if (c->mode < ETR_MODE_AUTO || c->mode > ETR_MODE_ECR) return ETR_ERR_ARG;
   if (c->gemm_impl < ETR_GEMM_AUTO || c->gemm_impl > ETR_GEMM_TCGEN05_2CTA_WIDE) return ETR_ERR_ARG;
+  if (c->fuse_dispatch < ETR_FUSE_AUTO || c->fuse_dispatch > ETR_FUSE_ON) return ETR_ERR_ARG;
   if (c->d % c->D != 0 || c->d % 8 != 0 || c->h % 8 != 0) return ETR_ERR_SHAPE;
   if (c->k > c->E || c->E > 256 || c->E > c->d / c->D) return ETR_ERR_SHAPE;
   if ((long long)c->T * c->E >= (1ll << 31)) return ETR_ERR_SHAPE;
@@ -209,7 +215,7 @@ etr_status etr_expert_ffn(const etr_config* c, const etr_route* route, const voi
   ETR_TRY(check_route(route));
   if (use_tc(c)) {
     ETR_TRY(check_ptrs({stats, ws}));
-    return tc_ffn_forward(c, route, Xp, W1g, W1u, W2, G, U, H, O, stats, ws, (cudaStream_t)stream);
+    return tc_ffn_forward(c, route, Xp, nullptr, W1g, W1u, W2, G, U, H, O, stats, ws, (cudaStream_t)stream);
   }
   return simt_ffn_forward(c, route, Xp, W1g, W1u, W2, G, U, H, O, (cudaStream_t)stream);
 }
@@ -240,7 +246,7 @@ etr_status etr_expert_ffn_bwd(const etr_config* c, const etr_route* route, const
   ETR_TRY(check_route(route));
   if (use_tc(c)) {
     ETR_TRY(check_ptrs({stats, ws}));
-    return tc_ffn_backward(c, route, dO, Xp, G, U, H, W1g, W1u, W2, dG, dU, dXp, dW1g, dW1u, dW2,
+    return tc_ffn_backward(c, route, dO, Xp, nullptr, G, U, H, W1g, W1u, W2, dG, dU, dXp, dW1g, dW1u, dW2,
                            stats, ws, (cudaStream_t)stream);
   }
   return simt_ffn_backward(c, route, dO, Xp, G, U, H, W1g, W1u, W2, dG, dU, dXp, dW1g, dW1u, dW2,
@@ -282,9 +288,15 @@ etr_status etr_layer_forward(const etr_config* c, const void* X, const float* R,
     return ETR_ERR_CUDA;
   ETR_TRY(etr_affinity(c, X, R, b->delta, b->Z, b->xnorm, b->rnorm, b->stats, stream));
   ETR_TRY(etr_select(c, b->delta, b->stats, &b->route, b->ws, stream));
-  ETR_TRY(etr_dispatch(c, X, &b->route, b->Xp, stream));
-  ETR_TRY(etr_expert_ffn(c, &b->route, b->Xp, W1g, W1u, W2, b->G, b->U, b->H, b->O, b->stats, b->ws,
-                         stream));
+  if (fuse_dispatch(c)) {       // the first GEMM gathers its rows from X: no Xp
+    ETR_TRY(check_ptrs({X, W1g, W1u, W2, b->G, b->U, b->H, b->O, b->ws}));
+    ETR_TRY(tc_ffn_forward(c, &b->route, nullptr, X, W1g, W1u, W2, b->G, b->U, b->H, b->O, b->stats, b->ws,
+                           (cudaStream_t)stream));
+  } else {
+    ETR_TRY(etr_dispatch(c, X, &b->route, b->Xp, stream));
+    ETR_TRY(etr_expert_ffn(c, &b->route, b->Xp, W1g, W1u, W2, b->G, b->U, b->H, b->O, b->stats, b->ws,
+                           stream));
+  }
   return etr_combine(c, &b->route, b->O, Y, stream);
 }
 
@@ -293,8 +305,16 @@ etr_status etr_layer_backward(const etr_config* c, const void* X, const float* R
                               void* dX, float* dR, void* dW1g, void* dW1u, void* dW2, void* stream) {
   if (b == nullptr) return ETR_ERR_ARG;
   ETR_TRY(etr_combine_bwd(c, &b->route, dY, b->O, b->dO, b->dgate, stream));
-  ETR_TRY(etr_expert_ffn_bwd(c, &b->route, b->dO, b->Xp, b->G, b->U, b->H, W1g, W1u, W2, b->dG, b->dU,
-                             b->dXp, dW1g, dW1u, dW2, b->stats, b->ws, stream));
+  if (fuse_dispatch(c)) {
+    ETR_TRY(etr_validate(c));
+    ETR_TRY(check_ptrs({X, b->dO, b->G, b->U, b->H, W1g, W1u, W2, b->dG, b->dU, b->dXp, dW1g, dW1u, dW2,
+                        b->stats, b->ws}));
+    ETR_TRY(tc_ffn_backward(c, &b->route, b->dO, nullptr, X, b->G, b->U, b->H, W1g, W1u, W2, b->dG, b->dU,
+                            b->dXp, dW1g, dW1u, dW2, b->stats, b->ws, (cudaStream_t)stream));
+  } else {
+    ETR_TRY(etr_expert_ffn_bwd(c, &b->route, b->dO, b->Xp, b->G, b->U, b->H, W1g, W1u, W2, b->dG, b->dU,
+                               b->dXp, dW1g, dW1u, dW2, b->stats, b->ws, stream));
+  }
   // dispatch backward and the router gradient in one pass over dX
   ETR_TRY(etr_select_bwd(c, &b->route, b->dgate));
   ETR_TRY(check_ptrs({X, R, dX, dR, b->dXp, b->ws}));

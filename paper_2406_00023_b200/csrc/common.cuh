@@ -132,12 +132,13 @@ etr_status simt_ffn_backward(const etr_config* cfg, const etr_route* route, cons
                              const void* Xp, const void* G, const void* U, const void* H,
                              const void* W1g, const void* W1u, const void* W2, void* dG, void* dU,
                              void* dXp, void* dW1g, void* dW1u, void* dW2, cudaStream_t st);
-// tcgen05 grouped GEMMs (bf16 only).
-etr_status tc_ffn_forward(const etr_config* cfg, const etr_route* route, const void* Xp,
+// tcgen05 grouped GEMMs (bf16 only).  X_tokens != nullptr: the token rows are gathered from X
+// through route->slot_token and Xp is not read (may be nullptr).
+etr_status tc_ffn_forward(const etr_config* cfg, const etr_route* route, const void* Xp, const void* X_tokens,
                           const void* W1g, const void* W1u, const void* W2, void* G, void* U,
                           void* H, void* O, etr_stats* stats, void* ws, cudaStream_t st);
 etr_status tc_ffn_backward(const etr_config* cfg, const etr_route* route, const void* dO,
-                           const void* Xp, const void* G, const void* U, const void* H,
+                           const void* Xp, const void* X_tokens, const void* G, const void* U, const void* H,
                            const void* W1g, const void* W1u, const void* W2, void* dG, void* dU,
                            void* dXp, void* dW1g, void* dW1u, void* dW2, etr_stats* stats,
                            void* ws, cudaStream_t st);

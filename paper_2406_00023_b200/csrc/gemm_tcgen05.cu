@@ -49,6 +49,15 @@ struct TcParams {
   int ld_out;
   uint32_t idesc;
   etr_stats* stats;
+  // Row gather (token rearrangement fused into the operand fetch): the rows of one operand are
+  // rows of the token matrix X named by slot_token, fetched four at a time by TMA gather.
+  // gather 1: the A operand's rows (row r of expert e is token slot_token[e*gather_ld + r]);
+  // gather 2: the B operand's K rows (contractions over the expert's rows).  Slots holding -1 fetch
+  // row gather_oob, which lies outside X and reads as zeros.  The gathered operand's map is mapA0
+  // (gather 1) or mapB0 (gather 2), a 2-D map of X with a one-row box.
+  int gather;
+  int gather_ld, gather_oob;
+  const int32_t* gather_idx;
 };
 
 // ---- PTX wrappers -----------------------------------------------------------------------------
@@ -562,6 +571,21 @@ __device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap
       " [%0], [%1, {%3, %4, %5}], [%2];"
       ::"r"(dst), "l"(map), "r"(bar_cluster), "r"(c0), "r"(c1), "r"(c2) : "memory");
 }
+// Four rows of a 2-D tensor (one-row box of 64 columns), 4 x 128 bytes written consecutively.
+__device__ __forceinline__ void tma_gather4_pair(uint32_t dst, const CUtensorMap* map, uint32_t bar_cluster,
+                                                 int col, int4 rows) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile::gather4.mbarrier::complete_tx::bytes.cta_group::2"
+      " [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar_cluster), "r"(col), "r"(rows.x), "r"(rows.y), "r"(rows.z), "r"(rows.w)
+      : "memory");
+}
+// Token ids of four consecutive slots, -1 replaced by the out-of-range row.
+__device__ __forceinline__ int4 gather_rows(const int32_t* idx, int oob) {
+  int4 r = __ldg(reinterpret_cast<const int4*>(idx));
+  r.x = r.x < 0 ? oob : r.x; r.y = r.y < 0 ? oob : r.y; r.z = r.z < 0 ? oob : r.z; r.w = r.w < 0 ? oob : r.w;
+  return r;
+}
 __device__ __forceinline__ void tc_commit_pair(uint32_t bar) {      // arrives on `bar` in both CTAs
   const uint16_t mask = 3;
   asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
@@ -653,16 +677,28 @@ tc_grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap mapA0, const __g
 
   if (warp == 0) {
     // ---- TMA producer (both CTAs) ---------------------------------------------------------------
-    if (lane == 0) {
+    // Without a gather lane 0 works alone.  With one, the whole warp walks the loop: lane l
+    // fetches rows 4l..4l+3 of the gathered operand's 128 (gather 1) or, for the two 64-column
+    // boxes of a K block, rows 4(l%16)..+3 of box l/16 (gather 2); lane 0 issues the rest.
+    if (lane == 0 || p.gather) {
       int e_cur = 0, stage = 0;
       uint32_t phase = 0;
       TileCoord tc;
       bool ok = true;
       for (int tile = pair; ok && tile_coord_pair(p, tile_prefix, tile, e_cur, N_TILE_COLS, tc); tile += npairs) {
         const int m0c = tc.m0 + 128 * (int)rank;
+        const int32_t* gidx = p.gather_idx + (size_t)tc.e * p.gather_ld;
+        int4 rows_a = make_int4(0, 0, 0, 0), rows_b = make_int4(0, 0, 0, 0);
+        if (p.gather == 1)      // a CTA's 128 rows lie inside the expert's C_stride slots or all past them
+          rows_a = m0c < p.M ? gather_rows(gidx + m0c + 4 * lane, p.gather_oob)
+                             : make_int4(p.gather_oob, p.gather_oob, p.gather_oob, p.gather_oob);
+        if (p.gather == 2 && tc.kblocks > 0) rows_b = gather_rows(gidx + 4 * (lane & 15), p.gather_oob);
         for (int kb = 0; kb < tc.kblocks; ++kb) {
+          int4 rows_next = rows_b;
+          if (p.gather == 2 && kb + 1 < tc.kblocks)
+            rows_next = gather_rows(gidx + (kb + 1) * TC_BK + 4 * (lane & 15), p.gather_oob);
           if (!mbar_wait_cluster(empty_bar + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
-          if (rank == 0) mbar_expect_tx(full_bar + 8 * stage, 2 * TC2_STAGE_BYTES);
+          if (rank == 0 && lane == 0) mbar_expect_tx(full_bar + 8 * stage, 2 * TC2_STAGE_BYTES);
           const uint32_t fb = leader_full + 8 * stage;
           const bool second = p.k1_blocks > 0 && kb >= p.k1_blocks;
           const int k0 = (second ? kb - p.k1_blocks : kb) * TC_BK;
@@ -671,13 +707,24 @@ tc_grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap mapA0, const __g
           const int nb = p.dual_b ? tc.n0 : tc.n0 + 128 * (int)rank;
           const uint32_t sa = tiles_base + stage * TC2_STAGE_BYTES;
           const uint32_t sb = sa + 2 * TC_BOX_BYTES;
+          if (p.gather == 1) tma_gather4_pair(sa + 512u * lane, &mapA0, fb, k0, rows_a);
+          if (p.gather == 2)
+            tma_gather4_pair(sb + (lane >> 4) * TC_BOX_BYTES + 512u * (lane & 15), &mapB0, fb,
+                             nb + 64 * (lane >> 4), rows_b);
+          if (lane == 0) {
 #pragma unroll
-          for (int j = 0; j < 2; ++j) {
-            if (p.a_mn) tma_load_3d_pair(sa + j * TC_BOX_BYTES, ma, fb, m0c + 64 * j, k0, tc.e);
-            else        tma_load_3d_pair(sa + j * TC_BOX_BYTES, ma, fb, k0, m0c + 64 * j, tc.e);
-            if (p.b_mn) tma_load_3d_pair(sb + j * TC_BOX_BYTES, mb, fb, nb + 64 * j, k0, tc.e);
-            else        tma_load_3d_pair(sb + j * TC_BOX_BYTES, mb, fb, k0, nb + 64 * j, tc.e);
+            for (int j = 0; j < 2; ++j) {
+              if (p.gather != 1) {
+                if (p.a_mn) tma_load_3d_pair(sa + j * TC_BOX_BYTES, ma, fb, m0c + 64 * j, k0, tc.e);
+                else        tma_load_3d_pair(sa + j * TC_BOX_BYTES, ma, fb, k0, m0c + 64 * j, tc.e);
+              }
+              if (p.gather != 2) {
+                if (p.b_mn) tma_load_3d_pair(sb + j * TC_BOX_BYTES, mb, fb, nb + 64 * j, k0, tc.e);
+                else        tma_load_3d_pair(sb + j * TC_BOX_BYTES, mb, fb, k0, nb + 64 * j, tc.e);
+              }
+            }
           }
+          rows_b = rows_next;
           if (++stage == TC2_STAGES) { stage = 0; phase ^= 1u; }
         }
       }
@@ -863,7 +910,9 @@ tc_grouped_gemm_pair_wide_kernel(const __grid_constant__ CUtensorMap mapA0, cons
 
   if (warp == 0) {
     // ---- TMA producer (both CTAs) ---------------------------------------------------------------
-    if (lane == 0) {
+    // Lane 0 alone, or with a gathered A operand the whole warp (lane l fetches rows 4l..4l+3 of
+    // the CTA's 128 rows of A; lane 0 also issues the B boxes).
+    if (lane == 0 || p.gather) {
       int e_cur = 0, stage = 0;
       uint32_t phase = 0;
       TileCoord tc;
@@ -871,28 +920,37 @@ tc_grouped_gemm_pair_wide_kernel(const __grid_constant__ CUtensorMap mapA0, cons
       for (int tile = pair; ok && tile_coord_wide(p, tile_prefix, tile, e_cur, N_TILE_COLS, tc); tile += npairs) {
         const int m0c = tc.m0 + 128 * (int)rank;
         const bool two = tc.n0 + N_TILE_COLS < p.N;
+        int4 rows_a = make_int4(0, 0, 0, 0);
+        if (p.gather == 1)
+          rows_a = m0c < p.M ? gather_rows(p.gather_idx + (size_t)tc.e * p.gather_ld + m0c + 4 * lane, p.gather_oob)
+                             : make_int4(p.gather_oob, p.gather_oob, p.gather_oob, p.gather_oob);
         for (int kb = 0; kb < tc.kblocks; ++kb) {
           if (!mbar_wait_cluster(empty_bar + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
-          if (rank == 0) mbar_expect_tx(full_bar + 8 * stage, 2 * (two ? 6 : 4) * TC_BOX_BYTES);
+          if (rank == 0 && lane == 0) mbar_expect_tx(full_bar + 8 * stage, 2 * (two ? 6 : 4) * TC_BOX_BYTES);
           const uint32_t fb = leader_full + 8 * stage;
           const bool second = p.k1_blocks > 0 && kb >= p.k1_blocks;
           const int k0 = (second ? kb - p.k1_blocks : kb) * TC_BK;
           const CUtensorMap* ma = second ? &mapA1 : &mapA0;
           const CUtensorMap* mb = p.dual_b ? (rank ? &mapB1 : &mapB0) : (second ? &mapB1 : &mapB0);
           const uint32_t sa = tiles_base + stage * TCW_STAGE_BYTES;
+          if (p.gather == 1) tma_gather4_pair(sa + 512u * lane, &mapA0, fb, k0, rows_a);
+          if (lane == 0) {
+            if (p.gather != 1) {
 #pragma unroll
-          for (int j = 0; j < 2; ++j) {
-            if (p.a_mn) tma_load_3d_pair(sa + j * TC_BOX_BYTES, ma, fb, m0c + 64 * j, k0, tc.e);
-            else        tma_load_3d_pair(sa + j * TC_BOX_BYTES, ma, fb, k0, m0c + 64 * j, tc.e);
-          }
-          for (int hf = 0; hf < (two ? 2 : 1); ++hf) {
-            const uint32_t sb = sa + (2 + 2 * hf) * TC_BOX_BYTES;
-            const int nh = tc.n0 + hf * N_TILE_COLS;
-            const int nb = p.dual_b ? nh : nh + 128 * (int)rank;
+              for (int j = 0; j < 2; ++j) {
+                if (p.a_mn) tma_load_3d_pair(sa + j * TC_BOX_BYTES, ma, fb, m0c + 64 * j, k0, tc.e);
+                else        tma_load_3d_pair(sa + j * TC_BOX_BYTES, ma, fb, k0, m0c + 64 * j, tc.e);
+              }
+            }
+            for (int hf = 0; hf < (two ? 2 : 1); ++hf) {
+              const uint32_t sb = sa + (2 + 2 * hf) * TC_BOX_BYTES;
+              const int nh = tc.n0 + hf * N_TILE_COLS;
+              const int nb = p.dual_b ? nh : nh + 128 * (int)rank;
 #pragma unroll
-            for (int j = 0; j < 2; ++j) {
-              if (p.b_mn) tma_load_3d_pair(sb + j * TC_BOX_BYTES, mb, fb, nb + 64 * j, k0, tc.e);
-              else        tma_load_3d_pair(sb + j * TC_BOX_BYTES, mb, fb, k0, nb + 64 * j, tc.e);
+              for (int j = 0; j < 2; ++j) {
+                if (p.b_mn) tma_load_3d_pair(sb + j * TC_BOX_BYTES, mb, fb, nb + 64 * j, k0, tc.e);
+                else        tma_load_3d_pair(sb + j * TC_BOX_BYTES, mb, fb, k0, nb + 64 * j, tc.e);
+              }
             }
           }
           if (++stage == TCW_STAGES) { stage = 0; phase ^= 1u; }
@@ -1091,6 +1149,21 @@ static etr_status make_map(CUtensorMap* m, const void* base, int cols, int rows,
   return r == CUDA_SUCCESS ? ETR_OK : ETR_ERR_CUDA;
 }
 
+// Row-major bf16 token matrix [T, d] as a 2-D map (d, T) with a one-row box of 64 columns, for row
+// gathers; rows at or past T read as zeros.
+static etr_status make_gather_map(CUtensorMap* m, const void* base, int cols, int rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return ETR_ERR_CUDA;
+  const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+  const cuuint32_t box[2] = {64, 1};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box,
+                        estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                        CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? ETR_OK : ETR_ERR_CUDA;
+}
+
 static uint32_t make_idesc(int a_mn, int b_mn, int n, int m_instr = TC_BM) {
   uint32_t d = 0;
   d |= 1u << 4;                     // accumulator fp32
@@ -1209,6 +1282,10 @@ enum TcForm { TC_FORM_SINGLE, TC_FORM_PAIR, TC_FORM_PAIR_WIDE };
 // gradients (short contraction over the expert's rows, large outputs) and the SwiGLU derivative
 // (its epilogue also fetches G and U) measured faster on 256 x 256 tiles.
 static TcForm tc_form_of(const etr_config* c, int epi, const TcParams& p) {
+  if (p.gather) {      // the pair kernels fetch gathered rows; wide only where it is chosen anyway
+    if (c->gemm_impl == ETR_GEMM_TCGEN05_2CTA_WIDE && p.gather == 1) return TC_FORM_PAIR_WIDE;
+    if (c->gemm_impl != ETR_GEMM_AUTO || p.gather == 2) return TC_FORM_PAIR;
+  }
   if (c->gemm_impl == ETR_GEMM_TCGEN05) return TC_FORM_SINGLE;
   if (c->gemm_impl == ETR_GEMM_TCGEN05_2CTA) return TC_FORM_PAIR;
   if (c->gemm_impl == ETR_GEMM_TCGEN05_2CTA_WIDE) return TC_FORM_PAIR_WIDE;
@@ -1221,7 +1298,7 @@ static TcForm tc_form_of(const etr_config* c, int epi, const TcParams& p) {
   // Few tiles (small layers): for the plain stores, 128-row tiles on single CTAs balance better and
   // pad the expert's rows to 128 instead of 256.
   const long long pair_tiles = (long long)p.E * ceil_div(p.M, 256) * ceil_div(p.N, 256);
-  return (epi == TC_EPI_STORE && pair_tiles < rounds) ? TC_FORM_SINGLE : TC_FORM_PAIR;
+  return (epi == TC_EPI_STORE && pair_tiles < rounds && !p.gather) ? TC_FORM_SINGLE : TC_FORM_PAIR;
 }
 template <int EPI>
 static etr_status tc_run(TcForm form, const char* name, const CUtensorMap& a0, const CUtensorMap& a1,
@@ -1235,12 +1312,13 @@ static etr_status tc_run(TcForm form, const char* name, const CUtensorMap& a0, c
 size_t tc_workspace_bytes(const etr_config*) { return 0; }
 bool tc_available() { return true; }
 
-etr_status tc_ffn_forward(const etr_config* c, const etr_route* rt, const void* Xp, const void* W1g,
+etr_status tc_ffn_forward(const etr_config* c, const etr_route* rt, const void* Xp, const void* Xtok, const void* W1g,
                           const void* W1u, const void* W2, void* G, void* U, void* H, void* O,
                           etr_stats* stats, void*, cudaStream_t st) {
   const int d = c->d, h = c->h, Cs = c_stride_of(c), E = c->E;
   CUtensorMap mXp, mW1g, mW1u, mW2, mH;
-  ETR_TRY(make_map(&mXp, Xp, d, Cs, E));
+  if (Xtok) ETR_TRY(make_gather_map(&mXp, Xtok, d, c->T));
+  else ETR_TRY(make_map(&mXp, Xp, d, Cs, E));
   ETR_TRY(make_map(&mW1g, W1g, d, h, E));
   ETR_TRY(make_map(&mW1u, W1u, d, h, E));
   ETR_TRY(make_map(&mW2, W2, h, d, E));
@@ -1248,6 +1326,7 @@ etr_status tc_ffn_forward(const etr_config* c, const etr_route* rt, const void* 
   const int mt = Cs / TC_BM;
   {  // G, U, H = SwiGLU(Xp W1g^T, Xp W1u^T)
     TcParams p = {};
+    if (Xtok) { p.gather = 1; p.gather_ld = Cs; p.gather_oob = c->T; p.gather_idx = rt->slot_token; }
     p.dual_b = 1; p.M = Cs; p.N = h; p.K = d; p.dyn = TC_DYN_M; p.E = E; p.counts = rt->counts;
     p.out0 = (__nv_bfloat16*)G; p.out1 = (__nv_bfloat16*)U; p.out2 = (__nv_bfloat16*)H;
     p.out_bs = (long long)Cs * h; p.ld_out = h; p.stats = stats;
@@ -1264,13 +1343,14 @@ etr_status tc_ffn_forward(const etr_config* c, const etr_route* rt, const void* 
 }
 
 etr_status tc_ffn_backward(const etr_config* c, const etr_route* rt, const void* dO, const void* Xp,
-                           const void* G, const void* U, const void* H, const void* W1g,
+                           const void* Xtok, const void* G, const void* U, const void* H, const void* W1g,
                            const void* W1u, const void* W2, void* dG, void* dU, void* dXp, void* dW1g,
                            void* dW1u, void* dW2, etr_stats* stats, void*, cudaStream_t st) {
   const int d = c->d, h = c->h, Cs = c_stride_of(c), E = c->E;
   CUtensorMap mdO, mXp, mH, mdG, mdU, mW1g, mW1u, mW2;
   ETR_TRY(make_map(&mdO, dO, d, Cs, E));
-  ETR_TRY(make_map(&mXp, Xp, d, Cs, E));
+  if (Xtok) ETR_TRY(make_gather_map(&mXp, Xtok, d, c->T));
+  else ETR_TRY(make_map(&mXp, Xp, d, Cs, E));
   ETR_TRY(make_map(&mH, H, h, Cs, E));
   ETR_TRY(make_map(&mdG, dG, h, Cs, E));
   ETR_TRY(make_map(&mdU, dU, h, Cs, E));
@@ -1305,6 +1385,7 @@ etr_status tc_ffn_backward(const etr_config* c, const etr_route* rt, const void*
   for (int which = 0; which < 2; ++which) {  // dW1g = dG^T Xp, dW1u = dU^T Xp
     TcParams p = {};
     p.a_mn = 1; p.b_mn = 1; p.M = h; p.N = d; p.dyn = TC_DYN_K; p.E = E; p.counts = rt->counts;
+    if (Xtok) { p.gather = 2; p.gather_ld = Cs; p.gather_oob = c->T; p.gather_idx = rt->slot_token; }
     p.out0 = (__nv_bfloat16*)(which ? dW1u : dW1g); p.out_bs = (long long)h * d; p.ld_out = d; p.stats = stats;
     const CUtensorMap& ma = which ? mdU : mdG;
     ETR_TRY((tc_run<TC_EPI_STORE>(tc_form_of(c, TC_EPI_STORE, p), "tc_gemm_dw1", ma, ma, mXp, mXp, p,

@@ -18,6 +18,7 @@ OK, ERR_ARG, ERR_SHAPE, ERR_ALIGN, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_UNS
 F32, BF16 = 0, 1
 MODE_AUTO, MODE_TCR, MODE_ECR = 0, 1, 2
 GEMM_AUTO, GEMM_SIMT, GEMM_TCGEN05, GEMM_TCGEN05_2CTA, GEMM_TCGEN05_2CTA_WIDE = 0, 1, 2, 3, 4
+FUSE_AUTO, FUSE_OFF, FUSE_ON = 0, 1, 2
 
 EXPORTS = [
     "etr_status_string", "etr_validate", "etr_c_stride", "etr_workspace_bytes", "etr_buffers_bytes",
@@ -34,7 +35,7 @@ class Config(C.Structure):
                 ("k", C.c_int32), ("h", C.c_int32), ("capacity", C.c_int32), ("c_floor", C.c_int32),
                 ("adaptive", C.c_int32), ("delta_max_override", C.c_float),
                 ("step", C.c_int64), ("switch_step", C.c_int64), ("mode", C.c_int32),
-                ("dtype", C.c_int32), ("gemm_impl", C.c_int32), ("reserved", C.c_int32)]
+                ("dtype", C.c_int32), ("gemm_impl", C.c_int32), ("fuse_dispatch", C.c_int32)]
 
 
 class Stats(C.Structure):
@@ -121,11 +122,12 @@ def _stream():
 
 
 def make_config(*, T, d, D, E, k, h, capacity, dtype, mode=MODE_AUTO, step=0, switch_step=0,
-                adaptive=False, c_floor=1, delta_max_override=-1.0, gemm_impl=GEMM_AUTO) -> Config:
+                adaptive=False, c_floor=1, delta_max_override=-1.0, gemm_impl=GEMM_AUTO,
+                fuse_dispatch=0) -> Config:
     return Config(T=T, d=d, D=D, E=E, k=k, h=h, capacity=capacity, c_floor=c_floor,
                   adaptive=int(bool(adaptive)), delta_max_override=float(delta_max_override),
                   step=int(step), switch_step=int(switch_step), mode=int(mode), dtype=int(dtype),
-                  gemm_impl=int(gemm_impl), reserved=0)
+                  gemm_impl=int(gemm_impl), fuse_dispatch=int(fuse_dispatch))
 
 
 def torch_dtype(cfg: Config):

@@ -304,6 +304,30 @@ def test_layer_is_deterministic_and_host_step_matches():
         assert torch.equal(a[k].cpu(), c[k].cpu()), k
 
 
+@pytest.mark.parametrize("impl", [etr.GEMM_AUTO, etr.GEMM_TCGEN05_2CTA, etr.GEMM_TCGEN05_2CTA_WIDE])
+@pytest.mark.parametrize("name", ["small_s", "mid_s", "sweep_s_tcr", "sweep_s_ecr"])
+def test_fused_dispatch_gives_the_same_bits(name, impl):
+    """With the token rearrangement fused into the operand fetch (TMA row gathers from X) the GEMMs
+    see the same operands in the same order: every output must equal the unfused path bit for bit,
+    and Xp must not have been touched."""
+    w, inp, o, fw, bw = case(name)
+    ov = override_of(name) if w.adaptive else -1.0
+    _, ref = run_layer(w, inp, hz.make_cfg(w, gemm_impl=impl, delta_max_override=ov, fuse_dispatch=etr.FUSE_OFF))
+    cfg = hz.make_cfg(w, gemm_impl=impl, delta_max_override=ov, fuse_dispatch=etr.FUSE_ON)
+    dev = hz.upload(w, inp)
+    buf = etr.LayerBuffers(cfg)
+    buf.Xp.fill_(float("nan"))
+    out = {k: torch.empty_like(v) for k, v in ref.items()}
+    etr.layer_forward(cfg, dev.X, dev.R, dev.W1g, dev.W1u, dev.W2, buf, out["Y"])
+    etr.layer_backward(cfg, dev.X, dev.R, dev.W1g, dev.W1u, dev.W2, dev.dY, buf, out["dX"], out["dR"],
+                       out["dW1g"], out["dW1u"], out["dW2"])
+    torch.cuda.synchronize()
+    assert buf.read_stats().error_word == 0
+    assert bool(torch.isnan(buf.Xp).all()), "Xp was written"
+    for k in ref:
+        assert torch.equal(out[k], ref[k]), k
+
+
 def test_pipelined_host_steps_match_the_layer_calls():
     """Six steps through etr_layer_step_host_begin on two slots, alternating between two different
     batches, with no wait between them: every step must deliver exactly what the layer calls give
