@@ -207,6 +207,28 @@ class Oracle:
         self._f("select_bwd")(route.T, route.E, route.C_stride, _p(route.slot_token), _p(dgate), _p(dd))
         return dd
 
+    def softmax_gate(self, delta, route):
+        """Gates of the softmax variant: softmax of each token's affinities over all experts."""
+        delta = self.arr(delta)
+        gate = np.empty(route.E * route.C_stride, self.np)
+        self._f("softmax_gate")(route.T, route.E, route.C_stride, _p(delta), _p(route.slot_token), _p(gate))
+        return gate
+
+    def softmax_gate_bwd(self, delta, dgate, route):
+        delta, dgate = self.arr(delta), self.arr(dgate)
+        dd = np.empty((route.T, route.E), self.np)
+        self._f("softmax_gate_bwd")(route.T, route.E, route.C_stride, _p(delta), _p(route.slot_token),
+                                    _p(dgate), _p(dd))
+        return dd
+
+    def load_stats(self, route, gate=None):
+        """(load, gate_mean): tokens per expert / T, and summed gates per expert / T."""
+        gate = self.arr(route.gate if gate is None else gate)
+        load, gm = np.empty(route.E, self.np), np.empty(route.E, self.np)
+        self._f("load_stats")(route.T, route.E, route.C_stride, _p(route.counts), _p(route.slot_token),
+                              _p(gate), _p(load), _p(gm))
+        return load, gm
+
     def affinity_bwd(self, X, R, D, delta, xnorm, rnorm, ddelta, dX):
         """Accumulates the router path's gradient into dX (in place); returns (dX, dR)."""
         X, R, delta, xnorm, rnorm, ddelta = map(self.arr, (X, R, delta, xnorm, rnorm, ddelta))
@@ -220,7 +242,8 @@ class Oracle:
 
     # -- the whole layer: the stages above in order ---------------------------------------
     def forward(self, X, R, W1g, W1u, W2, *, D, k, capacity, C_stride=None, mode=None, step=0,
-                switch_step=0, adaptive=False, c_floor=1, delta_max_override=-1.0, route=None):
+                switch_step=0, adaptive=False, c_floor=1, delta_max_override=-1.0, route=None,
+                softmax_gate=False):
         d = X.shape[1]
         E = R.shape[0]
         if C_stride is None:
@@ -238,11 +261,13 @@ class Oracle:
             v = route.slot_token >= 0
             rows = np.nonzero(v)[0]
             gate[rows] = delta[route.slot_token[rows], rows // route.C_stride]
+        if softmax_gate:
+            gate = self.softmax_gate(delta, route)
         Xp = self.dispatch(X, route)
         G, U, H, O = self.expert_ffn(Xp, route, W1g, W1u, W2)
         Y = self.combine(O, route, gate)
         return SimpleNamespace(delta=delta, xnorm=xnorm, rnorm=rnorm, delta_max=dmax, route=route,
-                               gate=gate, Xp=Xp, G=G, U=U, H=H, O=O, Y=Y, D=D)
+                               gate=gate, Xp=Xp, G=G, U=U, H=H, O=O, Y=Y, D=D, softmax_gate=softmax_gate)
 
     def backward(self, fwd, X, R, W1g, W1u, W2, dY):
         rt = fwd.route
@@ -250,7 +275,10 @@ class Oracle:
         dG, dU, dXp, dW1g, dW1u, dW2 = self.expert_ffn_bwd(dO, fwd.Xp, fwd.G, fwd.U, fwd.H, rt,
                                                             W1g, W1u, W2)
         dX_ffn = self.dispatch_bwd(dXp, rt)
-        ddelta = self.select_bwd(dgate, rt)
+        if getattr(fwd, "softmax_gate", False):
+            ddelta = self.softmax_gate_bwd(fwd.delta, dgate, rt)
+        else:
+            ddelta = self.select_bwd(dgate, rt)
         dX = dX_ffn.copy()
         dX, dR = self.affinity_bwd(X, R, fwd.D, fwd.delta, fwd.xnorm, fwd.rnorm, ddelta, dX)
         return SimpleNamespace(dO=dO, dgate=dgate, dG=dG, dU=dU, dXp=dXp, dW1g=dW1g, dW1u=dW1u,

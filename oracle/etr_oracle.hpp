@@ -25,7 +25,9 @@
 // SwiGLU for E = 1, central finite differences for every gradient, permutation
 // equivariance.  Parity unpinned: the TCR->ECR switch rule (a caller-supplied step
 // threshold), the source of delta_max (batch maximum), the clamp of C_min into
-// [c_floor, capacity], and the raw-affinity gate; the paper under-specifies these.
+// [c_floor, capacity], and the raw-affinity gate; the paper under-specifies these.  The
+// softmax-gate variant and the load statistics are pinned by library softmax / autograd, finite
+// differences and closed forms.
 #pragma once
 #include <algorithm>
 #include <cmath>
@@ -363,6 +365,73 @@ void select_bwd(int T, int E, int C_stride, const int32_t* slot_token, const S* 
       const size_t r = (size_t)i * C_stride + p;
       if (slot_token[r] >= 0) ddelta[(size_t)slot_token[r] * E + i] = dgate[r];
     }
+}
+
+// ---- softmax gate (variant) ---------------------------------------------------------------------
+// The general MoE form names G(x) = Softmax(.) as its example of a gating weight.  In this variant
+// the gate of a selected pair (t, i) is the softmax of token t's affinities over ALL n experts,
+//   p_ti = exp(delta_ti) / sum_j exp(delta_tj),
+// instead of the raw affinity delta_ti.  Rows without a token keep gate 0.
+template <class S>
+void softmax_gate(int T, int E, int C_stride, const S* delta, const int32_t* slot_token, S* gate) {
+  (void)T;
+  for (int i = 0; i < E; ++i)
+    for (int p = 0; p < C_stride; ++p) {
+      const size_t r = (size_t)i * C_stride + p;
+      const int t = slot_token[r];
+      if (t < 0) { gate[r] = (S)0; continue; }
+      const S* dt = delta + (size_t)t * E;
+      double mx = (double)dt[0];
+      for (int j = 1; j < E; ++j) mx = std::max(mx, (double)dt[j]);
+      double den = 0.0;
+      for (int j = 0; j < E; ++j) den += std::exp((double)dt[j] - mx);
+      gate[r] = (S)(std::exp((double)dt[i] - mx) / den);
+    }
+}
+
+// Its backward.  With g_ti the incoming gradient of the gate of a selected pair (0 for pairs not
+// selected) and s_t = sum_i g_ti p_ti over the selected experts of token t,
+//   d delta_tj = p_tj (g_tj - s_t)        for every expert j (the softmax couples them all).
+template <class S>
+void softmax_gate_bwd(int T, int E, int C_stride, const S* delta, const int32_t* slot_token,
+                      const S* dgate, S* ddelta) {
+  std::vector<double> g((size_t)T * E, 0.0);
+  for (int i = 0; i < E; ++i)
+    for (int p = 0; p < C_stride; ++p) {
+      const size_t r = (size_t)i * C_stride + p;
+      if (slot_token[r] >= 0) g[(size_t)slot_token[r] * E + i] = (double)dgate[r];
+    }
+  for (int t = 0; t < T; ++t) {
+    const S* dt = delta + (size_t)t * E;
+    double mx = (double)dt[0];
+    for (int j = 1; j < E; ++j) mx = std::max(mx, (double)dt[j]);
+    double den = 0.0;
+    for (int j = 0; j < E; ++j) den += std::exp((double)dt[j] - mx);
+    double st = 0.0;
+    for (int j = 0; j < E; ++j) st += g[(size_t)t * E + j] * (std::exp((double)dt[j] - mx) / den);
+    for (int j = 0; j < E; ++j) {
+      const double pj = std::exp((double)dt[j] - mx) / den;
+      ddelta[(size_t)t * E + j] = (S)(pj * (g[(size_t)t * E + j] - st));
+    }
+  }
+}
+
+// ---- load statistics (inputs of the auxiliary and locality losses) -------------------------------
+// load[i] = counts[i] / T, the share of the batch's tokens expert i processes;
+// gate_mean[i] = (1/T) sum of the gates of expert i's rows (its mean gate over all T tokens, a
+// token it does not process counting as 0).
+template <class S>
+void load_stats(int T, int E, int C_stride, const int32_t* counts, const int32_t* slot_token,
+                const S* gate, S* load, S* gate_mean) {
+  for (int i = 0; i < E; ++i) {
+    double acc = 0.0;
+    for (int p = 0; p < C_stride; ++p) {
+      const size_t r = (size_t)i * C_stride + p;
+      if (slot_token[r] >= 0) acc += (double)gate[r];
+    }
+    load[i] = (S)((double)counts[i] / (double)T);
+    gate_mean[i] = (S)(acc / (double)T);
+  }
 }
 
 // ---- backward of the affinity ----------------------------------------------------------------

@@ -74,6 +74,20 @@ using namespace etr_oracle;
                                               S* ddelta) {                                           \
     select_bwd<S>(T, E, C_stride, slot_token, dgate, ddelta);                                        \
   }                                                                                                  \
+  extern "C" void etr_oracle_softmax_gate_##SUF(int T, int E, int C_stride, const S* delta,          \
+                                                const int32_t* slot_token, S* gate) {                \
+    softmax_gate<S>(T, E, C_stride, delta, slot_token, gate);                                        \
+  }                                                                                                  \
+  extern "C" void etr_oracle_softmax_gate_bwd_##SUF(int T, int E, int C_stride, const S* delta,      \
+                                                    const int32_t* slot_token, const S* dgate,       \
+                                                    S* ddelta) {                                     \
+    softmax_gate_bwd<S>(T, E, C_stride, delta, slot_token, dgate, ddelta);                           \
+  }                                                                                                  \
+  extern "C" void etr_oracle_load_stats_##SUF(int T, int E, int C_stride, const int32_t* counts,     \
+                                              const int32_t* slot_token, const S* gate, S* load,     \
+                                              S* gate_mean) {                                        \
+    load_stats<S>(T, E, C_stride, counts, slot_token, gate, load, gate_mean);                        \
+  }                                                                                                  \
   extern "C" void etr_oracle_affinity_bwd_##SUF(int T, int d, int D, int E, const S* X, const S* R,  \
                                                 const S* delta, const S* xnorm, const S* rnorm,      \
                                                 const S* ddelta, S* dX, S* dR) {                     \

@@ -150,6 +150,79 @@ def test_gradients_by_finite_differences(o64, mode, cap):
             assert abs(fd - g.reshape(-1)[idx]) <= 2e-7 * scale + 1e-9, (name, idx, fd, g.reshape(-1)[idx])
 
 
+def test_softmax_gate_is_library_softmax(o64):
+    p = problem(9, T=20)
+    fw = o64.forward(p["X"], p["R"], p["W1g"], p["W1u"], p["W2"], D=2, k=2, capacity=9, mode=ob.MODE_TCR,
+                     softmax_gate=True)
+    rt = fw.route
+    want = torch.softmax(torch_affinity(torch.from_numpy(p["X"]), torch.from_numpy(p["R"]), 2), dim=1).numpy()
+    rows = np.nonzero(rt.slot_token >= 0)[0]
+    assert len(rows) > 0 and rt.dropped > 0
+    assert np.allclose(fw.gate[rows], want[rt.slot_token[rows], rows // rt.C_stride], rtol=1e-13, atol=0)
+    assert np.all(fw.gate[rt.slot_token < 0] == 0)
+
+
+def test_softmax_gate_dense_moe_fwd_bwd(o64):
+    """Expert choice with C = T and the softmax gate is the general MoE form with
+    G(x) = Softmax(affinities): forward and all five gradients against torch.autograd."""
+    p = problem(10)
+    fw = o64.forward(p["X"], p["R"], p["W1g"], p["W1u"], p["W2"], D=2, k=2, capacity=12,
+                     mode=ob.MODE_ECR, softmax_gate=True)
+    bw = o64.backward(fw, p["X"], p["R"], p["W1g"], p["W1u"], p["W2"], p["dY"])
+    t = {k: torch.from_numpy(v).requires_grad_(k != "dY") for k, v in p.items()}
+    gate = torch.softmax(torch_affinity(t["X"], t["R"], 2), dim=1)
+    Y = 0
+    for i in range(3):
+        Y = Y + gate[:, i:i + 1] * torch_swiglu(t["X"], t["W1g"][i], t["W1u"][i], t["W2"][i])
+    (Y * t["dY"]).sum().backward()
+    assert np.allclose(fw.Y, Y.detach().numpy(), rtol=1e-12, atol=1e-13)
+    for name, got in [("X", bw.dX), ("R", bw.dR), ("W1g", bw.dW1g), ("W1u", bw.dW1u), ("W2", bw.dW2)]:
+        assert np.allclose(got, t[name].grad.numpy(), rtol=1e-10, atol=1e-12), name
+
+
+def test_softmax_gate_gradients_by_finite_differences(o64):
+    """Sparse selection (capacity active): the softmax still couples all experts of a token."""
+    p = problem(11)
+    kw = dict(D=2, k=2, capacity=5, mode=ob.MODE_TCR, softmax_gate=True)
+    fw = o64.forward(p["X"], p["R"], p["W1g"], p["W1u"], p["W2"], **kw)
+    assert fw.route.dropped > 0
+    bw = o64.backward(fw, p["X"], p["R"], p["W1g"], p["W1u"], p["W2"], p["dY"])
+
+    def loss(q):
+        y = o64.forward(q["X"], q["R"], q["W1g"], q["W1u"], q["W2"], route=fw.route, **kw).Y
+        return float((y * p["dY"]).sum())
+
+    eps = 1e-6
+    for name, g in dict(X=bw.dX, R=bw.dR).items():
+        scale = np.abs(g).max()
+        for idx in range(p[name].size):
+            q = {k: v.copy() for k, v in p.items()}
+            q[name].reshape(-1)[idx] += eps
+            up = loss(q)
+            q[name].reshape(-1)[idx] -= 2 * eps
+            fd = (up - loss(q)) / (2 * eps)
+            assert abs(fd - g.reshape(-1)[idx]) <= 2e-7 * scale + 1e-9, (name, idx, fd, g.reshape(-1)[idx])
+
+
+def test_load_statistics(o64):
+    p = problem(12, T=24)
+    # expert choice with C = T: every expert processes every token; its mean gate is the column mean
+    fw = o64.forward(p["X"], p["R"], p["W1g"], p["W1u"], p["W2"], D=2, k=2, capacity=24, mode=ob.MODE_ECR)
+    load, gm = o64.load_stats(fw.route)
+    assert np.array_equal(load, np.ones(3))
+    assert np.allclose(gm, fw.delta.mean(axis=0), rtol=1e-13, atol=1e-15)
+    # token choice under an active capacity: loads add up to the rows kept, and the summed gates are
+    # what combining rows of ones gives
+    fw = o64.forward(p["X"], p["R"], p["W1g"], p["W1u"], p["W2"], D=2, k=2, capacity=9, mode=ob.MODE_TCR)
+    rt = fw.route
+    load, gm = o64.load_stats(rt)
+    assert rt.dropped > 0 and np.allclose(load * 24, rt.counts) and abs(load.sum() * 24 - rt.counts.sum()) < 1e-12
+    ones = np.ones((3 * rt.C_stride, 1))
+    assert abs(gm.sum() * 24 - o64.combine(ones, rt).sum()) < 1e-12
+    by_hand = [sum(fw.delta[rt.slot_token[i * rt.C_stride + q], i] for q in range(rt.counts[i])) / 24 for i in range(3)]
+    assert np.allclose(gm, by_hand, rtol=1e-13)
+
+
 def test_router_gradient_orthogonality(o64):
     """The cosine ignores the scale of x_t and of R_i, so the router path's gradient
     satisfies <dX_router[t], x_t> = 0 and <dR_i, R_i> = 0."""
