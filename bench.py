@@ -91,6 +91,10 @@ def algorithmic_work(w, rows, kernel, unrouted=0):
         "affinity_bwd_dx_fused_kernel": (T_routed * d * b + rows * d * b + T * d * b, "bytes"),
         "affinity_bwd_dr_partial_kernel": (rows * m * 4, "bytes"),
         "affinity_bwd_dr_final_kernel": (E * m * 8, "bytes"),
+        "affinity_bwd_dr_dense_partial_kernel": (T * m * 4 + T * E * 8, "bytes"),
+        "gate_softmax_kernel": (T * E * 4 + rows * 12 + T * 4, "bytes"),
+        "gate_softmax_bwd_kernel": (2 * T * E * 4 + rows * 12, "bytes"),
+        "load_stats_kernel": (rows * 4, "bytes"),
         "gemm_simt_kernel": (18 * rows * d * h, "flops"),
         # tcgen05 grouped GEMMs: selected rows only (not the rows padding a 128-row tile)
         "tc_gemm_swiglu": (4 * rows * d * h, "flops"),
@@ -213,6 +217,8 @@ def main():
     ap.add_argument("--gemm", default="auto", choices=["auto", "simt", "tcgen05", "tcgen05_2cta", "tcgen05_2cta_wide"])
     ap.add_argument("--fuse", default="auto", choices=["auto", "off", "on"],
                     help="token rearrangement fused into the GEMM operand fetch (TMA row gathers)")
+    ap.add_argument("--gate", default="affinity", choices=["affinity", "softmax"],
+                    help="gate of a selected pair: raw affinity (default) or softmax over the experts")
     ap.add_argument("--cpu-tokens", type=int, default=128, help="tokens in the CPU-oracle sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--set", default="", help="override workload fields, e.g. T=32768,h=512 (profiling cases)")
@@ -275,7 +281,8 @@ def main():
                           dtype=etr.BF16 if w.dtype == "bf16" else etr.F32,
                           mode=etr.MODE_TCR if mode_name(w) == "tcr" else etr.MODE_ECR,
                           step=w.step, switch_step=w.switch_step, adaptive=w.adaptive, gemm_impl=impl,
-                          fuse_dispatch={"auto": etr.FUSE_AUTO, "off": etr.FUSE_OFF, "on": etr.FUSE_ON}[args.fuse])
+                          fuse_dispatch={"auto": etr.FUSE_AUTO, "off": etr.FUSE_OFF, "on": etr.FUSE_ON}[args.fuse],
+                          gate_mode=etr.GATE_SOFTMAX if args.gate == "softmax" else etr.GATE_AFFINITY)
     buf = etr.LayerBuffers(cfg, host_staging=True, device=dev)
     Y, dX = torch.empty_like(X), torch.empty_like(X)
     dR = torch.empty_like(R)

@@ -69,6 +69,12 @@ typedef enum { ETR_GEMM_AUTO = 0, ETR_GEMM_SIMT = 1, ETR_GEMM_TCGEN05 = 2, ETR_G
  * read.  The stage calls are unaffected.  ETR_FUSE_AUTO lets the library choose. */
 typedef enum { ETR_FUSE_AUTO = 0, ETR_FUSE_OFF = 1, ETR_FUSE_ON = 2 } etr_fuse;
 
+/* Gate of a selected pair (t, i).  AFFINITY (default): the raw affinity delta_ti ("the affinity
+ * matrix is employed as the gating weight").  SOFTMAX: p_ti = exp(delta_ti) / sum_j exp(delta_tj)
+ * over all E experts of the token, the example gate of the general MoE equation; its backward
+ * gives every expert of a routed token a gradient (a dense d delta), see etr_gate_softmax_bwd. */
+typedef enum { ETR_GATE_AFFINITY = 0, ETR_GATE_SOFTMAX = 1 } etr_gate;
+
 /* Immutable description of one layer call (host struct, passed by pointer). */
 typedef struct etr_config {
   int32_t T, d, D, E, k, h;
@@ -81,6 +87,8 @@ typedef struct etr_config {
   int32_t dtype;              /* etr_dtype of activations and expert weights */
   int32_t gemm_impl;          /* etr_gemm_impl; AUTO = CTA-pair tcgen05 for bf16, SIMT for fp32 */
   int32_t fuse_dispatch;      /* etr_fuse: token rearrangement fused into the GEMM operand fetch */
+  int32_t gate_mode;          /* etr_gate: what weighs an expert's output in the combine */
+  int32_t reserved;
 } etr_config;
 
 /* Per-call scalars produced and consumed on the device (device struct, 64 bytes). */
@@ -121,6 +129,8 @@ typedef struct etr_buffers {
   size_t ws_bytes;
   /* staging used only by etr_layer_step_host */
   void* X_dev; void* dY_dev; void* Y_dev; void* dX_dev;
+  /* softmax gate only (NULL otherwise): per-token log-sum-exp [T] and the dense d delta [T,E] */
+  float* lse; float* ddelta;
 } etr_buffers;
 
 const char* etr_status_string(etr_status s);
@@ -239,9 +249,41 @@ etr_status etr_affinity_bwd(const etr_config* cfg, const void* X, const float* R
                             const float* rnorm, const etr_route* route, const float* dgate,
                             void* dX, float* dR, void* ws, void* stream);
 
+/* ---- softmax-gate variant and load statistics --------------------------------------------- */
+
+/* Softmax gate (the Softmax example of the gating weight in the general MoE equation): replaces
+ * route->gate[r] of every row in use by p_ti = exp(delta_ti - lse[t]) with
+ * lse[t] = log sum_j exp(delta_tj) over all E experts, and writes lse [T].  Call after etr_select;
+ * rows not in use keep gate 0. */
+etr_status etr_gate_softmax(const etr_config* cfg, const float* delta, const etr_route* route,
+                            float* lse, void* stream);
+
+/* Its backward (calculus; the paper has none): with g_tj = dgate of the row of pair (t, j) if the
+ * pair is selected and 0 otherwise, and s_t = sum_j g_tj p_tj,
+ *   ddelta[t][j] = p_tj (g_tj - s_t)   for every expert j;  rows of tokens without a row are 0.
+ * ddelta is [T,E] fp32; route->gate must still hold the softmax gates. */
+etr_status etr_gate_softmax_bwd(const etr_config* cfg, const float* delta, const float* lse,
+                                const etr_route* route, const float* dgate, float* ddelta,
+                                void* stream);
+
+/* etr_affinity_bwd for a dense d delta [T,E] (what etr_gate_softmax_bwd produces): same outputs,
+ * dX accumulated into, dR overwritten; `route` is read only to skip tokens without rows.
+ * ws: etr_workspace_bytes of a config whose gate_mode is ETR_GATE_SOFTMAX. */
+etr_status etr_affinity_bwd_dense(const etr_config* cfg, const void* X, const float* R,
+                                  const float* delta, const float* Z, const float* xnorm,
+                                  const float* rnorm, const etr_route* route, const float* ddelta,
+                                  void* dX, float* dR, void* ws, void* stream);
+
+/* Load statistics, the inputs of the auxiliary and locality losses ("Locality Loss"), which are
+ * not part of the layer: load[i] = counts[i] / T, the share of the batch's tokens expert i
+ * processes, and gate_mean[i] = (sum of the gates of expert i's rows) / T.  Both [E] fp32. */
+etr_status etr_load_stats(const etr_config* cfg, const etr_route* route, float* load,
+                          float* gate_mean, void* stream);
+
 /* ---- whole layer ---------------------------------------------------------------------- */
 
-/* Zeroes stats, then affinity, select, dispatch, expert_ffn, combine, in that order. */
+/* Zeroes stats, then affinity, select, (gate_softmax,) dispatch, expert_ffn, combine, in that
+ * order. */
 etr_status etr_layer_forward(const etr_config* cfg, const void* X, const float* R,
                              const void* W1g, const void* W1u, const void* W2,
                              const etr_buffers* buf, void* Y, void* stream);

@@ -517,8 +517,8 @@ affinity_bwd_dx_kernel(const T* __restrict__ X, const float* __restrict__ R,
                        const float* __restrict__ delta, const float* __restrict__ xnorm,
                        const float* __restrict__ rnorm, const int32_t* __restrict__ tok_ptr,
                        const int32_t* __restrict__ tok_row, const float* __restrict__ dgate,
-                       const T* __restrict__ dXp, T* __restrict__ dX, int Ttok, int d, int D, int E,
-                       int m, int C_stride) {
+                       const float* __restrict__ ddelta, const T* __restrict__ dXp, T* __restrict__ dX,
+                       int Ttok, int d, int D, int E, int m, int C_stride) {
   extern __shared__ __align__(16) float smem[];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   float* cz = smem + (size_t)warp * m;
@@ -536,7 +536,17 @@ affinity_bwd_dx_kernel(const T* __restrict__ X, const float* __restrict__ R,
   for (int j = lane; j < m; j += 32) cz[j] = 0.f;
   float beta = 0.f;
   const float sqD = sqrtf((float)D);
-  if (a != 0.f) {
+  if (a != 0.f && ddelta != nullptr) {
+    // dense d delta (softmax gate): every expert contributes, in ascending expert order
+    for (int i = 0; i < E; ++i) {
+      const float b = rnorm[i], dg = ddelta[(size_t)t * E + i];
+      if (b == 0.f || dg == 0.f) continue;
+      const float w = dg * sqD / (a * b) / (float)D;
+      beta += dg * delta[(size_t)t * E + i];
+      for (int j = lane; j < m; j += 32) cz[j] = fmaf(w, R[(size_t)i * m + j], cz[j]);
+    }
+    beta /= (a * a);
+  } else if (a != 0.f) {
     for (int q = beg; q < end; ++q) {
       const int r = tok_row[q], i = r / C_stride;
       const float b = rnorm[i], dg = dgate[r];
@@ -636,6 +646,66 @@ affinity_bwd_dr_partial_kernel(const float* __restrict__ Z, const float* __restr
   if (tid == 0) out[m] = sdd;
 }
 
+// The same partial sums for a dense d delta [T, E] (softmax gate): chunks of DR_DENSE_TOKENS
+// consecutive tokens, every expert.  A block takes one chunk and 32 experts at a time: thread j keeps
+// column j of the 32 partial rows, so each Z value is loaded once per 32 experts; tokens in ascending
+// order (sub-chunks of 128 staged in shared memory).
+constexpr int DR_DENSE_TOKENS = 256;
+__global__ void __launch_bounds__(256)
+affinity_bwd_dr_dense_partial_kernel(const float* __restrict__ Z, const float* __restrict__ delta,
+                                     const float* __restrict__ xnorm, const float* __restrict__ rnorm,
+                                     const float* __restrict__ ddelta, float* __restrict__ part,
+                                     int Ttok, int E, int m, int nch, float sqD) {
+  __shared__ __align__(16) float s_w[DR_CHUNK][32];
+  __shared__ float s_dd[DR_CHUNK][32];
+  const int ch = blockIdx.x, tid = threadIdx.x;
+  const int t_beg = ch * DR_DENSE_TOKENS, t_end = min(Ttok, t_beg + DR_DENSE_TOKENS);
+  for (int e0 = 0; e0 < E; e0 += 32) {
+    for (int j0 = 0; j0 < m; j0 += 256) {
+      const int j = j0 + tid;
+      float acc[32];
+#pragma unroll
+      for (int ii = 0; ii < 32; ++ii) acc[ii] = 0.f;
+      float sdd = 0.f;
+      for (int t0 = t_beg; t0 < t_end; t0 += DR_CHUNK) {
+        const int np = min(DR_CHUNK, t_end - t0);
+        __syncthreads();
+        for (int idx = tid; idx < DR_CHUNK * 32; idx += 256) {
+          const int p = idx >> 5, i = e0 + (idx & 31);
+          float w = 0.f, dd = 0.f;
+          if (p < np && i < E) {
+            const int t = t0 + p;
+            const float a = xnorm[t], b = rnorm[i], dg = ddelta[(size_t)t * E + i];
+            if (a != 0.f && b != 0.f) { w = dg * sqD / (a * b); dd = dg * delta[(size_t)t * E + i]; }
+          }
+          s_w[p][idx & 31] = w;
+          s_dd[p][idx & 31] = dd;
+        }
+        __syncthreads();
+        if (j < m) {
+          for (int p = 0; p < np; ++p) {
+            const float zv = Z[(size_t)(t0 + p) * m + j];
+#pragma unroll
+            for (int q4 = 0; q4 < 8; ++q4) {
+              const float4 w = *reinterpret_cast<const float4*>(&s_w[p][4 * q4]);
+              acc[4 * q4] = fmaf(w.x, zv, acc[4 * q4]);         acc[4 * q4 + 1] = fmaf(w.y, zv, acc[4 * q4 + 1]);
+              acc[4 * q4 + 2] = fmaf(w.z, zv, acc[4 * q4 + 2]); acc[4 * q4 + 3] = fmaf(w.w, zv, acc[4 * q4 + 3]);
+            }
+          }
+        }
+        if (j0 == 0 && tid < 32)
+          for (int p = 0; p < np; ++p) sdd += s_dd[p][tid];
+      }
+      if (j < m) {
+#pragma unroll
+        for (int ii = 0; ii < 32; ++ii)
+          if (e0 + ii < E) part[((size_t)(e0 + ii) * nch + ch) * (m + 1) + j] = acc[ii];
+      }
+      if (j0 == 0 && tid < 32 && e0 + tid < E) part[((size_t)(e0 + tid) * nch + ch) * (m + 1) + m] = sdd;
+    }
+  }
+}
+
 // dR[i][j] = sum_ch part[i][ch][j] - (sum_ch part[i][ch][m]) R[i][j] / b_i^2, chunks in order.
 __global__ void __launch_bounds__(256)
 affinity_bwd_dr_final_kernel(const float* __restrict__ part, const float* __restrict__ R,
@@ -644,9 +714,11 @@ affinity_bwd_dr_final_kernel(const float* __restrict__ part, const float* __rest
   const float b = rnorm[i];
   const float* base = part + (size_t)i * nch * (m + 1);
   float sdd = 0.f;
+#pragma unroll 8
   for (int ch = 0; ch < nch; ++ch) sdd += base[(size_t)ch * (m + 1) + m];
   for (int j = threadIdx.x; j < m; j += 256) {
     float acc = 0.f;
+#pragma unroll 8
     for (int ch = 0; ch < nch; ++ch) acc += base[(size_t)ch * (m + 1) + j];
     dR[(size_t)i * m + j] = b == 0.f ? 0.f : acc - sdd * R[(size_t)i * m + j] / (b * b);
   }
@@ -794,53 +866,63 @@ etr_status affinity_forward(const etr_config* c, const void* X, const float* R, 
 }
 
 size_t affinity_bwd_workspace_bytes(const etr_config* c) {
-  const int m = c->d / c->D, nch = c_stride_of(c) / DR_CHUNK;
+  const int m = c->d / c->D;
+  const int nch = c->gate_mode == ETR_GATE_SOFTMAX ? std::max(c_stride_of(c) / DR_CHUNK, ceil_div(c->T, DR_DENSE_TOKENS))
+                                                   : c_stride_of(c) / DR_CHUNK;
   return (size_t)c->E * nch * (m + 1) * sizeof(float);
 }
 
 template <class T>
 static etr_status launch_bwd_dx(const etr_config* c, const void* X, const float* R, const float* delta,
                                 const float* xnorm, const float* rnorm, const etr_route* rt,
-                                const float* dgate, const void* dXp_fused, void* dX, size_t smem,
-                                cudaStream_t st) {
+                                const float* dgate, const float* ddelta, const void* dXp_fused, void* dX,
+                                size_t smem, cudaStream_t st) {
   const int m = c->d / c->D, Cs = c_stride_of(c), grid = ceil_div(c->T, 8);
   if (dXp_fused) {
     auto k = affinity_bwd_dx_kernel<T, true>;
     if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
       return ETR_ERR_CUDA;
     ETR_TIME_BEGIN("affinity_bwd_dx_fused_kernel");
-    k<<<grid, 256, smem, st>>>((const T*)X, R, delta, xnorm, rnorm, rt->tok_ptr, rt->tok_row, dgate,
+    k<<<grid, 256, smem, st>>>((const T*)X, R, delta, xnorm, rnorm, rt->tok_ptr, rt->tok_row, dgate, ddelta,
                                (const T*)dXp_fused, (T*)dX, c->T, c->d, c->D, c->E, m, Cs);
   } else {
     auto k = affinity_bwd_dx_kernel<T, false>;
     if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
       return ETR_ERR_CUDA;
     ETR_TIME_BEGIN("affinity_bwd_dx_kernel");
-    k<<<grid, 256, smem, st>>>((const T*)X, R, delta, xnorm, rnorm, rt->tok_ptr, rt->tok_row, dgate,
+    k<<<grid, 256, smem, st>>>((const T*)X, R, delta, xnorm, rnorm, rt->tok_ptr, rt->tok_row, dgate, ddelta,
                                (const T*)nullptr, (T*)dX, c->T, c->d, c->D, c->E, m, Cs);
   }
   ETR_LAUNCH_CHECK();
   return ETR_OK;
 }
 
-// dXp_fused != nullptr: dX is produced here in one pass (dispatch backward + router gradient)
+// dXp_fused != nullptr: dX is produced here in one pass (dispatch backward + router gradient).
+// ddelta != nullptr: the gradient of the affinities is that dense [T, E] matrix (softmax gate)
+// instead of dgate on the selected pairs.
 etr_status affinity_backward(const etr_config* c, const void* X, const float* R, const float* delta,
                              const float* Z, const float* xnorm, const float* rnorm,
-                             const etr_route* rt, const float* dgate, const void* dXp_fused, void* dX,
-                             float* dR, void* ws, cudaStream_t st) {
-  const int m = c->d / c->D, Cs = c_stride_of(c), nch = Cs / DR_CHUNK;
+                             const etr_route* rt, const float* dgate, const float* ddelta,
+                             const void* dXp_fused, void* dX, float* dR, void* ws, cudaStream_t st) {
+  const int m = c->d / c->D, Cs = c_stride_of(c);
+  const int nch = ddelta ? ceil_div(c->T, DR_DENSE_TOKENS) : Cs / DR_CHUNK;
   if (m > 256 * DR_MAXJ) return ETR_ERR_UNSUPPORTED;
   const size_t smem = (size_t)8 * m * sizeof(float);
   if (smem > 200 * 1024) return ETR_ERR_UNSUPPORTED;
-  const int grid = ceil_div(c->T, 8);
   ETR_TRY((c->dtype == ETR_BF16
-               ? launch_bwd_dx<__nv_bfloat16>(c, X, R, delta, xnorm, rnorm, rt, dgate, dXp_fused, dX, smem, st)
-               : launch_bwd_dx<float>(c, X, R, delta, xnorm, rnorm, rt, dgate, dXp_fused, dX, smem, st)));
+               ? launch_bwd_dx<__nv_bfloat16>(c, X, R, delta, xnorm, rnorm, rt, dgate, ddelta, dXp_fused, dX, smem, st)
+               : launch_bwd_dx<float>(c, X, R, delta, xnorm, rnorm, rt, dgate, ddelta, dXp_fused, dX, smem, st)));
   float* part = (float*)ws;
-  ETR_TIME_BEGIN("affinity_bwd_dr_partial_kernel");
-  affinity_bwd_dr_partial_kernel<<<dim3(c->E, nch), 256, 0, st>>>(
-      Z, delta, xnorm, rnorm, rt->counts, rt->slot_token, dgate, part, c->E, m, Cs, nch,
-      sqrtf((float)c->D));
+  if (ddelta) {
+    ETR_TIME_BEGIN("affinity_bwd_dr_dense_partial_kernel");
+    affinity_bwd_dr_dense_partial_kernel<<<nch, 256, 0, st>>>(Z, delta, xnorm, rnorm, ddelta, part, c->T, c->E,
+                                                              m, nch, sqrtf((float)c->D));
+  } else {
+    ETR_TIME_BEGIN("affinity_bwd_dr_partial_kernel");
+    affinity_bwd_dr_partial_kernel<<<dim3(c->E, nch), 256, 0, st>>>(
+        Z, delta, xnorm, rnorm, rt->counts, rt->slot_token, dgate, part, c->E, m, Cs, nch,
+        sqrtf((float)c->D));
+  }
   ETR_LAUNCH_CHECK();
   ETR_TIME_BEGIN("affinity_bwd_dr_final_kernel");
   affinity_bwd_dr_final_kernel<<<c->E, 256, 0, st>>>(part, R, rnorm, dR, m, nch);

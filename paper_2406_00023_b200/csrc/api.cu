@@ -109,6 +109,10 @@ static void carve(const etr_config* c, int staging, char* base, etr_buffers* b, 
     t.Y_dev = cv.take(T * d * eb);
     t.dX_dev = cv.take(T * d * eb);
   }
+  if (c->gate_mode == ETR_GATE_SOFTMAX) {
+    t.lse = (float*)cv.take(T * 4);
+    t.ddelta = (float*)cv.take(T * E * 4);
+  }
   if (b) *b = t;
   *total = align_up(cv.off, 256);
 }
@@ -141,6 +145,7 @@ etr_status etr_validate(const etr_config* c) {
   if (c->mode < ETR_MODE_AUTO || c->mode > ETR_MODE_ECR) return ETR_ERR_ARG;
   if (c->gemm_impl < ETR_GEMM_AUTO || c->gemm_impl > ETR_GEMM_TCGEN05_2CTA_WIDE) return ETR_ERR_ARG;
   if (c->fuse_dispatch < ETR_FUSE_AUTO || c->fuse_dispatch > ETR_FUSE_ON) return ETR_ERR_ARG;
+  if (c->gate_mode != ETR_GATE_AFFINITY && c->gate_mode != ETR_GATE_SOFTMAX) return ETR_ERR_ARG;
   if (c->d % c->D != 0 || c->d % 8 != 0 || c->h % 8 != 0) return ETR_ERR_SHAPE;
   if (c->k > c->E || c->E > 256 || c->E > c->d / c->D) return ETR_ERR_SHAPE;
   if ((long long)c->T * c->E >= (1ll << 31)) return ETR_ERR_SHAPE;
@@ -274,8 +279,44 @@ etr_status etr_affinity_bwd(const etr_config* c, const void* X, const float* R, 
   ETR_TRY(etr_validate(c));
   ETR_TRY(check_ptrs({X, R, delta, Z, xnorm, rnorm, dgate, dX, dR, ws}));
   ETR_TRY(check_route(route));
-  return affinity_backward(c, X, R, delta, Z, xnorm, rnorm, route, dgate, nullptr, dX, dR, ws,
+  return affinity_backward(c, X, R, delta, Z, xnorm, rnorm, route, dgate, nullptr, nullptr, dX, dR, ws,
                            (cudaStream_t)stream);
+}
+
+etr_status etr_gate_softmax(const etr_config* c, const float* delta, const etr_route* route, float* lse,
+                            void* stream) {
+  ETR_TRY(etr_validate(c));
+  ETR_TRY(check_ptrs({delta, lse}));
+  ETR_TRY(check_route(route));
+  return gate_softmax_forward(c, delta, route, lse, (cudaStream_t)stream);
+}
+
+etr_status etr_gate_softmax_bwd(const etr_config* c, const float* delta, const float* lse,
+                                const etr_route* route, const float* dgate, float* ddelta,
+                                void* stream) {
+  ETR_TRY(etr_validate(c));
+  ETR_TRY(check_ptrs({delta, lse, dgate, ddelta}));
+  ETR_TRY(check_route(route));
+  return gate_softmax_backward(c, delta, lse, route, dgate, ddelta, (cudaStream_t)stream);
+}
+
+etr_status etr_affinity_bwd_dense(const etr_config* c, const void* X, const float* R, const float* delta,
+                                  const float* Z, const float* xnorm, const float* rnorm,
+                                  const etr_route* route, const float* ddelta, void* dX, float* dR,
+                                  void* ws, void* stream) {
+  ETR_TRY(etr_validate(c));
+  ETR_TRY(check_ptrs({X, R, delta, Z, xnorm, rnorm, ddelta, dX, dR, ws}));
+  ETR_TRY(check_route(route));
+  return affinity_backward(c, X, R, delta, Z, xnorm, rnorm, route, nullptr, ddelta, nullptr, dX, dR, ws,
+                           (cudaStream_t)stream);
+}
+
+etr_status etr_load_stats(const etr_config* c, const etr_route* route, float* load, float* gate_mean,
+                          void* stream) {
+  ETR_TRY(etr_validate(c));
+  ETR_TRY(check_ptrs({load, gate_mean}));
+  ETR_TRY(check_route(route));
+  return load_stats_launch(c, route, load, gate_mean, (cudaStream_t)stream);
 }
 
 etr_status etr_layer_forward(const etr_config* c, const void* X, const float* R, const void* W1g,
@@ -288,6 +329,7 @@ etr_status etr_layer_forward(const etr_config* c, const void* X, const float* R,
     return ETR_ERR_CUDA;
   ETR_TRY(etr_affinity(c, X, R, b->delta, b->Z, b->xnorm, b->rnorm, b->stats, stream));
   ETR_TRY(etr_select(c, b->delta, b->stats, &b->route, b->ws, stream));
+  if (c->gate_mode == ETR_GATE_SOFTMAX) ETR_TRY(etr_gate_softmax(c, b->delta, &b->route, b->lse, stream));
   if (fuse_dispatch(c)) {       // the first GEMM gathers its rows from X: no Xp
     ETR_TRY(check_ptrs({X, W1g, W1u, W2, b->G, b->U, b->H, b->O, b->ws}));
     ETR_TRY(tc_ffn_forward(c, &b->route, nullptr, X, W1g, W1u, W2, b->G, b->U, b->H, b->O, b->stats, b->ws,
@@ -318,8 +360,13 @@ etr_status etr_layer_backward(const etr_config* c, const void* X, const float* R
   // dispatch backward and the router gradient in one pass over dX
   ETR_TRY(etr_select_bwd(c, &b->route, b->dgate));
   ETR_TRY(check_ptrs({X, R, dX, dR, b->dXp, b->ws}));
-  return affinity_backward(c, X, R, b->delta, b->Z, b->xnorm, b->rnorm, &b->route, b->dgate, b->dXp, dX,
-                           dR, b->ws, (cudaStream_t)stream);
+  const float* ddelta = nullptr;
+  if (c->gate_mode == ETR_GATE_SOFTMAX) {
+    ETR_TRY(etr_gate_softmax_bwd(c, b->delta, b->lse, &b->route, b->dgate, b->ddelta, stream));
+    ddelta = b->ddelta;
+  }
+  return affinity_backward(c, X, R, b->delta, b->Z, b->xnorm, b->rnorm, &b->route, b->dgate, ddelta,
+                           b->dXp, dX, dR, b->ws, (cudaStream_t)stream);
 }
 
 // Side streams and events for the host-buffer step (host-side objects, created once per device).

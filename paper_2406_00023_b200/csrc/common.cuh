@@ -112,8 +112,15 @@ etr_status affinity_forward(const etr_config* c, const void* X, const float* R, 
 size_t affinity_bwd_workspace_bytes(const etr_config* c);
 etr_status affinity_backward(const etr_config* c, const void* X, const float* R, const float* delta,
                              const float* Z, const float* xnorm, const float* rnorm,
-                             const etr_route* rt, const float* dgate, const void* dXp_fused, void* dX,
-                             float* dR, void* ws, cudaStream_t st);
+                             const etr_route* rt, const float* dgate, const float* ddelta,
+                             const void* dXp_fused, void* dX, float* dR, void* ws, cudaStream_t st);
+// softmax-gate variant and load statistics (gate.cu)
+etr_status gate_softmax_forward(const etr_config* c, const float* delta, const etr_route* rt, float* lse,
+                                cudaStream_t st);
+etr_status gate_softmax_backward(const etr_config* c, const float* delta, const float* lse,
+                                 const etr_route* rt, const float* dgate, float* ddelta, cudaStream_t st);
+etr_status load_stats_launch(const etr_config* c, const etr_route* rt, float* load, float* gate_mean,
+                             cudaStream_t st);
 size_t select_workspace_bytes(const etr_config* c);
 int resolve_mode(const etr_config* c);
 etr_status select_forward(const etr_config* c, const float* delta, etr_stats* stats,

@@ -19,11 +19,13 @@ F32, BF16 = 0, 1
 MODE_AUTO, MODE_TCR, MODE_ECR = 0, 1, 2
 GEMM_AUTO, GEMM_SIMT, GEMM_TCGEN05, GEMM_TCGEN05_2CTA, GEMM_TCGEN05_2CTA_WIDE = 0, 1, 2, 3, 4
 FUSE_AUTO, FUSE_OFF, FUSE_ON = 0, 1, 2
+GATE_AFFINITY, GATE_SOFTMAX = 0, 1
 
 EXPORTS = [
     "etr_status_string", "etr_validate", "etr_c_stride", "etr_workspace_bytes", "etr_buffers_bytes",
     "etr_buffers_bind", "etr_affinity", "etr_select", "etr_select_static", "etr_dispatch", "etr_expert_ffn", "etr_combine",
     "etr_combine_bwd", "etr_expert_ffn_bwd", "etr_dispatch_bwd", "etr_select_bwd", "etr_affinity_bwd",
+    "etr_gate_softmax", "etr_gate_softmax_bwd", "etr_affinity_bwd_dense", "etr_load_stats",
     "etr_layer_forward", "etr_layer_backward", "etr_layer_step_host", "etr_layer_step_host_begin",
     "etr_layer_step_host_wait", "etr_read_stats",
     "etr_launch_count", "etr_timing_enable", "etr_timing_collect",
@@ -35,7 +37,8 @@ class Config(C.Structure):
                 ("k", C.c_int32), ("h", C.c_int32), ("capacity", C.c_int32), ("c_floor", C.c_int32),
                 ("adaptive", C.c_int32), ("delta_max_override", C.c_float),
                 ("step", C.c_int64), ("switch_step", C.c_int64), ("mode", C.c_int32),
-                ("dtype", C.c_int32), ("gemm_impl", C.c_int32), ("fuse_dispatch", C.c_int32)]
+                ("dtype", C.c_int32), ("gemm_impl", C.c_int32), ("fuse_dispatch", C.c_int32),
+                ("gate_mode", C.c_int32), ("reserved", C.c_int32)]
 
 
 class Stats(C.Structure):
@@ -54,7 +57,7 @@ class Buffers(C.Structure):
                [(n, C.c_void_p) for n in ("delta", "Z", "xnorm", "rnorm", "Xp", "G", "U", "H", "O",
                                           "dO", "dG", "dU", "dXp", "dgate", "ws")] + \
                [("ws_bytes", C.c_size_t)] + \
-               [(n, C.c_void_p) for n in ("X_dev", "dY_dev", "Y_dev", "dX_dev")]
+               [(n, C.c_void_p) for n in ("X_dev", "dY_dev", "Y_dev", "dX_dev", "lse", "ddelta")]
 
 
 class EtrError(RuntimeError):
@@ -123,11 +126,11 @@ def _stream():
 
 def make_config(*, T, d, D, E, k, h, capacity, dtype, mode=MODE_AUTO, step=0, switch_step=0,
                 adaptive=False, c_floor=1, delta_max_override=-1.0, gemm_impl=GEMM_AUTO,
-                fuse_dispatch=0) -> Config:
+                fuse_dispatch=0, gate_mode=0) -> Config:
     return Config(T=T, d=d, D=D, E=E, k=k, h=h, capacity=capacity, c_floor=c_floor,
                   adaptive=int(bool(adaptive)), delta_max_override=float(delta_max_override),
                   step=int(step), switch_step=int(switch_step), mode=int(mode), dtype=int(dtype),
-                  gemm_impl=int(gemm_impl), fuse_dispatch=int(fuse_dispatch))
+                  gemm_impl=int(gemm_impl), fuse_dispatch=int(fuse_dispatch), gate_mode=int(gate_mode), reserved=0)
 
 
 def torch_dtype(cfg: Config):
@@ -184,6 +187,9 @@ class LayerBuffers:
         if host_staging:
             for name in ("X_dev", "dY_dev", "Y_dev", "dX_dev"):
                 setattr(self, name, self._view(getattr(self.c, name), (T, d), act))
+        if cfg.gate_mode == GATE_SOFTMAX:
+            self.lse = self._view(self.c.lse, (T,), torch.float32)
+            self.ddelta = self._view(self.c.ddelta, (T, E), torch.float32)
 
     def _view(self, ptr, shape, dtype):
         off = ptr - self.block.data_ptr()
@@ -269,6 +275,27 @@ def affinity_bwd(cfg, X, R, delta, Z, xnorm, rnorm, route: Route, dgate, dX, dR,
     _check(lib().etr_affinity_bwd(C.byref(cfg), _p(X), _p(R), _p(delta), _p(Z), _p(xnorm), _p(rnorm),
                                   C.byref(route), _p(dgate), _p(dX), _p(dR), _p(ws), _stream()),
            "etr_affinity_bwd")
+
+
+def gate_softmax(cfg, delta, route: Route, lse):
+    _check(lib().etr_gate_softmax(C.byref(cfg), _p(delta), C.byref(route), _p(lse), _stream()),
+           "etr_gate_softmax")
+
+
+def gate_softmax_bwd(cfg, delta, lse, route: Route, dgate, ddelta):
+    _check(lib().etr_gate_softmax_bwd(C.byref(cfg), _p(delta), _p(lse), C.byref(route), _p(dgate),
+                                      _p(ddelta), _stream()), "etr_gate_softmax_bwd")
+
+
+def affinity_bwd_dense(cfg, X, R, delta, Z, xnorm, rnorm, route: Route, ddelta, dX, dR, ws):
+    _check(lib().etr_affinity_bwd_dense(C.byref(cfg), _p(X), _p(R), _p(delta), _p(Z), _p(xnorm), _p(rnorm),
+                                        C.byref(route), _p(ddelta), _p(dX), _p(dR), _p(ws), _stream()),
+           "etr_affinity_bwd_dense")
+
+
+def load_stats(cfg, route: Route, load, gate_mean):
+    _check(lib().etr_load_stats(C.byref(cfg), C.byref(route), _p(load), _p(gate_mean), _stream()),
+           "etr_load_stats")
 
 
 def layer_forward(cfg, X, R, W1g, W1u, W2, buf: LayerBuffers, Y):

@@ -42,4 +42,4 @@ def test_host_side_validation_needs_no_gpu():
     n = ctypes.c_size_t(0)
     assert etr.lib().etr_buffers_bytes(ctypes.byref(good), 1, ctypes.byref(n)) == etr.OK and n.value > 1 << 20
     # struct layouts the binding relies on
-    assert ctypes.sizeof(etr.Config) == 72 and ctypes.sizeof(etr.Stats) == 64
+    assert ctypes.sizeof(etr.Config) == 80 and ctypes.sizeof(etr.Stats) == 64
