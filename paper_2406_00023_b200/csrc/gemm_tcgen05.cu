@@ -623,7 +623,9 @@ __device__ __forceinline__ bool tile_coord_pair(const TcParams& p, const int* ti
   return true;
 }
 
-template <int EPI>
+// GATHER is TcParams::gather as a compile-time constant: the producer loop is on the kernel's
+// critical path, and even branches not taken cost there.
+template <int EPI, int GATHER>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 tc_grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtensorMap mapA1,
                             const __grid_constant__ CUtensorMap mapB0, const __grid_constant__ CUtensorMap mapB1,
@@ -680,7 +682,7 @@ tc_grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap mapA0, const __g
     // Without a gather lane 0 works alone.  With one, the whole warp walks the loop: lane l
     // fetches rows 4l..4l+3 of the gathered operand's 128 (gather 1) or, for the two 64-column
     // boxes of a K block, rows 4(l%16)..+3 of box l/16 (gather 2); lane 0 issues the rest.
-    if (lane == 0 || p.gather) {
+    if (lane == 0 || GATHER) {
       int e_cur = 0, stage = 0;
       uint32_t phase = 0;
       TileCoord tc;
@@ -689,13 +691,13 @@ tc_grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap mapA0, const __g
         const int m0c = tc.m0 + 128 * (int)rank;
         const int32_t* gidx = p.gather_idx + (size_t)tc.e * p.gather_ld;
         int4 rows_a = make_int4(0, 0, 0, 0), rows_b = make_int4(0, 0, 0, 0);
-        if (p.gather == 1)      // a CTA's 128 rows lie inside the expert's C_stride slots or all past them
+        if (GATHER == 1)      // a CTA's 128 rows lie inside the expert's C_stride slots or all past them
           rows_a = m0c < p.M ? gather_rows(gidx + m0c + 4 * lane, p.gather_oob)
                              : make_int4(p.gather_oob, p.gather_oob, p.gather_oob, p.gather_oob);
-        if (p.gather == 2 && tc.kblocks > 0) rows_b = gather_rows(gidx + 4 * (lane & 15), p.gather_oob);
+        if (GATHER == 2 && tc.kblocks > 0) rows_b = gather_rows(gidx + 4 * (lane & 15), p.gather_oob);
         for (int kb = 0; kb < tc.kblocks; ++kb) {
           int4 rows_next = rows_b;
-          if (p.gather == 2 && kb + 1 < tc.kblocks)
+          if (GATHER == 2 && kb + 1 < tc.kblocks)
             rows_next = gather_rows(gidx + (kb + 1) * TC_BK + 4 * (lane & 15), p.gather_oob);
           if (!mbar_wait_cluster(empty_bar + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
           if (rank == 0 && lane == 0) mbar_expect_tx(full_bar + 8 * stage, 2 * TC2_STAGE_BYTES);
@@ -707,18 +709,18 @@ tc_grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap mapA0, const __g
           const int nb = p.dual_b ? tc.n0 : tc.n0 + 128 * (int)rank;
           const uint32_t sa = tiles_base + stage * TC2_STAGE_BYTES;
           const uint32_t sb = sa + 2 * TC_BOX_BYTES;
-          if (p.gather == 1) tma_gather4_pair(sa + 512u * lane, &mapA0, fb, k0, rows_a);
-          if (p.gather == 2)
+          if (GATHER == 1) tma_gather4_pair(sa + 512u * lane, &mapA0, fb, k0, rows_a);
+          if (GATHER == 2)
             tma_gather4_pair(sb + (lane >> 4) * TC_BOX_BYTES + 512u * (lane & 15), &mapB0, fb,
                              nb + 64 * (lane >> 4), rows_b);
           if (lane == 0) {
 #pragma unroll
             for (int j = 0; j < 2; ++j) {
-              if (p.gather != 1) {
+              if (GATHER != 1) {
                 if (p.a_mn) tma_load_3d_pair(sa + j * TC_BOX_BYTES, ma, fb, m0c + 64 * j, k0, tc.e);
                 else        tma_load_3d_pair(sa + j * TC_BOX_BYTES, ma, fb, k0, m0c + 64 * j, tc.e);
               }
-              if (p.gather != 2) {
+              if (GATHER != 2) {
                 if (p.b_mn) tma_load_3d_pair(sb + j * TC_BOX_BYTES, mb, fb, nb + 64 * j, k0, tc.e);
                 else        tma_load_3d_pair(sb + j * TC_BOX_BYTES, mb, fb, k0, nb + 64 * j, tc.e);
               }
@@ -855,7 +857,7 @@ __device__ __forceinline__ bool tile_coord_wide(const TcParams& p, const int* ti
   return true;
 }
 
-template <int EPI>
+template <int EPI, int GATHER>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 tc_grouped_gemm_pair_wide_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtensorMap mapA1,
                                  const __grid_constant__ CUtensorMap mapB0, const __grid_constant__ CUtensorMap mapB1,
@@ -912,7 +914,7 @@ tc_grouped_gemm_pair_wide_kernel(const __grid_constant__ CUtensorMap mapA0, cons
     // ---- TMA producer (both CTAs) ---------------------------------------------------------------
     // Lane 0 alone, or with a gathered A operand the whole warp (lane l fetches rows 4l..4l+3 of
     // the CTA's 128 rows of A; lane 0 also issues the B boxes).
-    if (lane == 0 || p.gather) {
+    if (lane == 0 || GATHER) {
       int e_cur = 0, stage = 0;
       uint32_t phase = 0;
       TileCoord tc;
@@ -921,7 +923,7 @@ tc_grouped_gemm_pair_wide_kernel(const __grid_constant__ CUtensorMap mapA0, cons
         const int m0c = tc.m0 + 128 * (int)rank;
         const bool two = tc.n0 + N_TILE_COLS < p.N;
         int4 rows_a = make_int4(0, 0, 0, 0);
-        if (p.gather == 1)
+        if (GATHER == 1)
           rows_a = m0c < p.M ? gather_rows(p.gather_idx + (size_t)tc.e * p.gather_ld + m0c + 4 * lane, p.gather_oob)
                              : make_int4(p.gather_oob, p.gather_oob, p.gather_oob, p.gather_oob);
         for (int kb = 0; kb < tc.kblocks; ++kb) {
@@ -933,9 +935,9 @@ tc_grouped_gemm_pair_wide_kernel(const __grid_constant__ CUtensorMap mapA0, cons
           const CUtensorMap* ma = second ? &mapA1 : &mapA0;
           const CUtensorMap* mb = p.dual_b ? (rank ? &mapB1 : &mapB0) : (second ? &mapB1 : &mapB0);
           const uint32_t sa = tiles_base + stage * TCW_STAGE_BYTES;
-          if (p.gather == 1) tma_gather4_pair(sa + 512u * lane, &mapA0, fb, k0, rows_a);
+          if (GATHER == 1) tma_gather4_pair(sa + 512u * lane, &mapA0, fb, k0, rows_a);
           if (lane == 0) {
-            if (p.gather != 1) {
+            if (GATHER != 1) {
 #pragma unroll
               for (int j = 0; j < 2; ++j) {
                 if (p.a_mn) tma_load_3d_pair(sa + j * TC_BOX_BYTES, ma, fb, m0c + 64 * j, k0, tc.e);
@@ -1207,12 +1209,12 @@ static etr_status tc_launch(const char* name, const CUtensorMap& a0, const CUten
   return ETR_OK;
 }
 
-template <int EPI>
+template <int EPI, int GATHER>
 static etr_status tc_launch_pair(const char* name, const CUtensorMap& a0, const CUtensorMap& a1,
                                  const CUtensorMap& b0, const CUtensorMap& b1, TcParams p, int max_tiles,
                                  cudaStream_t st) {
   constexpr size_t smem = (size_t)TC2_STAGES * TC2_STAGE_BYTES + 1024 + 8 * TC_SCRATCH_BYTES;
-  auto k = tc_grouped_gemm_pair_kernel<EPI>;
+  auto k = tc_grouped_gemm_pair_kernel<EPI, GATHER>;
   static bool attr_set = false;
   if (!attr_set) {
     if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
@@ -1238,12 +1240,12 @@ static etr_status tc_launch_pair(const char* name, const CUtensorMap& a0, const 
   return ETR_OK;
 }
 
-template <int EPI>
+template <int EPI, int GATHER>
 static etr_status tc_launch_pair_wide(const char* name, const CUtensorMap& a0, const CUtensorMap& a1,
                                       const CUtensorMap& b0, const CUtensorMap& b1, TcParams p, int max_tiles,
                                       cudaStream_t st) {
   constexpr size_t smem = (size_t)TCW_STAGES * TCW_STAGE_BYTES + 1024 + 8 * TC_SCRATCH_BYTES;
-  auto k = tc_grouped_gemm_pair_wide_kernel<EPI>;
+  auto k = tc_grouped_gemm_pair_wide_kernel<EPI, GATHER>;
   static bool attr_set = false;
   if (!attr_set) {
     if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
@@ -1304,8 +1306,22 @@ template <int EPI>
 static etr_status tc_run(TcForm form, const char* name, const CUtensorMap& a0, const CUtensorMap& a1,
                          const CUtensorMap& b0, const CUtensorMap& b1, const TcParams& p, int max_tiles,
                          cudaStream_t st) {
-  if (form == TC_FORM_PAIR_WIDE) return tc_launch_pair_wide<EPI>(name, a0, a1, b0, b1, p, (max_tiles + 1) / 2, st);
-  if (form == TC_FORM_PAIR) return tc_launch_pair<EPI>(name, a0, a1, b0, b1, p, (max_tiles + 1) / 2, st);
+  // gathered operands exist for the SwiGLU GEMM (A rows) and the plain-store weight gradients (K rows)
+  if (form == TC_FORM_PAIR_WIDE) {
+    if (EPI == TC_EPI_SWIGLU && p.gather == 1)
+      return tc_launch_pair_wide<EPI, EPI == TC_EPI_SWIGLU ? 1 : 0>(name, a0, a1, b0, b1, p, (max_tiles + 1) / 2, st);
+    if (p.gather) return ETR_ERR_UNSUPPORTED;
+    return tc_launch_pair_wide<EPI, 0>(name, a0, a1, b0, b1, p, (max_tiles + 1) / 2, st);
+  }
+  if (form == TC_FORM_PAIR) {
+    if (EPI == TC_EPI_SWIGLU && p.gather == 1)
+      return tc_launch_pair<EPI, EPI == TC_EPI_SWIGLU ? 1 : 0>(name, a0, a1, b0, b1, p, (max_tiles + 1) / 2, st);
+    if (EPI == TC_EPI_STORE && p.gather == 2)
+      return tc_launch_pair<EPI, EPI == TC_EPI_STORE ? 2 : 0>(name, a0, a1, b0, b1, p, (max_tiles + 1) / 2, st);
+    if (p.gather) return ETR_ERR_UNSUPPORTED;
+    return tc_launch_pair<EPI, 0>(name, a0, a1, b0, b1, p, (max_tiles + 1) / 2, st);
+  }
+  if (p.gather) return ETR_ERR_UNSUPPORTED;
   return tc_launch<256, EPI>(name, a0, a1, b0, b1, p, max_tiles, st);
 }
 
