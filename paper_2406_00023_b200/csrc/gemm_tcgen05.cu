@@ -623,9 +623,12 @@ __device__ __forceinline__ bool tile_coord_pair(const TcParams& p, const int* ti
   return true;
 }
 
-// GATHER is TcParams::gather as a compile-time constant: the producer loop is on the kernel's
-// critical path, and even branches not taken cost there.
-template <int EPI, int GATHER>
+// GATHER is TcParams::gather, and CFG the operand modes (a_mn, b_mn, dual_b, two K ranges), as
+// compile-time constants: the single-lane producer and MMA loops are on the kernel's critical path,
+// and run-time branches cost there even when not taken (6-8 % of a GEMM for the operand modes,
+// 10 % per gather branch).  CFG = -1 keeps the run-time forms for combinations without an
+// instantiation of their own.
+template <int EPI, int GATHER, int CFG>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 tc_grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtensorMap mapA1,
                             const __grid_constant__ CUtensorMap mapB0, const __grid_constant__ CUtensorMap mapB1,
@@ -633,6 +636,9 @@ tc_grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap mapA0, const __g
   constexpr int BN = 256;
   constexpr int N_TILE_COLS = (EPI == TC_EPI_SWIGLU) ? BN / 2 : BN;
   constexpr uint32_t TMEM_COLS = 512;
+  // operand modes as compile-time constants when CFG >= 0 (bit 0 a_mn, 1 b_mn, 2 dual_b, 3 two K ranges)
+  const bool A_MN = CFG < 0 ? p.a_mn != 0 : (CFG & 1) != 0, B_MN = CFG < 0 ? p.b_mn != 0 : (CFG & 2) != 0;
+  const bool DUAL_B = CFG < 0 ? p.dual_b != 0 : (CFG & 4) != 0, TWO_K = CFG < 0 ? p.k1_blocks > 0 : (CFG & 8) != 0;
 
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t bars[2 * TC2_STAGES + 4];
@@ -702,11 +708,11 @@ tc_grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap mapA0, const __g
           if (!mbar_wait_cluster(empty_bar + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
           if (rank == 0 && lane == 0) mbar_expect_tx(full_bar + 8 * stage, 2 * TC2_STAGE_BYTES);
           const uint32_t fb = leader_full + 8 * stage;
-          const bool second = p.k1_blocks > 0 && kb >= p.k1_blocks;
+          const bool second = TWO_K && kb >= p.k1_blocks;
           const int k0 = (second ? kb - p.k1_blocks : kb) * TC_BK;
           const CUtensorMap* ma = second ? &mapA1 : &mapA0;
-          const CUtensorMap* mb = p.dual_b ? (rank ? &mapB1 : &mapB0) : (second ? &mapB1 : &mapB0);
-          const int nb = p.dual_b ? tc.n0 : tc.n0 + 128 * (int)rank;
+          const CUtensorMap* mb = DUAL_B ? (rank ? &mapB1 : &mapB0) : (second ? &mapB1 : &mapB0);
+          const int nb = DUAL_B ? tc.n0 : tc.n0 + 128 * (int)rank;
           const uint32_t sa = tiles_base + stage * TC2_STAGE_BYTES;
           const uint32_t sb = sa + 2 * TC_BOX_BYTES;
           if (GATHER == 1) tma_gather4_pair(sa + 512u * lane, &mapA0, fb, k0, rows_a);
@@ -717,11 +723,11 @@ tc_grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap mapA0, const __g
 #pragma unroll
             for (int j = 0; j < 2; ++j) {
               if (GATHER != 1) {
-                if (p.a_mn) tma_load_3d_pair(sa + j * TC_BOX_BYTES, ma, fb, m0c + 64 * j, k0, tc.e);
+                if (A_MN) tma_load_3d_pair(sa + j * TC_BOX_BYTES, ma, fb, m0c + 64 * j, k0, tc.e);
                 else        tma_load_3d_pair(sa + j * TC_BOX_BYTES, ma, fb, k0, m0c + 64 * j, tc.e);
               }
               if (GATHER != 2) {
-                if (p.b_mn) tma_load_3d_pair(sb + j * TC_BOX_BYTES, mb, fb, nb + 64 * j, k0, tc.e);
+                if (B_MN) tma_load_3d_pair(sb + j * TC_BOX_BYTES, mb, fb, nb + 64 * j, k0, tc.e);
                 else        tma_load_3d_pair(sb + j * TC_BOX_BYTES, mb, fb, k0, nb + 64 * j, tc.e);
               }
             }
@@ -738,8 +744,8 @@ tc_grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap mapA0, const __g
       uint32_t phase = 0, acc_phase = 0;
       TileCoord tc;
       bool ok = true;
-      const uint32_t a_lbo = p.a_mn ? TC_BOX_BYTES : 16u, b_lbo = p.b_mn ? TC_BOX_BYTES : 16u;
-      const uint32_t a_kstep = p.a_mn ? 2048u : 32u, b_kstep = p.b_mn ? 2048u : 32u;
+      const uint32_t a_lbo = A_MN ? TC_BOX_BYTES : 16u, b_lbo = B_MN ? TC_BOX_BYTES : 16u;
+      const uint32_t a_kstep = A_MN ? 2048u : 32u, b_kstep = B_MN ? 2048u : 32u;
       for (int tile = pair; ok && tile_coord_pair(p, tile_prefix, tile, e_cur, N_TILE_COLS, tc); tile += npairs) {
         if (tc.kblocks == 0) continue;
         if (!mbar_wait_cluster(tempty_bar + 8 * acc_stage, acc_phase ^ 1u, abort_flag)) { ok = false; break; }
@@ -857,7 +863,7 @@ __device__ __forceinline__ bool tile_coord_wide(const TcParams& p, const int* ti
   return true;
 }
 
-template <int EPI, int GATHER>
+template <int EPI, int GATHER, int CFG>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 tc_grouped_gemm_pair_wide_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_constant__ CUtensorMap mapA1,
                                  const __grid_constant__ CUtensorMap mapB0, const __grid_constant__ CUtensorMap mapB1,
@@ -865,6 +871,9 @@ tc_grouped_gemm_pair_wide_kernel(const __grid_constant__ CUtensorMap mapA0, cons
   constexpr int BN = 256;
   constexpr int N_TILE_COLS = (EPI == TC_EPI_SWIGLU) ? BN / 2 : BN;
   constexpr uint32_t TMEM_COLS = 512;
+  // operand modes as compile-time constants when CFG >= 0 (bit 0 a_mn, 1 b_mn, 2 dual_b, 3 two K ranges)
+  const bool A_MN = CFG < 0 ? p.a_mn != 0 : (CFG & 1) != 0, B_MN = CFG < 0 ? p.b_mn != 0 : (CFG & 2) != 0;
+  const bool DUAL_B = CFG < 0 ? p.dual_b != 0 : (CFG & 4) != 0, TWO_K = CFG < 0 ? p.k1_blocks > 0 : (CFG & 8) != 0;
 
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t bars[2 * TCW_STAGES + 3];
@@ -930,27 +939,27 @@ tc_grouped_gemm_pair_wide_kernel(const __grid_constant__ CUtensorMap mapA0, cons
           if (!mbar_wait_cluster(empty_bar + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
           if (rank == 0 && lane == 0) mbar_expect_tx(full_bar + 8 * stage, 2 * (two ? 6 : 4) * TC_BOX_BYTES);
           const uint32_t fb = leader_full + 8 * stage;
-          const bool second = p.k1_blocks > 0 && kb >= p.k1_blocks;
+          const bool second = TWO_K && kb >= p.k1_blocks;
           const int k0 = (second ? kb - p.k1_blocks : kb) * TC_BK;
           const CUtensorMap* ma = second ? &mapA1 : &mapA0;
-          const CUtensorMap* mb = p.dual_b ? (rank ? &mapB1 : &mapB0) : (second ? &mapB1 : &mapB0);
+          const CUtensorMap* mb = DUAL_B ? (rank ? &mapB1 : &mapB0) : (second ? &mapB1 : &mapB0);
           const uint32_t sa = tiles_base + stage * TCW_STAGE_BYTES;
           if (GATHER == 1) tma_gather4_pair(sa + 512u * lane, &mapA0, fb, k0, rows_a);
           if (lane == 0) {
             if (GATHER != 1) {
 #pragma unroll
               for (int j = 0; j < 2; ++j) {
-                if (p.a_mn) tma_load_3d_pair(sa + j * TC_BOX_BYTES, ma, fb, m0c + 64 * j, k0, tc.e);
+                if (A_MN) tma_load_3d_pair(sa + j * TC_BOX_BYTES, ma, fb, m0c + 64 * j, k0, tc.e);
                 else        tma_load_3d_pair(sa + j * TC_BOX_BYTES, ma, fb, k0, m0c + 64 * j, tc.e);
               }
             }
             for (int hf = 0; hf < (two ? 2 : 1); ++hf) {
               const uint32_t sb = sa + (2 + 2 * hf) * TC_BOX_BYTES;
               const int nh = tc.n0 + hf * N_TILE_COLS;
-              const int nb = p.dual_b ? nh : nh + 128 * (int)rank;
+              const int nb = DUAL_B ? nh : nh + 128 * (int)rank;
 #pragma unroll
               for (int j = 0; j < 2; ++j) {
-                if (p.b_mn) tma_load_3d_pair(sb + j * TC_BOX_BYTES, mb, fb, nb + 64 * j, k0, tc.e);
+                if (B_MN) tma_load_3d_pair(sb + j * TC_BOX_BYTES, mb, fb, nb + 64 * j, k0, tc.e);
                 else        tma_load_3d_pair(sb + j * TC_BOX_BYTES, mb, fb, k0, nb + 64 * j, tc.e);
               }
             }
@@ -966,8 +975,8 @@ tc_grouped_gemm_pair_wide_kernel(const __grid_constant__ CUtensorMap mapA0, cons
       uint32_t phase = 0, acc_phase = 0;
       TileCoord tc;
       bool ok = true;
-      const uint32_t a_lbo = p.a_mn ? TC_BOX_BYTES : 16u, b_lbo = p.b_mn ? TC_BOX_BYTES : 16u;
-      const uint32_t a_kstep = p.a_mn ? 2048u : 32u, b_kstep = p.b_mn ? 2048u : 32u;
+      const uint32_t a_lbo = A_MN ? TC_BOX_BYTES : 16u, b_lbo = B_MN ? TC_BOX_BYTES : 16u;
+      const uint32_t a_kstep = A_MN ? 2048u : 32u, b_kstep = B_MN ? 2048u : 32u;
       // one K block of one half: 4 MMAs of 256 x 256 x 16
       auto issue = [&](int st, int hf, bool first_block) {
         const uint32_t sa = tiles_base + st * TCW_STAGE_BYTES;
@@ -1209,12 +1218,12 @@ static etr_status tc_launch(const char* name, const CUtensorMap& a0, const CUten
   return ETR_OK;
 }
 
-template <int EPI, int GATHER>
-static etr_status tc_launch_pair(const char* name, const CUtensorMap& a0, const CUtensorMap& a1,
+template <int EPI, int GATHER, int CFG>
+static etr_status tc_launch_pair_cfg(const char* name, const CUtensorMap& a0, const CUtensorMap& a1,
                                  const CUtensorMap& b0, const CUtensorMap& b1, TcParams p, int max_tiles,
                                  cudaStream_t st) {
   constexpr size_t smem = (size_t)TC2_STAGES * TC2_STAGE_BYTES + 1024 + 8 * TC_SCRATCH_BYTES;
-  auto k = tc_grouped_gemm_pair_kernel<EPI, GATHER>;
+  auto k = tc_grouped_gemm_pair_kernel<EPI, GATHER, CFG>;
   static bool attr_set = false;
   if (!attr_set) {
     if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
@@ -1240,12 +1249,12 @@ static etr_status tc_launch_pair(const char* name, const CUtensorMap& a0, const 
   return ETR_OK;
 }
 
-template <int EPI, int GATHER>
-static etr_status tc_launch_pair_wide(const char* name, const CUtensorMap& a0, const CUtensorMap& a1,
+template <int EPI, int GATHER, int CFG>
+static etr_status tc_launch_pair_wide_cfg(const char* name, const CUtensorMap& a0, const CUtensorMap& a1,
                                       const CUtensorMap& b0, const CUtensorMap& b1, TcParams p, int max_tiles,
                                       cudaStream_t st) {
   constexpr size_t smem = (size_t)TCW_STAGES * TCW_STAGE_BYTES + 1024 + 8 * TC_SCRATCH_BYTES;
-  auto k = tc_grouped_gemm_pair_wide_kernel<EPI, GATHER>;
+  auto k = tc_grouped_gemm_pair_wide_kernel<EPI, GATHER, CFG>;
   static bool attr_set = false;
   if (!attr_set) {
     if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
@@ -1269,6 +1278,33 @@ static etr_status tc_launch_pair_wide(const char* name, const CUtensorMap& a0, c
   if (cudaLaunchKernelEx(&cfg, k, a0, a1, b0, b1, p) != cudaSuccess) { timing_end(st); return ETR_ERR_CUDA; }
   ETR_LAUNCH_CHECK();
   return ETR_OK;
+}
+
+
+// The operand modes each epilogue is used with get their own instantiation; anything else runs the
+// generic one (CFG = -1).
+template <int EPI, int GATHER>
+static etr_status tc_launch_pair(const char* name, const CUtensorMap& a0, const CUtensorMap& a1,
+                                 const CUtensorMap& b0, const CUtensorMap& b1, TcParams p, int max_tiles,
+                                 cudaStream_t st) {
+  const int cfg = (p.a_mn ? 1 : 0) | (p.b_mn ? 2 : 0) | (p.dual_b ? 4 : 0) | (p.k1_blocks > 0 ? 8 : 0);
+  constexpr int C0 = EPI == TC_EPI_SWIGLU ? 4 : EPI == TC_EPI_DSWIGLU ? 2 : 0;      // first use
+  constexpr int C1 = EPI == TC_EPI_STORE ? 3 : C0, C2 = EPI == TC_EPI_STORE ? 10 : C0;
+  if (cfg == C0) return tc_launch_pair_cfg<EPI, GATHER, C0>(name, a0, a1, b0, b1, p, max_tiles, st);
+  if (cfg == C1) return tc_launch_pair_cfg<EPI, GATHER, C1>(name, a0, a1, b0, b1, p, max_tiles, st);
+  if (cfg == C2) return tc_launch_pair_cfg<EPI, GATHER, C2>(name, a0, a1, b0, b1, p, max_tiles, st);
+  return tc_launch_pair_cfg<EPI, GATHER, -1>(name, a0, a1, b0, b1, p, max_tiles, st);
+}
+template <int EPI, int GATHER>
+static etr_status tc_launch_pair_wide(const char* name, const CUtensorMap& a0, const CUtensorMap& a1,
+                                      const CUtensorMap& b0, const CUtensorMap& b1, TcParams p, int max_tiles,
+                                      cudaStream_t st) {
+  const int cfg = (p.a_mn ? 1 : 0) | (p.b_mn ? 2 : 0) | (p.dual_b ? 4 : 0) | (p.k1_blocks > 0 ? 8 : 0);
+  constexpr int C0 = EPI == TC_EPI_SWIGLU ? 4 : EPI == TC_EPI_DSWIGLU ? 2 : 0;
+  constexpr int C2 = EPI == TC_EPI_STORE ? 10 : C0;
+  if (cfg == C0) return tc_launch_pair_wide_cfg<EPI, GATHER, C0>(name, a0, a1, b0, b1, p, max_tiles, st);
+  if (cfg == C2) return tc_launch_pair_wide_cfg<EPI, GATHER, C2>(name, a0, a1, b0, b1, p, max_tiles, st);
+  return tc_launch_pair_wide_cfg<EPI, GATHER, -1>(name, a0, a1, b0, b1, p, max_tiles, st);
 }
 
 // The three forms of one contraction; max_tiles is an upper bound counted in 128-row tiles of one
