@@ -300,12 +300,13 @@ __device__ __forceinline__ void epilogue_chunks(const TcParams& p, int n0, uint3
 
 
 // Tile index -> coordinates.  tile_prefix[e] = first tile of expert e.
-__device__ __forceinline__ bool tile_coord(const TcParams& p, const int* tile_prefix, int tile, int& e_cur,
+__device__ __forceinline__ bool tile_coord(const TcParams& p, const int* tile_prefix, const int* counts_s,
+    int tile, int& e_cur,
                                            int n_tile_cols, TileCoord& tc) {
   if (tile >= tile_prefix[p.E]) return false;
   while (tile >= tile_prefix[e_cur + 1]) ++e_cur;
   const int local = tile - tile_prefix[e_cur];
-  const int n_e = p.counts[e_cur];
+  const int n_e = counts_s[e_cur];
   int mt_count;
   if (p.dyn == TC_DYN_M) {
     mt_count = (min(n_e, p.M) + TC_BM - 1) / TC_BM;
@@ -338,6 +339,7 @@ tc_grouped_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_c
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag_s;
   __shared__ int tile_prefix[257];
+  __shared__ int s_counts[256];      // the experts' row counts, read from global memory once
 
   volatile int* abort_flag = &abort_flag_s;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -348,6 +350,8 @@ tc_grouped_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_c
   const uint32_t tempty_bar = smem_u32(&bars[2 * TC_STAGES + 2]); // [2]
 
   // ---- set-up ---------------------------------------------------------------------------------
+  for (int e = tid; e < p.E; e += TC_THREADS) s_counts[e] = p.counts[e];
+  __syncthreads();
   if (tid == 0) {
     abort_flag_s = 0;
     for (int s = 0; s < TC_STAGES; ++s) { mbar_init(full_bar + 8 * s, 1); mbar_init(empty_bar + 8 * s, 1); }
@@ -357,7 +361,7 @@ tc_grouped_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_c
     int acc = 0;
     for (int e = 0; e < p.E; ++e) {
       tile_prefix[e] = acc;
-      const int n_e = p.counts[e];
+      const int n_e = s_counts[e];
       const int mt = p.dyn == TC_DYN_M ? (min(n_e, p.M) + TC_BM - 1) / TC_BM : (p.M + TC_BM - 1) / TC_BM;
       acc += mt * nt;
     }
@@ -379,7 +383,7 @@ tc_grouped_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_c
       uint32_t phase = 0;
       TileCoord tc;
       bool ok = true;
-      for (int tile = blockIdx.x; ok && tile_coord(p, tile_prefix, tile, e_cur, N_TILE_COLS, tc); tile += gridDim.x) {
+      for (int tile = blockIdx.x; ok && tile_coord(p, tile_prefix, s_counts, tile, e_cur, N_TILE_COLS, tc); tile += gridDim.x) {
         for (int kb = 0; kb < tc.kblocks; ++kb) {
           if (!mbar_wait(empty_bar + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
           const uint32_t fb = full_bar + 8 * stage;
@@ -419,7 +423,7 @@ tc_grouped_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_c
       bool ok = true;
       const uint32_t a_lbo = p.a_mn ? TC_BOX_BYTES : 16u, b_lbo = p.b_mn ? TC_BOX_BYTES : 16u;
       const uint32_t a_kstep = p.a_mn ? 2048u : 32u, b_kstep = p.b_mn ? 2048u : 32u;
-      for (int tile = blockIdx.x; ok && tile_coord(p, tile_prefix, tile, e_cur, N_TILE_COLS, tc); tile += gridDim.x) {
+      for (int tile = blockIdx.x; ok && tile_coord(p, tile_prefix, s_counts, tile, e_cur, N_TILE_COLS, tc); tile += gridDim.x) {
         if (tc.kblocks == 0) continue;
         if (!mbar_wait(tempty_bar + 8 * acc_stage, acc_phase ^ 1u, abort_flag)) { ok = false; break; }
         tc_fence_after();
@@ -454,7 +458,7 @@ tc_grouped_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_c
     uint32_t acc_phase = 0;
     TileCoord tc;
     bool ok = true;
-    for (int tile = blockIdx.x; ok && tile_coord(p, tile_prefix, tile, e_cur, N_TILE_COLS, tc); tile += gridDim.x) {
+    for (int tile = blockIdx.x; ok && tile_coord(p, tile_prefix, s_counts, tile, e_cur, N_TILE_COLS, tc); tile += gridDim.x) {
       const int grow = tc.m0 + row_in_tile;
       const bool row_ok = grow < tc.m_lim;
       const int c_beg = half * NCH;
@@ -601,12 +605,13 @@ __device__ __forceinline__ void tc_mma_pair(uint32_t d_tmem, uint64_t adesc, uin
 }
 
 // Pair-tile index -> coordinates (256 rows per pair tile).
-__device__ __forceinline__ bool tile_coord_pair(const TcParams& p, const int* tile_prefix, int tile, int& e_cur,
+__device__ __forceinline__ bool tile_coord_pair(const TcParams& p, const int* tile_prefix, const int* counts_s,
+    int tile, int& e_cur,
                                                 int n_tile_cols, TileCoord& tc) {
   if (tile >= tile_prefix[p.E]) return false;
   while (tile >= tile_prefix[e_cur + 1]) ++e_cur;
   const int local = tile - tile_prefix[e_cur];
-  const int n_e = p.counts[e_cur];
+  const int n_e = counts_s[e_cur];
   int mt_count;
   if (p.dyn == TC_DYN_M) {
     mt_count = (min(n_e, p.M) + 255) / 256;
@@ -645,6 +650,7 @@ tc_grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap mapA0, const __g
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag_s;
   __shared__ int tile_prefix[257];
+  __shared__ int s_counts[256];      // the experts' row counts, read from global memory once
 
   volatile int* abort_flag = &abort_flag_s;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -656,6 +662,8 @@ tc_grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap mapA0, const __g
   const uint32_t tfull_bar = smem_u32(&bars[2 * TC2_STAGES]);      // [2]           in each CTA
   const uint32_t tempty_bar = smem_u32(&bars[2 * TC2_STAGES + 2]); // [2]           used in the leader
 
+  for (int e = tid; e < p.E; e += TC_THREADS) s_counts[e] = p.counts[e];
+  __syncthreads();
   if (tid == 0) {
     abort_flag_s = 0;
     for (int s = 0; s < TC2_STAGES; ++s) { mbar_init(full_bar + 8 * s, 1); mbar_init(empty_bar + 8 * s, 1); }
@@ -665,7 +673,7 @@ tc_grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap mapA0, const __g
     int acc = 0;
     for (int e = 0; e < p.E; ++e) {
       tile_prefix[e] = acc;
-      const int n_e = p.counts[e];
+      const int n_e = s_counts[e];
       const int mt = p.dyn == TC_DYN_M ? (min(n_e, p.M) + 255) / 256 : (p.M + 255) / 256;
       acc += mt * nt;
     }
@@ -693,7 +701,7 @@ tc_grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap mapA0, const __g
       uint32_t phase = 0;
       TileCoord tc;
       bool ok = true;
-      for (int tile = pair; ok && tile_coord_pair(p, tile_prefix, tile, e_cur, N_TILE_COLS, tc); tile += npairs) {
+      for (int tile = pair; ok && tile_coord_pair(p, tile_prefix, s_counts, tile, e_cur, N_TILE_COLS, tc); tile += npairs) {
         const int m0c = tc.m0 + 128 * (int)rank;
         const int32_t* gidx = p.gather_idx + (size_t)tc.e * p.gather_ld;
         int4 rows_a = make_int4(0, 0, 0, 0), rows_b = make_int4(0, 0, 0, 0);
@@ -746,7 +754,7 @@ tc_grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap mapA0, const __g
       bool ok = true;
       const uint32_t a_lbo = A_MN ? TC_BOX_BYTES : 16u, b_lbo = B_MN ? TC_BOX_BYTES : 16u;
       const uint32_t a_kstep = A_MN ? 2048u : 32u, b_kstep = B_MN ? 2048u : 32u;
-      for (int tile = pair; ok && tile_coord_pair(p, tile_prefix, tile, e_cur, N_TILE_COLS, tc); tile += npairs) {
+      for (int tile = pair; ok && tile_coord_pair(p, tile_prefix, s_counts, tile, e_cur, N_TILE_COLS, tc); tile += npairs) {
         if (tc.kblocks == 0) continue;
         if (!mbar_wait_cluster(tempty_bar + 8 * acc_stage, acc_phase ^ 1u, abort_flag)) { ok = false; break; }
         tc_fence_after();
@@ -781,7 +789,7 @@ tc_grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap mapA0, const __g
     uint32_t acc_phase = 0;
     TileCoord tc;
     bool ok = true;
-    for (int tile = pair; ok && tile_coord_pair(p, tile_prefix, tile, e_cur, N_TILE_COLS, tc); tile += npairs) {
+    for (int tile = pair; ok && tile_coord_pair(p, tile_prefix, s_counts, tile, e_cur, N_TILE_COLS, tc); tile += npairs) {
       const int grow = tc.m0 + row_in_tile;
       const bool row_ok = grow < tc.m_lim;
       const int c_beg = half * NCH;
@@ -841,12 +849,13 @@ constexpr int TCW_STAGES = 4;
 constexpr uint32_t TCW_STAGE_BYTES = 6 * TC_BOX_BYTES;       // per CTA: 2 boxes of A, 2 + 2 of B
 constexpr int TCW_LEAD = TCW_STAGES - 1;                     // K blocks half 0 may run ahead of half 1
 
-__device__ __forceinline__ bool tile_coord_wide(const TcParams& p, const int* tile_prefix, int tile, int& e_cur,
+__device__ __forceinline__ bool tile_coord_wide(const TcParams& p, const int* tile_prefix, const int* counts_s,
+    int tile, int& e_cur,
                                                 int n_tile_cols, TileCoord& tc) {
   if (tile >= tile_prefix[p.E]) return false;
   while (tile >= tile_prefix[e_cur + 1]) ++e_cur;
   const int local = tile - tile_prefix[e_cur];
-  const int n_e = p.counts[e_cur];
+  const int n_e = counts_s[e_cur];
   int mt_count;
   if (p.dyn == TC_DYN_M) {
     mt_count = (min(n_e, p.M) + 255) / 256;
@@ -880,6 +889,7 @@ tc_grouped_gemm_pair_wide_kernel(const __grid_constant__ CUtensorMap mapA0, cons
   __shared__ uint32_t tmem_base_slot;
   __shared__ int abort_flag_s;
   __shared__ int tile_prefix[257];
+  __shared__ int s_counts[256];      // the experts' row counts, read from global memory once
 
   volatile int* abort_flag = &abort_flag_s;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -891,6 +901,8 @@ tc_grouped_gemm_pair_wide_kernel(const __grid_constant__ CUtensorMap mapA0, cons
   const uint32_t tfull_bar = smem_u32(&bars[2 * TCW_STAGES]);      // [1]           in each CTA
   const uint32_t tempty_bar = smem_u32(&bars[2 * TCW_STAGES + 1]); // [2]           used in the leader
 
+  for (int e = tid; e < p.E; e += TC_THREADS) s_counts[e] = p.counts[e];
+  __syncthreads();
   if (tid == 0) {
     abort_flag_s = 0;
     for (int s = 0; s < TCW_STAGES; ++s) { mbar_init(full_bar + 8 * s, 1); mbar_init(empty_bar + 8 * s, 1); }
@@ -901,7 +913,7 @@ tc_grouped_gemm_pair_wide_kernel(const __grid_constant__ CUtensorMap mapA0, cons
     int acc = 0;
     for (int e = 0; e < p.E; ++e) {
       tile_prefix[e] = acc;
-      const int n_e = p.counts[e];
+      const int n_e = s_counts[e];
       const int mt = p.dyn == TC_DYN_M ? (min(n_e, p.M) + 255) / 256 : (p.M + 255) / 256;
       acc += mt * nt;
     }
@@ -928,7 +940,7 @@ tc_grouped_gemm_pair_wide_kernel(const __grid_constant__ CUtensorMap mapA0, cons
       uint32_t phase = 0;
       TileCoord tc;
       bool ok = true;
-      for (int tile = pair; ok && tile_coord_wide(p, tile_prefix, tile, e_cur, N_TILE_COLS, tc); tile += npairs) {
+      for (int tile = pair; ok && tile_coord_wide(p, tile_prefix, s_counts, tile, e_cur, N_TILE_COLS, tc); tile += npairs) {
         const int m0c = tc.m0 + 128 * (int)rank;
         const bool two = tc.n0 + N_TILE_COLS < p.N;
         int4 rows_a = make_int4(0, 0, 0, 0);
@@ -988,7 +1000,7 @@ tc_grouped_gemm_pair_wide_kernel(const __grid_constant__ CUtensorMap mapA0, cons
           tc_mma_pair(tmem_base + (uint32_t)(hf * 256), ad, bd, p.idesc, (!first_block || kk > 0) ? 1u : 0u);
         }
       };
-      for (int tile = pair; ok && tile_coord_wide(p, tile_prefix, tile, e_cur, N_TILE_COLS, tc); tile += npairs) {
+      for (int tile = pair; ok && tile_coord_wide(p, tile_prefix, s_counts, tile, e_cur, N_TILE_COLS, tc); tile += npairs) {
         if (tc.kblocks == 0) continue;
         const bool two = tc.n0 + N_TILE_COLS < p.N;
         if (!mbar_wait_cluster(tempty_bar, acc_phase ^ 1u, abort_flag)) { ok = false; break; }
@@ -1032,7 +1044,7 @@ tc_grouped_gemm_pair_wide_kernel(const __grid_constant__ CUtensorMap mapA0, cons
     uint32_t acc_phase = 0;
     TileCoord tc;
     bool ok = true;
-    for (int tile = pair; ok && tile_coord_wide(p, tile_prefix, tile, e_cur, N_TILE_COLS, tc); tile += npairs) {
+    for (int tile = pair; ok && tile_coord_wide(p, tile_prefix, s_counts, tile, e_cur, N_TILE_COLS, tc); tile += npairs) {
       const int grow = tc.m0 + row_in_tile;
       const bool row_ok = grow < tc.m_lim;
       const int c_beg = half * NCH;
