@@ -511,7 +511,7 @@ affinity_fwd_kernel(const T* __restrict__ X, const float* __restrict__ R, float*
 // beta = sum_r dgate_r delta_ti / a^2 over the rows r of token t.  One warp per token.
 // FUSED: dX is not read; the FFN path's gradient is gathered here from dXp (the backward of the
 // token rearrangement, dX[t] = sum of the token's rows of dXp), so dX is written exactly once.
-template <class T, bool FUSED>
+template <class T, bool FUSED, bool DENSE>
 __global__ void __launch_bounds__(256)
 affinity_bwd_dx_kernel(const T* __restrict__ X, const float* __restrict__ R,
                        const float* __restrict__ delta, const float* __restrict__ xnorm,
@@ -536,7 +536,7 @@ affinity_bwd_dx_kernel(const T* __restrict__ X, const float* __restrict__ R,
   for (int j = lane; j < m; j += 32) cz[j] = 0.f;
   float beta = 0.f;
   const float sqD = sqrtf((float)D);
-  if (a != 0.f && ddelta != nullptr) {
+  if (DENSE && a != 0.f) {
     // dense d delta (softmax gate): every expert contributes, in ascending expert order
     for (int i = 0; i < E; ++i) {
       const float b = rnorm[i], dg = ddelta[(size_t)t * E + i];
@@ -546,7 +546,7 @@ affinity_bwd_dx_kernel(const T* __restrict__ X, const float* __restrict__ R,
       for (int j = lane; j < m; j += 32) cz[j] = fmaf(w, R[(size_t)i * m + j], cz[j]);
     }
     beta /= (a * a);
-  } else if (a != 0.f) {
+  } else if (!DENSE && a != 0.f) {
     for (int q = beg; q < end; ++q) {
       const int r = tok_row[q], i = r / C_stride;
       const float b = rnorm[i], dg = dgate[r];
@@ -878,20 +878,20 @@ static etr_status launch_bwd_dx(const etr_config* c, const void* X, const float*
                                 const float* dgate, const float* ddelta, const void* dXp_fused, void* dX,
                                 size_t smem, cudaStream_t st) {
   const int m = c->d / c->D, Cs = c_stride_of(c), grid = ceil_div(c->T, 8);
-  if (dXp_fused) {
-    auto k = affinity_bwd_dx_kernel<T, true>;
+  auto launch = [&](auto k, const char* name) -> etr_status {
     if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
       return ETR_ERR_CUDA;
-    ETR_TIME_BEGIN("affinity_bwd_dx_fused_kernel");
+    ETR_TIME_BEGIN(name);
     k<<<grid, 256, smem, st>>>((const T*)X, R, delta, xnorm, rnorm, rt->tok_ptr, rt->tok_row, dgate, ddelta,
                                (const T*)dXp_fused, (T*)dX, c->T, c->d, c->D, c->E, m, Cs);
+    return ETR_OK;
+  };
+  if (dXp_fused) {
+    if (ddelta) ETR_TRY(launch(affinity_bwd_dx_kernel<T, true, true>, "affinity_bwd_dx_fused_kernel"));
+    else ETR_TRY(launch(affinity_bwd_dx_kernel<T, true, false>, "affinity_bwd_dx_fused_kernel"));
   } else {
-    auto k = affinity_bwd_dx_kernel<T, false>;
-    if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-      return ETR_ERR_CUDA;
-    ETR_TIME_BEGIN("affinity_bwd_dx_kernel");
-    k<<<grid, 256, smem, st>>>((const T*)X, R, delta, xnorm, rnorm, rt->tok_ptr, rt->tok_row, dgate, ddelta,
-                               (const T*)nullptr, (T*)dX, c->T, c->d, c->D, c->E, m, Cs);
+    if (ddelta) ETR_TRY(launch(affinity_bwd_dx_kernel<T, false, true>, "affinity_bwd_dx_kernel"));
+    else ETR_TRY(launch(affinity_bwd_dx_kernel<T, false, false>, "affinity_bwd_dx_kernel"));
   }
   ETR_LAUNCH_CHECK();
   return ETR_OK;
