@@ -1101,6 +1101,46 @@ tc_grouped_gemm_pair_wide_kernel(const __grid_constant__ CUtensorMap mapA0, cons
                 store32_warp_packed(scratch, lane, nvalid, p.out0 + wb + 32 * (c_beg + c), p.ld_out, pk[c]);
           }
         }
+      } else if (EPI == TC_EPI_SWIGLU) {
+        // Fused SwiGLU: G and U of a half are read, H computed, and all three packed to bf16 in
+        // registers before the half is released; the stores follow.
+        static_assert(EPI != TC_EPI_SWIGLU || NCH == 2, "two chunks of 32 gate columns per warp and half");
+        for (int hf = 0; hf < 2; ++hf) {
+          uint32_t pk[NCH][3][16];
+          const int n0h = tc.n0 + hf * N_TILE_COLS;
+          const bool live = hf == 0 || two;
+          if (live) {
+            const uint32_t taddr = tmem_base + (uint32_t)(hf * 256) + ((uint32_t)(32 * q) << 16);
+#pragma unroll
+            for (int c = 0; c < NCH; ++c) {
+              uint32_t r0[32], r1[32];
+              tc_ld32(taddr + 32 * (c_beg + c), r0);
+              tc_ld32(taddr + BN / 2 + 32 * (c_beg + c), r1);
+              tc_wait_ld();
+#pragma unroll
+              for (int i = 0; i < 16; ++i) {
+                const float g0 = __uint_as_float(r0[2 * i]), g1 = __uint_as_float(r0[2 * i + 1]);
+                const float u0 = __uint_as_float(r1[2 * i]), u1 = __uint_as_float(r1[2 * i + 1]);
+                pk[c][0][i] = pack_bf16(g0, g1);
+                pk[c][1][i] = pack_bf16(u0, u1);
+                pk[c][2][i] = pack_bf16(__fdividef(g0, 1.0f + __expf(-g0)) * u0, __fdividef(g1, 1.0f + __expf(-g1)) * u1);
+              }
+            }
+          }
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive_cluster(leader_tempty + 8 * hf);
+          if (live) {
+            const long long wb = obase - (long long)lane * p.ld_out + hf * N_TILE_COLS;
+#pragma unroll
+            for (int c = 0; c < NCH; ++c)
+              if (n0h + 32 * (c_beg + c) < p.N) {
+                store32_warp_packed(scratch, lane, nvalid, p.out0 + wb + 32 * (c_beg + c), p.ld_out, pk[c][0]);
+                store32_warp_packed(scratch, lane, nvalid, p.out2 + wb + 32 * (c_beg + c), p.ld_out, pk[c][2]);
+                store32_warp_packed(scratch, lane, nvalid, p.out1 + wb + 32 * (c_beg + c), p.ld_out, pk[c][1]);
+              }
+          }
+        }
       } else {
         for (int hf = 0; hf < 2; ++hf) {
           if (hf == 0 || two) {
