@@ -1,12 +1,18 @@
 // Grouped GEMMs of the expert FFN on the 5th-generation tensor cores (bf16 in, fp32
-// accumulate in tensor memory).  One persistent, warp-specialised kernel serves all six
-// contractions of the forward and backward pass:
+// accumulate in tensor memory).  One persistent, warp-specialised design serves all six
+// contractions of the forward and backward pass, in three tile forms:
 //
-//   warp 0      TMA producer: 64x64-element boxes (128-byte swizzle) into a 4-stage ring
-//   warp 1      allocates tensor memory, issues tcgen05.mma (128 x 256 x 16 per instruction)
+//   tc_grouped_gemm_kernel            one CTA per 128 x 256 tile (cta_group::1), 4-stage ring
+//   tc_grouped_gemm_pair_kernel       a cluster of two CTAs per 256 x 256 tile (cta_group::2),
+//                                     6-stage ring, two accumulator stages
+//   tc_grouped_gemm_pair_wide_kernel  a cluster of two CTAs per 256 x 512 tile: two accumulators
+//                                     share the A operand, 4-stage ring, halves released separately
+//
+//   warp 0      TMA producer: 64x64-element boxes (128-byte swizzle) into the ring
+//   warp 1      allocates tensor memory, issues tcgen05.mma (the pair's leader CTA only)
 //   warps 2-9   epilogue: tcgen05.ld of the fp32 accumulator, fused SwiGLU / its derivative,
 //               bf16 stores (two warps per 32-lane quarter of tensor memory, half of the
-//               columns each); two accumulator stages so it overlaps the next tile's MMAs
+//               columns each); it overlaps the next tile's MMAs
 //
 // Every operand is fetched as 64x64 boxes of its row-major tensor, so one tensor map per
 // tensor serves both uses of it: "K-major" (the contraction index is contiguous in memory)
