@@ -29,8 +29,9 @@ dispatch_kernel(const T* __restrict__ X, const int32_t* __restrict__ counts,
 }
 
 // Y[t,:] = sum_{r in rows(t)} gate[r] O[r,:]   (gate == nullptr: plain sum, used for dX).
-// One thread per NV groups of 8 consecutive elements of a token, half a row apart, so every
-// row contributes NV independent 16-byte loads per thread.
+// One thread per NV groups of 8 consecutive elements of a token, 1/NV of a row apart, so every
+// row contributes NV independent 16-byte loads per thread (NV = 2 measured best: with 4 the
+// registers limit the kernel to four blocks per SM).
 template <class T, int NV>
 __global__ void __launch_bounds__(256)
 combine_kernel(const T* __restrict__ O, const float* __restrict__ gate,
@@ -111,9 +112,9 @@ static etr_status permute_launch(int which, const etr_config* c, const etr_route
     case 3: {
       const float* g = which == 1 ? rt->gate : nullptr;
       ETR_TIME_BEGIN("combine_kernel");
-      if (c->d % 32 == 0) {
-        const long long n = (long long)c->T * (c->d / 32);
-        combine_kernel<T, 4><<<(unsigned)((n + 255) / 256), 256, 0, st>>>((const T*)a, g, rt->tok_ptr,
+      if (c->d % 16 == 0) {
+        const long long n = (long long)c->T * (c->d / 16);
+        combine_kernel<T, 2><<<(unsigned)((n + 255) / 256), 256, 0, st>>>((const T*)a, g, rt->tok_ptr,
                                                                          rt->tok_row, (T*)out, c->T, c->d);
       } else {
         const long long n = (long long)c->T * (c->d / 8);
