@@ -29,37 +29,80 @@ dispatch_kernel(const T* __restrict__ X, const int32_t* __restrict__ counts,
 }
 
 // Y[t,:] = sum_{r in rows(t)} gate[r] O[r,:]   (gate == nullptr: plain sum, used for dX).
-// One thread per NV groups of 8 consecutive elements of a token, 1/NV of a row apart, so every
-// row contributes NV independent 16-byte loads per thread (NV = 2 measured best: with 4 the
-// registers limit the kernel to four blocks per SM).
+// A block takes COMBINE_TOKENS consecutive tokens.  It first copies their row lists and gates to
+// shared memory (two rounds of dependent loads for the whole chunk instead of two per token), then
+// every thread owns NV groups of 8 consecutive elements of a token, 1/NV of a row apart, and walks
+// the token's rows two at a time: 2 NV independent 16-byte loads in flight per thread, none of them
+// waiting for an index.  Rows are added in list order (the result does not depend on the chunking).
+constexpr int COMBINE_TOKENS = 8;
+constexpr int COMBINE_ROWS = 512;     // row entries held in shared memory; later ones are read in place
+
 template <class T, int NV>
 __global__ void __launch_bounds__(256)
 combine_kernel(const T* __restrict__ O, const float* __restrict__ gate,
                const int32_t* __restrict__ tok_ptr, const int32_t* __restrict__ tok_row,
                T* __restrict__ Y, int Ttok, int d) {
+  __shared__ int s_ptr[COMBINE_TOKENS + 1];
+  __shared__ int s_row[COMBINE_ROWS];
+  __shared__ float s_gate[COMBINE_ROWS];
+  const int tid = threadIdx.x;
+  const int t0 = blockIdx.x * COMBINE_TOKENS;
+  const int nt = min(COMBINE_TOKENS, Ttok - t0);
+  if (tid <= nt) s_ptr[tid] = tok_ptr[t0 + tid];
+  __syncthreads();
+  const int base = s_ptr[0];
+  const int staged = min(s_ptr[nt] - base, COMBINE_ROWS);
+  for (int i = tid; i < staged; i += 256) {
+    const int r = tok_row[base + i];
+    s_row[i] = r;
+    s_gate[i] = gate ? gate[r] : 1.0f;
+  }
+  __syncthreads();
+  auto entry = [&](int q, int& r, float& g) {
+    if (q < COMBINE_ROWS) { r = s_row[q]; g = s_gate[q]; }
+    else { r = tok_row[base + q]; g = gate ? gate[r] : 1.0f; }
+  };
   const int vpt = d / 8 / NV;                       // threads per token
-  const long long idx = (long long)blockIdx.x * 256 + threadIdx.x;
-  if (idx >= (long long)Ttok * vpt) return;
-  const int t = (int)(idx / vpt), v = (int)(idx - (long long)t * vpt);
-  float acc[NV][8];
-#pragma unroll
-  for (int u = 0; u < NV; ++u)
-#pragma unroll
-    for (int e = 0; e < 8; ++e) acc[u][e] = 0.f;
-  const int beg = tok_ptr[t], end = tok_ptr[t + 1];
-  for (int q = beg; q < end; ++q) {
-    const int r = tok_row[q];
-    const float g = gate ? gate[r] : 1.0f;
-    Vec8<T> o[NV];
-#pragma unroll
-    for (int u = 0; u < NV; ++u) o[u] = Vec8<T>::load(O + (size_t)r * d + (size_t)(v + u * vpt) * 8);
+  for (int w = tid; w < nt * vpt; w += 256) {
+    const int tl = w / vpt, v = w - tl * vpt;
+    const int end = s_ptr[tl + 1] - base;
+    float acc[NV][8];
 #pragma unroll
     for (int u = 0; u < NV; ++u)
 #pragma unroll
-      for (int e = 0; e < 8; ++e) acc[u][e] = fmaf(g, o[u].v[e], acc[u][e]);
-  }
+      for (int e = 0; e < 8; ++e) acc[u][e] = 0.f;
+    int q = s_ptr[tl] - base;
+    for (; q + 2 <= end; q += 2) {
+      int r0, r1;
+      float g0, g1;
+      entry(q, r0, g0);
+      entry(q + 1, r1, g1);
+      Vec8<T> o0[NV], o1[NV];
 #pragma unroll
-  for (int u = 0; u < NV; ++u) Vec8<T>::store(Y + (size_t)t * d + (size_t)(v + u * vpt) * 8, acc[u]);
+      for (int u = 0; u < NV; ++u) o0[u] = Vec8<T>::load(O + (size_t)r0 * d + (size_t)(v + u * vpt) * 8);
+#pragma unroll
+      for (int u = 0; u < NV; ++u) o1[u] = Vec8<T>::load(O + (size_t)r1 * d + (size_t)(v + u * vpt) * 8);
+#pragma unroll
+      for (int u = 0; u < NV; ++u)
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc[u][e] = fmaf(g1, o1[u].v[e], fmaf(g0, o0[u].v[e], acc[u][e]));
+    }
+    if (q < end) {
+      int r;
+      float g;
+      entry(q, r, g);
+      Vec8<T> o[NV];
+#pragma unroll
+      for (int u = 0; u < NV; ++u) o[u] = Vec8<T>::load(O + (size_t)r * d + (size_t)(v + u * vpt) * 8);
+#pragma unroll
+      for (int u = 0; u < NV; ++u)
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc[u][e] = fmaf(g, o[u].v[e], acc[u][e]);
+    }
+#pragma unroll
+    for (int u = 0; u < NV; ++u)
+      Vec8<T>::store(Y + (size_t)(t0 + tl) * d + (size_t)(v + u * vpt) * 8, acc[u]);
+  }
 }
 
 // dO[r,:] = gate[r] dY[t(r),:], dgate[r] = <dY[t(r),:], O[r,:]>; pad rows zero.  Warp per row.
@@ -112,15 +155,11 @@ static etr_status permute_launch(int which, const etr_config* c, const etr_route
     case 3: {
       const float* g = which == 1 ? rt->gate : nullptr;
       ETR_TIME_BEGIN("combine_kernel");
-      if (c->d % 16 == 0) {
-        const long long n = (long long)c->T * (c->d / 16);
-        combine_kernel<T, 2><<<(unsigned)((n + 255) / 256), 256, 0, st>>>((const T*)a, g, rt->tok_ptr,
-                                                                         rt->tok_row, (T*)out, c->T, c->d);
-      } else {
-        const long long n = (long long)c->T * (c->d / 8);
-        combine_kernel<T, 1><<<(unsigned)((n + 255) / 256), 256, 0, st>>>((const T*)a, g, rt->tok_ptr,
-                                                                         rt->tok_row, (T*)out, c->T, c->d);
-      }
+      const unsigned grid = (unsigned)ceil_div(c->T, COMBINE_TOKENS);
+      if (c->d % 16 == 0)
+        combine_kernel<T, 2><<<grid, 256, 0, st>>>((const T*)a, g, rt->tok_ptr, rt->tok_row, (T*)out, c->T, c->d);
+      else
+        combine_kernel<T, 1><<<grid, 256, 0, st>>>((const T*)a, g, rt->tok_ptr, rt->tok_row, (T*)out, c->T, c->d);
       break;
     }
     case 2:
