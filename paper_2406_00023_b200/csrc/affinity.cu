@@ -582,6 +582,154 @@ affinity_bwd_dx_kernel(const T* __restrict__ X, const float* __restrict__ R,
   }
 }
 
+// The fused form for selected pairs (the default of the layer backward), by chunks of tokens.  A block
+// takes `tpb` consecutive tokens: (1) all threads copy the chunk's row lists to shared memory together
+// with the per-row scalars (expert, weight of R_i in cz, dgate, delta), so the dependent chain
+// pointer -> row -> scalars is walked once per chunk and not once per token; (2) cz[tl][:] and
+// beta[tl] of every routed token of the chunk go to shared memory, one thread per pooled column,
+// rows in list order; (3) the streaming pass: every thread owns NV groups of 8 elements of a token,
+// 1/NV of a row apart, loads x and the token's rows of dXp two rows at a time (no load waits for an
+// index) and writes dX once.  Unrouted tokens get zeros without reading X.  Same arithmetic, in the
+// same order, as affinity_bwd_dx_kernel<T, true, false>: the results are bit-identical.
+constexpr int DXC_MAX_TOKENS = 16;
+constexpr int DXC_ROWS = 512;          // row entries held in shared memory; later ones are read in place
+
+template <class T, int NV, bool GROUP8>
+__global__ void __launch_bounds__(256, 4)
+affinity_bwd_dx_chunk_kernel(const T* __restrict__ X, const float* __restrict__ R,
+                             const float* __restrict__ delta, const float* __restrict__ xnorm,
+                             const float* __restrict__ rnorm, const int32_t* __restrict__ tok_ptr,
+                             const int32_t* __restrict__ tok_row, const float* __restrict__ dgate,
+                             const T* __restrict__ dXp, T* __restrict__ dX,
+                             int Ttok, int d, int D, int E, int m, int C_stride, int tpb, int d_shift) {
+  extern __shared__ __align__(16) float cz[];      // [tpb][m]
+  __shared__ int s_ptr[DXC_MAX_TOKENS + 1];
+  __shared__ int s_row[DXC_ROWS];
+  __shared__ int s_exp[DXC_ROWS];                  // expert of the entry, -1 if ||R_i|| = 0
+  __shared__ float s_w[DXC_ROWS];
+  __shared__ float s_dg[DXC_ROWS];
+  __shared__ float s_dl[DXC_ROWS];
+  __shared__ float s_a[DXC_MAX_TOKENS];
+  __shared__ float s_beta[DXC_MAX_TOKENS];
+  const int tid = threadIdx.x;
+  const int t0 = blockIdx.x * tpb;
+  const int nt = min(tpb, Ttok - t0);
+  if (tid <= nt) s_ptr[tid] = tok_ptr[t0 + tid];
+  if (tid < nt) s_a[tid] = xnorm[t0 + tid];
+  __syncthreads();
+  const int base = s_ptr[0];
+  const int staged = min(s_ptr[nt] - base, DXC_ROWS);
+  const float sqD = sqrtf((float)D);
+  for (int e = tid; e < staged; e += 256) {
+    const int r = tok_row[base + e];
+    int tl = 0;
+    while (s_ptr[tl + 1] - base <= e) ++tl;        // the entry's token (at most tpb steps)
+    const int i = r / C_stride;
+    const float a = s_a[tl], b = rnorm[i], dg = dgate[r];
+    s_row[e] = r;
+    s_exp[e] = b == 0.f ? -1 : i;
+    s_dg[e] = dg;
+    s_dl[e] = delta[(size_t)(t0 + tl) * E + i];
+    s_w[e] = dg * sqD / (a * b) / (float)D;
+  }
+  __syncthreads();
+  for (int it = tid; it < nt * m; it += 256) {
+    const int tl = it / m, j = it - tl * m;
+    const int beg = s_ptr[tl] - base, end = s_ptr[tl + 1] - base;
+    if (beg == end) continue;
+    const float a = s_a[tl];
+    float acc = 0.f, beta = 0.f;
+    if (a != 0.f) {
+      for (int q = beg; q < end; ++q) {
+        int i;
+        float w, dg, dl;
+        if (q < DXC_ROWS) {
+          i = s_exp[q]; w = s_w[q]; dg = s_dg[q]; dl = s_dl[q];
+        } else {
+          const int r = tok_row[base + q];
+          i = r / C_stride;
+          const float b = rnorm[i];
+          dg = dgate[r];
+          dl = delta[(size_t)(t0 + tl) * E + i];
+          w = dg * sqD / (a * b) / (float)D;
+          if (b == 0.f) i = -1;
+        }
+        if (i < 0) continue;
+        beta = fmaf(dg, dl, beta);
+        acc = fmaf(w, R[(size_t)i * m + j], acc);
+      }
+      beta /= (a * a);
+    }
+    cz[it] = acc;
+    if (j == 0) s_beta[tl] = beta;
+  }
+  __syncthreads();
+  const int vpt = d / 8 / NV;                      // threads per token
+  for (int wi = tid; wi < nt * vpt; wi += 256) {
+    const int tl = wi / vpt, v = wi - tl * vpt;
+    const int beg = s_ptr[tl] - base, end = s_ptr[tl + 1] - base;
+    T* g = dX + (size_t)(t0 + tl) * d;
+    float bs[NV][8];
+#pragma unroll
+    for (int u = 0; u < NV; ++u)
+#pragma unroll
+      for (int e = 0; e < 8; ++e) bs[u][e] = 0.f;
+    if (beg == end) {
+#pragma unroll
+      for (int u = 0; u < NV; ++u) Vec8<T>::store(g + (size_t)(v + u * vpt) * 8, bs[u]);
+      continue;
+    }
+    const T* x = X + (size_t)(t0 + tl) * d;
+    Vec8<T> xv[NV];
+#pragma unroll
+    for (int u = 0; u < NV; ++u) xv[u] = Vec8<T>::load(x + (size_t)(v + u * vpt) * 8);
+    int q = beg;
+    for (; q + 2 <= end; q += 2) {
+      const int r0 = q < DXC_ROWS ? s_row[q] : tok_row[base + q];
+      const int r1 = q + 1 < DXC_ROWS ? s_row[q + 1] : tok_row[base + q + 1];
+      Vec8<T> v0[NV], v1[NV];
+#pragma unroll
+      for (int u = 0; u < NV; ++u) v0[u] = Vec8<T>::load(dXp + (size_t)r0 * d + (size_t)(v + u * vpt) * 8);
+#pragma unroll
+      for (int u = 0; u < NV; ++u) v1[u] = Vec8<T>::load(dXp + (size_t)r1 * d + (size_t)(v + u * vpt) * 8);
+#pragma unroll
+      for (int u = 0; u < NV; ++u)
+#pragma unroll
+        for (int e = 0; e < 8; ++e) bs[u][e] = (bs[u][e] + v0[u].v[e]) + v1[u].v[e];
+    }
+    if (q < end) {
+      const int r = q < DXC_ROWS ? s_row[q] : tok_row[base + q];
+      Vec8<T> v0[NV];
+#pragma unroll
+      for (int u = 0; u < NV; ++u) v0[u] = Vec8<T>::load(dXp + (size_t)r * d + (size_t)(v + u * vpt) * 8);
+#pragma unroll
+      for (int u = 0; u < NV; ++u)
+#pragma unroll
+        for (int e = 0; e < 8; ++e) bs[u][e] += v0[u].v[e];
+    }
+    const float beta = s_beta[tl];
+    const float* czt = cz + (size_t)tl * m;
+#pragma unroll
+    for (int u = 0; u < NV; ++u) {
+      const int c0 = (v + u * vpt) * 8;
+      float out[8];
+      if (GROUP8) {                                // D = 2^d_shift >= 8: the 8 elements share one group
+        const float czv = czt[c0 >> d_shift];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) out[e] = bs[u][e] + (czv - beta * xv[u].v[e]);
+      } else {
+        int gi = c0 / D, rem = c0 - gi * D;        // group of the first element, then stepped
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          out[e] = bs[u][e] + (czt[gi] - beta * xv[u].v[e]);
+          if (++rem == D) { rem = 0; ++gi; }
+        }
+      }
+      Vec8<T>::store(g + (size_t)c0, out);
+    }
+  }
+}
+
 // Partial dR over chunks of 128 slots of one expert (fixed order inside a chunk):
 //   part[i][ch][j] = sum_p w_p Z[t_p][j], w_p = dgate_p sqrt(D)/(a_t b_i);
 //   part[i][ch][m] = sum_p dgate_p delta_ti
@@ -886,7 +1034,28 @@ static etr_status launch_bwd_dx(const etr_config* c, const void* X, const float*
                                (const T*)dXp_fused, (T*)dX, c->T, c->d, c->D, c->E, m, Cs);
     return ETR_OK;
   };
-  if (dXp_fused) {
+  // chunked form of the fused kernel: as many tokens per block as keep cz within 48 KiB (at most 16)
+  int tpb = DXC_MAX_TOKENS;
+  while (tpb > 2 && (size_t)tpb * m * sizeof(float) > 48 * 1024) tpb /= 2;
+  if (dXp_fused && !ddelta && (size_t)tpb * m * sizeof(float) <= 48 * 1024) {
+    const size_t csm = (size_t)tpb * m * sizeof(float);
+    ETR_TIME_BEGIN("affinity_bwd_dx_fused_kernel");
+    int d_shift = 0;
+    while ((1 << d_shift) < c->D) ++d_shift;
+    const bool group8 = c->D >= 8 && (1 << d_shift) == c->D;
+    auto go = [&](auto k) {
+      k<<<ceil_div(c->T, tpb), 256, csm, st>>>((const T*)X, R, delta, xnorm, rnorm, rt->tok_ptr, rt->tok_row, dgate,
+                                               (const T*)dXp_fused, (T*)dX, c->T, c->d, c->D, c->E, m, Cs, tpb,
+                                               d_shift);
+    };
+    if (c->d % 16 == 0) {
+      if (group8) go(affinity_bwd_dx_chunk_kernel<T, 2, true>);
+      else go(affinity_bwd_dx_chunk_kernel<T, 2, false>);
+    } else {
+      if (group8) go(affinity_bwd_dx_chunk_kernel<T, 1, true>);
+      else go(affinity_bwd_dx_chunk_kernel<T, 1, false>);
+    }
+  } else if (dXp_fused) {
     if (ddelta) ETR_TRY(launch(affinity_bwd_dx_kernel<T, true, true>, "affinity_bwd_dx_fused_kernel"));
     else ETR_TRY(launch(affinity_bwd_dx_kernel<T, true, false>, "affinity_bwd_dx_fused_kernel"));
   } else {
