@@ -1,6 +1,6 @@
 """Edge cases of the CUDA path against the oracle: experts that receive no token, Top-1
-routing (the paper's efficiency runs), k = E, capacity 1, a handful of tokens, and group
-sizes that take the generic pooling path."""
+routing (the paper's efficiency runs), k = E, capacity 1, a handful of tokens, group
+sizes that take the generic pooling path, and tokens with more rows than the gather kernels stage."""
 import numpy as np
 import pytest
 import torch
@@ -93,6 +93,18 @@ def test_group_sizes(D, dtype):
     d = 768 if D == 24 else 512
     w = gw.scaled(W["small"], T=200, d=d, D=D, E=8, h=64, dtype=dtype)
     layer_vs_oracle(w, gw.make_inputs(w), ob.MODE_TCR)
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_tokens_kept_by_every_expert_overflow_the_staged_row_lists(dtype):
+    """Expert choice with C = T and 128 experts: every token has 128 rows, so the chunks of 8
+    (combine) and 16 (fused dX) consecutive tokens hold 1024 and 2048 row entries, more than the
+    512 those kernels stage in shared memory: the entries beyond are read in place.  T = 40 also
+    leaves a ragged last chunk in both."""
+    w = gw.scaled(W["small"], T=40, d=1024, D=8, E=128, h=64, cf=64.0, dtype=dtype)
+    assert w.capacity == w.T
+    fw, got, out = layer_vs_oracle(w, gw.make_inputs(w), ob.MODE_ECR)
+    assert np.all(np.diff(got.tok_ptr) == w.E)
 
 
 def test_sweep_modes_follow_the_step():
