@@ -283,6 +283,132 @@ affinity_score_kernel(const float* __restrict__ Z, const float* __restrict__ xno
   }
 }
 
+// Kernel 2, tiled form (E <= 64, m a multiple of 32): the same products as affinity_score_kernel, in
+// the same order per (token, expert), laid out like a register-tiled fp32 GEMM.  A block of 8 warps
+// takes tiles of 256 tokens; a lane is (token group tg = lane / 8, expert group eg = lane % 8) and
+// owns 8 tokens (rows 4 u + tg of the warp's 32) x EPT experts (e 8 + eg): 8 EPT accumulators fed by
+// 8 + EPT 16-byte shared-memory loads per 4 k, every one of them a single wavefront (4 consecutive
+// token rows, 8 consecutive expert rows; both row strides are 4 banks modulo 32).  The pooled rows
+// arrive 32 columns at a time by asynchronous 16-byte copies into two buffers: the copy of a stage
+// runs under the products of the one before, one block barrier per stage.
+constexpr int SC_TM = 256;            // tokens per tile
+constexpr int SC_KC = 16;             // pooled columns per stage
+constexpr int SC_ZLD = SC_KC + 4;     // row stride of a stage buffer, in floats
+
+template <int EPT>
+__global__ void __launch_bounds__(256, 2)
+affinity_score_tile_kernel(const float* __restrict__ Z, const float* __restrict__ xnorm,
+                           const float* __restrict__ R, float* __restrict__ delta,
+                           float* __restrict__ rnorm, etr_stats* stats, int Ttok, int D, int E, int m,
+                           int ldm) {
+  extern __shared__ __align__(16) float smem[];
+  constexpr int EROWS = 8 * EPT;
+  float* Rs = smem;                               // [EROWS][ldm]
+  float* rn = Rs + (size_t)EROWS * ldm;           // [EROWS]
+  float* Zs = rn + EROWS;                         // [2][SC_TM][SC_ZLD]
+  __shared__ uint32_t red[8];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int eg = lane & 7, tg = lane >> 3;
+
+  for (int idx = tid; idx < EROWS * ldm; idx += 256) {
+    const int i = idx / ldm, j = idx - i * ldm;
+    Rs[idx] = (i < E && j < m) ? R[(size_t)i * m + j] : 0.f;
+  }
+  __syncthreads();
+  for (int i = warp; i < EROWS; i += 8) {
+    float q = 0.f;
+    for (int j = lane; j < m; j += 32) q += Rs[i * ldm + j] * Rs[i * ldm + j];
+    q = warp_sum(q);
+    if (lane == 0) {
+      rn[i] = sqrtf(q);
+      if (blockIdx.x == 0 && i < E) rnorm[i] = rn[i];
+    }
+  }
+  // (the first stage barrier below also orders rn before its first use)
+
+  const int ntiles = (Ttok + SC_TM - 1) / SC_TM, nk = m / SC_KC;
+  auto fetch = [&](int tile, int chunk, int buf) {
+    float* dst0 = Zs + (size_t)buf * SC_TM * SC_ZLD;
+#pragma unroll
+    for (int q = 0; q < SC_TM * (SC_KC / 4) / 256; ++q) {
+      const int idx = tid + 256 * q, row = idx / (SC_KC / 4), c4 = idx % (SC_KC / 4);
+      const int t = tile * SC_TM + row;
+      float* dst = dst0 + row * SC_ZLD + c4 * 4;
+      if (t < Ttok) {
+        const uint32_t sa = (uint32_t)__cvta_generic_to_shared(dst);
+        const float* src = Z + (size_t)t * m + chunk * SC_KC + c4 * 4;
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(sa), "l"(src) : "memory");
+      } else {
+        *reinterpret_cast<float4*>(dst) = make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  };
+
+  const float sqD = sqrtf((float)D);
+  const int rs4 = ldm / 4;
+  const float4* r4 = reinterpret_cast<const float4*>(Rs) + (size_t)eg * rs4;
+  float best = -INFINITY;
+  int stage = 0;
+  if ((int)blockIdx.x < ntiles) fetch(blockIdx.x, 0, 0);
+  for (int tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+    float acc[8][EPT];
+#pragma unroll
+    for (int u = 0; u < 8; ++u)
+#pragma unroll
+      for (int e = 0; e < EPT; ++e) acc[u][e] = 0.f;
+    for (int chunk = 0; chunk < nk; ++chunk, ++stage) {
+      asm volatile("cp.async.wait_group 0;" ::: "memory");
+      __syncthreads();             // this stage has landed; everyone is done with the other buffer
+      if (chunk + 1 < nk) fetch(tile, chunk + 1, (stage + 1) & 1);
+      else if (tile + (int)gridDim.x < ntiles) fetch(tile + gridDim.x, 0, (stage + 1) & 1);
+      const float4* z4 = reinterpret_cast<const float4*>(Zs + (size_t)(stage & 1) * SC_TM * SC_ZLD) +
+                         (size_t)(warp * 32 + tg) * (SC_ZLD / 4);
+      const float4* rc = r4 + chunk * (SC_KC / 4);
+#pragma unroll 1
+      for (int j = 0; j < SC_KC / 4; ++j) {
+        float4 r[EPT];
+#pragma unroll
+        for (int e = 0; e < EPT; ++e) r[e] = rc[(size_t)(8 * e) * rs4 + j];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          const float4 z = z4[(size_t)(4 * u) * (SC_ZLD / 4) + j];
+#pragma unroll
+          for (int e = 0; e < EPT; ++e) {
+            acc[u][e] = fmaf(z.x, r[e].x, acc[u][e]); acc[u][e] = fmaf(z.y, r[e].y, acc[u][e]);
+            acc[u][e] = fmaf(z.z, r[e].z, acc[u][e]); acc[u][e] = fmaf(z.w, r[e].w, acc[u][e]);
+          }
+        }
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int t = tile * SC_TM + warp * 32 + 4 * u + tg;
+      if (t >= Ttok) continue;
+      const float a = xnorm[t];
+#pragma unroll
+      for (int e = 0; e < EPT; ++e) {
+        const int i = 8 * e + eg;
+        if (i < E) {
+          const float den = a * rn[i];
+          const float v = den == 0.f ? 0.f : sqD * acc[u][e] / den;
+          delta[(size_t)t * E + i] = v;
+          best = fmaxf(best, v);
+        }
+      }
+    }
+  }
+  uint32_t key = best == -INFINITY ? 0u : ordered_key(best);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) key = max(key, __shfl_xor_sync(0xffffffffu, key, o));
+  if (lane == 0) red[warp] = key;
+  __syncthreads();
+  if (tid == 0) {
+    for (int w = 1; w < 8; ++w) key = max(key, red[w]);
+    if (key) atomicMax(&stats->delta_max_key, key);
+  }
+}
+
 // ---- forward, warp-autonomous persistent form (the default) ------------------------------------
 // R stays in shared memory for the life of the CTA; every warp owns a private slice for the
 // pooled rows of TPG tokens and loops on its own: pool TPG tokens (16-byte loads, one pass
@@ -959,6 +1085,25 @@ static etr_status launch_score(const etr_config* c, const float* Z, const float*
   return ETR_OK;
 }
 
+// tiled score kernel: *done is false when the shape is not one it takes
+template <int EPT>
+static etr_status launch_score_tile(const etr_config* c, const float* Z, const float* xnorm, const float* R,
+                                    float* delta, float* rnorm, etr_stats* stats, cudaStream_t st, bool* done) {
+  const int m = c->d / c->D, ldm = m + 4;
+  *done = false;
+  const size_t smem = ((size_t)8 * EPT * ldm + 8 * EPT + (size_t)2 * SC_TM * SC_ZLD) * sizeof(float);
+  if (smem > 110 * 1024) return ETR_OK;          // two blocks per SM
+  auto k = affinity_score_tile_kernel<EPT>;
+  if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+    return ETR_ERR_CUDA;
+  const int grid = std::min(2 * device_sm_count(), ceil_div(c->T, SC_TM));
+  ETR_TIME_BEGIN("affinity_score_kernel");
+  k<<<grid, 256, smem, st>>>(Z, xnorm, R, delta, rnorm, stats, c->T, c->D, c->E, m, ldm);
+  ETR_LAUNCH_CHECK();
+  *done = true;
+  return ETR_OK;
+}
+
 // pool + score as two kernels; *done is false if the score kernel's shared memory does not fit
 static etr_status affinity_forward_split(const etr_config* c, const void* X, const float* R, float* delta,
                                          float* Z, float* xnorm, float* rnorm, etr_stats* stats,
@@ -970,6 +1115,12 @@ static etr_status affinity_forward_split(const etr_config* c, const void* X, con
   if (((size_t)(32 * EPL + 4 * TPG) * ldm + 32 * EPL) * sizeof(float) > 220 * 1024) return ETR_OK;
   if (c->dtype == ETR_BF16) ETR_TRY(launch_pool<__nv_bfloat16>(c, X, Z, xnorm, st));
   else ETR_TRY(launch_pool<float>(c, X, Z, xnorm, st));
+  if (c->E <= 64 && m % SC_KC == 0) {
+    if (c->E <= 16) ETR_TRY(launch_score_tile<2>(c, Z, xnorm, R, delta, rnorm, stats, st, done));
+    else if (c->E <= 32) ETR_TRY(launch_score_tile<4>(c, Z, xnorm, R, delta, rnorm, stats, st, done));
+    else ETR_TRY(launch_score_tile<8>(c, Z, xnorm, R, delta, rnorm, stats, st, done));
+    if (*done) return ETR_OK;
+  }
   if (EPL == 1) return launch_score<1, 8>(c, Z, xnorm, R, delta, rnorm, stats, st, done);
   if (EPL == 2) return launch_score<2, 8>(c, Z, xnorm, R, delta, rnorm, stats, st, done);
   if (EPL == 4) return launch_score<4, 4>(c, Z, xnorm, R, delta, rnorm, stats, st, done);
