@@ -1115,7 +1115,8 @@ static etr_status affinity_forward_split(const etr_config* c, const void* X, con
   if (((size_t)(32 * EPL + 4 * TPG) * ldm + 32 * EPL) * sizeof(float) > 220 * 1024) return ETR_OK;
   if (c->dtype == ETR_BF16) ETR_TRY(launch_pool<__nv_bfloat16>(c, X, Z, xnorm, st));
   else ETR_TRY(launch_pool<float>(c, X, Z, xnorm, st));
-  if (c->E <= 64 && m % SC_KC == 0) {
+  // the tiled form needs a tile of 256 tokens for every SM to pay for its set-up (R and its norms per block)
+  if (c->E <= 64 && m % SC_KC == 0 && ceil_div(c->T, SC_TM) >= device_sm_count()) {
     if (c->E <= 16) ETR_TRY(launch_score_tile<2>(c, Z, xnorm, R, delta, rnorm, stats, st, done));
     else if (c->E <= 32) ETR_TRY(launch_score_tile<4>(c, Z, xnorm, R, delta, rnorm, stats, st, done));
     else ETR_TRY(launch_score_tile<8>(c, Z, xnorm, R, delta, rnorm, stats, st, done));

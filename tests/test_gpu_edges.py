@@ -107,6 +107,31 @@ def test_tokens_kept_by_every_expert_overflow_the_staged_row_lists(dtype):
     assert np.all(np.diff(got.tok_ptr) == w.E)
 
 
+@pytest.mark.parametrize("E,dtype", [(16, "bf16"), (32, "f32"), (64, "bf16")])
+def test_affinity_with_a_score_tile_for_every_sm(E, dtype):
+    """38100 tokens: at least one 256-token tile per SM, which is when the score kernel takes its
+    register-tiled form (2, 4 or 8 experts per lane for E <= 16, 32, 64), and a ragged last tile."""
+    w = gw.scaled(W["small"], T=38100, d=512, D=8, E=E, h=64, dtype=dtype)
+    inp = gw.make_inputs(w, weights=False)
+    delta_ref, *_ = ob.Oracle("f32").affinity(inp["X"], inp["R"], w.D)
+    cfg = hz.make_cfg(w)
+    X = hz.to_dev(inp["X"], w)
+    R = torch.from_numpy(inp["R"]).cuda()
+    T, m = w.T, w.d // w.D
+    delta = torch.empty(T, E, dtype=torch.float32, device="cuda")
+    Z = torch.empty(T, m, dtype=torch.float32, device="cuda")
+    xnorm = torch.empty(T, dtype=torch.float32, device="cuda")
+    rnorm = torch.empty(E, dtype=torch.float32, device="cuda")
+    stats = torch.zeros(16, dtype=torch.int32, device="cuda")
+    etr.affinity(cfg, X, R, delta, Z, xnorm, rnorm, stats)
+    torch.cuda.synchronize()
+    got = hz.to_np(delta)
+    hz.assert_affinity_close(got, delta_ref)
+    u = int(np.float32(got.max()).view(np.uint32))
+    key = (~u & 0xffffffff) if (u & 0x80000000) else (u | 0x80000000)
+    assert int(stats[5].item()) & 0xffffffff == key
+
+
 def test_sweep_modes_follow_the_step():
     """ETR_MODE_AUTO picks token choice before switch_step and expert choice from it on."""
     for step, want in ((999, etr.MODE_TCR), (1000, etr.MODE_ECR)):
