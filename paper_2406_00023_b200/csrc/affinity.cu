@@ -1,13 +1,23 @@
 // GrAP pooling + cosine affinity (forward) and the router gradient (backward).
 //
-// Forward, one CTA per tile of TB tokens:
-//   phase 0  R -> shared memory (rows padded so 128-bit reads of 8 different rows hit
-//            32 different banks), ||R_i|| by one warp per row
-//   phase 1  each warp streams its tokens' rows of X once with 16-byte loads, pools the
-//            D-groups in registers, accumulates ||x||^2, leaves z_t in shared memory
-//   phase 2  s = Z R^T register-tiled (2 tokens x 4 experts per thread, float4 operands),
-//            delta = sqrt(D) s / (||x|| ||R||), batch max through one atomicMax on the
-//            order-preserving integer image (exact and order independent)
+// Forward, in the order the host code tries them:
+//   split form (the caller keeps Z, which the backward pass needs anyway):
+//     grap_pool_kernel             one streaming pass over X: pooled rows Z and ||x_t||
+//     affinity_score_tile_kernel   s = Z R^T as a register-tiled fp32 GEMM, cosine, batch max
+//                                  (E <= 64, 16 | m, a 256-token tile for every SM)
+//     affinity_score_kernel        the same products with lane = expert, 8 tokens per warp
+//   affinity_fwd_warp_kernel       one pass, pooling and score per warp (no Z kept)
+//   affinity_fwd_kernel            one CTA per tile of AFF_TB tokens (shapes the others do not take):
+//     phase 0  R -> shared memory (rows padded so 128-bit reads of 8 different rows hit
+//              32 different banks), ||R_i|| by one warp per row
+//     phase 1  each warp streams its tokens' rows of X once with 16-byte loads, pools the
+//              D-groups in registers, accumulates ||x||^2, leaves z_t in shared memory
+//     phase 2  s = Z R^T register-tiled (2 tokens x 4 experts per thread, float4 operands),
+//              delta = sqrt(D) s / (||x|| ||R||), batch max through one atomicMax on the
+//              order-preserving integer image (exact and order independent)
+// Backward: affinity_bwd_dx_chunk_kernel (dX with the dispatch backward fused in, by chunks of
+// tokens), affinity_bwd_dx_kernel (stage form, dense d delta, shapes the chunked form does not take),
+// affinity_bwd_dr_*_kernel (dR in two fixed-order stages).
 #include <algorithm>
 
 #include "common.cuh"
