@@ -78,7 +78,7 @@ def algorithmic_work(w, rows, kernel, unrouted=0):
         "affinity_fwd_kernel": (T * d * b + T * E * 4 + T * m * 4 + T * 4, "bytes"),
         "affinity_fwd_warp_kernel": (T * d * b + T * E * 4 + T * m * 4 + T * 4, "bytes"),
         "grap_pool_kernel": (T * d * b + T * m * 4 + T * 4, "bytes"),
-        "affinity_score_kernel": (T * m * 4 + T * E * 4, "bytes"),
+        "affinity_score_kernel": (2 * T * m * E, "fp32_flops"),        # the product z R^T: fp32 FMA issue, not HBM
         "select_token_side_kernel": (2 * T * E * 4, "bytes"),
         "select_expert_side_kernel": (T * E * 4 + rows * 8, "bytes"),
         "csr_count_kernel": (T * E * 4, "bytes"),
@@ -376,6 +376,11 @@ def main():
         avg_ms = ms / n
         if kind == "flops":
             ach, peak, unit, bound = per_launch / (avg_ms * 1e-3) / 1e12, peaks["bf16_tflops_sustained"], "TFLOP/s", "tensor"
+        elif kind == "fp32_flops":
+            # plain fp32 multiply-adds: SMs x 128 lanes x 2 flop at the maximum SM clock (nominal, not measured)
+            sms = torch.cuda.get_device_properties(dev).multi_processor_count
+            peak = sms * 128 * 2 * (clocks.get("sm_max_mhz") or 1965.0) * 1e6 / 1e12
+            ach, unit, bound = per_launch / (avg_ms * 1e-3) / 1e12, "TFLOP/s", "alu"
         else:
             ach, peak, unit, bound = per_launch / (avg_ms * 1e-3) / 1e9, peaks["hbm_gbs"], "GB/s", "hbm"
         kernels.append({"kernel": name, "launches_per_step": n / args.steps, "ms_per_step": ms / args.steps,
