@@ -91,36 +91,153 @@ def assert_affinity_close(got, ref, what="delta"):
 
 BF16_HALF_ULP = 2.0 ** -8     # worst-case relative error of rounding one value to bfloat16
 
+# Every value comparison leaves a record here: (what, elements, max|err|/rms, rms(err)/rms,
+# number of elements beyond the plain 2e-2 * rms).  tests/conftest.py prints them at the end of
+# a run and writes them to the file named by ETR_PARITY_REPORT.
+PARITY_LOG = []
+_log_context = [""]
 
-def assert_close_rms(got, ref, rel, what, chain=1, rms=None):
-    """|got - ref| <= rel * rms(ref) + chain * 2^-8 * |ref|, element by element.
 
-    The first term is the target's bound (2e-2 of the reference tensor's RMS for bf16
-    compute, 1e-4 for fp32).  The second exists only for bf16 storage (rel >= 1e-2) and
-    covers what rounding to the bf16 grid does to a single large element, which no kernel
-    writing bf16 can avoid: each rounding costs up to half an ulp, 2^-8 of the value (an
-    element 5 RMS large already carries 2e-2 RMS of it).  `chain` is the number of
-    bf16-stored tensors on the multiplicative path from the test's inputs to this output,
-    the output's own store included: 1 for a stage fed with inputs already on the grid.
+def parity_context(label: str) -> None:
+    """Names the case whose comparisons follow (prefix of the records)."""
+    _log_context[0] = label
 
-    For bf16 the bound is a max over millions of elements of an error whose RMS is a few
-    tenths of a percent of rms(ref) per stored intermediate, i.e. it sits in the extreme
-    tail; up to 2e-5 of the elements (at least one) may exceed it, none by more than 2x.
-    fp32 comparisons allow no outliers."""
-    storage = chain * BF16_HALF_ULP if rel >= 1e-2 else 0.0
+
+def error_stats(got, ref, rms=None):
+    """(max|err|/rms, rms(err)/rms, count of |err| > 2e-2*rms, rms) of got against ref; rms is
+    that of ref unless the caller passes the RMS of the whole tensor a sample was taken from."""
     ref64 = ref.astype(np.float64)
-    if rms is None:       # callers comparing a sample pass the RMS of the whole tensor
-        rms = np.sqrt((ref64 ** 2).mean()) if ref.size else 0.0
+    if rms is None:
+        rms = float(np.sqrt((ref64 ** 2).mean())) if ref.size else 0.0
     err = np.abs(got.astype(np.float64) - ref64)
-    tol = rel * rms + storage * np.abs(ref64) + 1e-30
+    if not ref.size or rms == 0.0:
+        return 0.0, 0.0, int((err > 0).sum()), rms
+    return (float(err.max() / rms), float(np.sqrt((err ** 2).mean()) / rms),
+            int((err > 2e-2 * rms).sum()), rms)
+
+
+def _record(what, n, stats):
+    PARITY_LOG.append((f"{_log_context[0]}:{what}" if _log_context[0] else what, int(n)) + tuple(stats[:3]))
+
+
+# Rounding one value to bf16 leaves a relative error uniform within half an ulp: at most 2^-8,
+# RMS about 1.66e-3 of the value (measured on G, U, H: 1.66e-3).  Each bf16-stored tensor on the
+# path to an output adds that much, incoherently, so rms(err) ~ 1.66e-3 * sqrt(chain) * rms(ref)
+# (measured: O 2.35e-3, Y 2.87e-3, dX 3.5-3.8e-3).  Asserted with a 20 % margin.
+RMS_ERR_PER_STORE = 2e-3
+OUTLIER_FRACTION = 2e-5       # measured: at most 2.0e-5 of a tensor's elements (2 of 102400)
+OUTLIER_CEILING = 2.0         # measured: none beyond 1.8x the element's tolerance
+
+
+def assert_close_rms(got, ref, rel, what, chain=1, rms=None, outlier_fraction=OUTLIER_FRACTION):
+    """Value comparison against the fp32 oracle.
+
+    fp32 layers (rel < 1e-2): |err| <= rel * rms(ref) element by element, no exceptions.
+
+    bf16 storage (rel >= 1e-2), with `chain` the number of bf16-stored tensors on the
+    multiplicative path from the test's inputs to this output, its own store included (1 for a
+    stage fed with inputs already on the grid):
+      1. rms(err) <= 2e-3 * sqrt(chain) * rms(ref): the size of the error as a whole, 20 % above
+         what the roundings alone give.
+      2. |err| <= rel * rms(ref) + chain * 2^-8 * |ref| element by element.  The first term is the
+         target's bound.  The second is what storing bf16 costs a single large element, which no
+         kernel writing bf16 can avoid: each rounding moves a value by up to 2^-8 of itself (an
+         element 5 RMS large already carries 2e-2 RMS of it), and the factors of an elementwise
+         product (dG = dH * U * s'(G)) each pass their own on.  This bound is the maximum over up
+         to 10^7 elements of an error whose scale also varies from row to row (tokens with
+         several rows or a large gate), so it sits in the far tail: up to 2e-5 of the elements
+         may miss it, none by more than 2x (`outlier_fraction` is raised by the one caller whose
+         tensor has a known heavier tail, and says why).  The sharp, exception-free comparison is
+         the one against the oracle composed on the storage grid (storage_grid_reference).
+    Every call records max|err|/rms, rms(err)/rms and the number of elements beyond the plain
+    rel * rms in PARITY_LOG."""
+    ref64 = ref.astype(np.float64)
+    stats = error_stats(got, ref, rms)
+    rms = stats[3]
+    _record(what, ref.size, stats)
+    err = np.abs(got.astype(np.float64) - ref64)
+    if rel < 1e-2:
+        worst = float((err / (rel * rms + 1e-30)).max()) if ref.size else 0.0
+        assert worst <= 1.0, f"{what}: worst err {err.max():.3e}, rms {rms:.3e}, err/tol {worst:.2f}"
+        return worst
+    assert stats[1] <= RMS_ERR_PER_STORE * np.sqrt(chain), (
+        f"{what}: rms(err)/rms(ref) = {stats[1]:.2e} > {RMS_ERR_PER_STORE * np.sqrt(chain):.2e}")
+    tol = rel * rms + chain * BF16_HALF_ULP * np.abs(ref64) + 1e-30
     ratio = err / tol
     n_bad = int((ratio > 1.0).sum())
-    allowed = max(1, int(2e-5 * ref.size)) if rel >= 1e-2 else 0
+    allowed = max(1, int(outlier_fraction * ref.size))
     worst = float(ratio.max()) if ref.size else 0.0
-    assert n_bad <= allowed and worst <= 2.0, (
-        f"{what}: {n_bad} of {ref.size} elements outside tolerance (allowed {allowed}); worst "
-        f"err {err.max():.3e}, rms {rms:.3e}, worst err/tol {worst:.2f}")
+    assert n_bad <= allowed and worst <= OUTLIER_CEILING, (
+        f"{what}: {n_bad} of {ref.size} elements outside {rel:g}*rms + {chain}*2^-8|ref| (allowed {allowed}); "
+        f"worst err {err.max():.3e}, rms {rms:.3e}, worst err/tol {worst:.2f}, max|err|/rms {stats[0]:.3e}")
     return worst
+
+
+BF16_ULP = 2.0 ** -7
+
+
+def assert_on_grid(got, ref, what, rms_rel=2e-2, ulps=1):
+    """Comparison with the oracle composed on the storage grid, no exceptions:
+    |err| <= ulps * 2^-7 * |ref| + rms_rel * rms(ref).  One ulp is the element's own last-bit
+    flip (the two sides sum in a different order before they round); elementwise products of
+    stored tensors also pass on the flips of their factors (ulps = 2 or 3).  rms_rel is 2e-2, the
+    target's bound, for tensors downstream of a stored tensor, and 2e-4 for tensors computed from
+    exact inputs.  Records what the worst element needs beyond its ulps, in units of the RMS."""
+    ref64 = ref.astype(np.float64)
+    rms = float(np.sqrt((ref64 ** 2).mean()))
+    err = np.abs(got.astype(np.float64) - ref64)
+    excess = float(np.max(err - ulps * BF16_ULP * np.abs(ref64)) / rms)
+    PARITY_LOG.append((f"{_log_context[0]}:{what} vs grid, beyond {ulps} ulp", int(ref.size), excess,
+                       float(np.sqrt((err ** 2).mean()) / rms), int((err > 2e-2 * rms).sum())))
+    assert excess <= rms_rel, f"{what}: an element is {excess:.2e} rms beyond {ulps} ulp (allowed {rms_rel:g})"
+
+
+def assert_within(got, ref, rel, what, rms=None):
+    """The target's bound as it is written: max|err| <= rel * rms(ref), no exceptions."""
+    stats = error_stats(got, ref, rms)
+    _record(what, ref.size, stats)
+    assert stats[0] <= rel, f"{what}: max|err|/rms = {stats[0]:.3e} > {rel:g} ({stats[2]} elements beyond 2e-2)"
+    return stats[0]
+
+
+def storage_grid_reference(o, w, inp, fw, softmax_gate=False):
+    """The oracle's stages composed with the roundings the CUDA path applies when it stores a
+    tensor in bf16 (G, U, H, O, Y, dO, dG, dU, dXp, dX and the weight gradients; fp32 layers round
+    nothing).  Every stage is the oracle's own function, called on the rounded output of the stage
+    before it, so what remains between this reference and the device is fp32-vs-double summation
+    order and the odd flip of a final rounding.  `fw` is the oracle's forward on the same route."""
+    rnd = gw.round_to_bf16 if w.dtype == "bf16" else (lambda a: np.ascontiguousarray(a, dtype=np.float32))
+    rt, Cs = fw.route, fw.route.C_stride
+    W1g, W1u, W2 = inp["W1g"], inp["W1u"], inp["W2"]
+    g = SimpleNamespace()
+    g.G, g.U, g.H = rnd(fw.G), rnd(fw.U), rnd(fw.H)          # H is formed from the unrounded G and U
+    g.O = rnd(o.expert_ffn_down(g.H, rt, W2))
+    g.Y = rnd(o.combine(g.O, rt, fw.gate))
+    dO, g.dgate = o.combine_bwd(inp["dY"], g.O, rt, fw.gate)
+    g.dO = rnd(dO)
+    dG, dU, _, _, _, _ = o.expert_ffn_bwd(g.dO, fw.Xp, g.G, g.U, g.H, rt, W1g, W1u, W2)
+    g.dG, g.dU = rnd(dG), rnd(dU)
+    # dXp = dG W1g + dU W1u from the stored dG, dU: two "down" products with the weights transposed
+    W1gT = np.ascontiguousarray(W1g.transpose(0, 2, 1))
+    W1uT = np.ascontiguousarray(W1u.transpose(0, 2, 1))
+    g.dXp = rnd(o.expert_ffn_down(g.dG, rt, W1gT).astype(np.float64)
+                + o.expert_ffn_down(g.dU, rt, W1uT).astype(np.float64))
+    g.dW1g, g.dW1u, g.dW2 = (np.zeros_like(W1g), np.zeros_like(W1u), np.zeros_like(W2))
+    for e in range(rt.E):
+        n = int(rt.counts[e])
+        if n == 0:
+            continue
+        sl = slice(e * Cs, e * Cs + n)
+        a, b, c = o.ffn_weight_grads(g.dO[sl], g.H[sl], g.dG[sl], g.dU[sl], fw.Xp[sl])
+        g.dW1g[e], g.dW1u[e], g.dW2[e] = rnd(a), rnd(b), rnd(c)
+    dX = o.dispatch_bwd(g.dXp, rt)                           # the fused kernel keeps this sum in fp32
+    if softmax_gate:
+        ddelta = o.softmax_gate_bwd(fw.delta, g.dgate, rt)
+    else:
+        ddelta = o.select_bwd(g.dgate, rt)
+    dX, g.dR = o.affinity_bwd(inp["X"], inp["R"], w.D, fw.delta, fw.xnorm, fw.rnorm, ddelta, dX.copy())
+    g.dX = rnd(dX)
+    return g
 
 
 def assert_routes_match(delta_ref: np.ndarray, ref, got, mode: int, margin: float = MARGIN):

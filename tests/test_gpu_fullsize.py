@@ -146,7 +146,7 @@ def test_full_size(name):
         dd = np.zeros((n, E), np.float32)
         dd[:, i] = dgate
         _, dR_sub = o.affinity_bwd(X[toks], R, D, delta[toks], xnorm[toks], rnorm, dd, np.zeros((n, d), np.float32))
-        hz.assert_close_rms(hz.to_np(out["dR"][i]), dR_sub[i], tol, "dR[i]")
+        hz.assert_close_rms(hz.to_np(out["dR"][i]), dR_sub[i], tol, "dR[i]", chain=4)
 
     # ---- sampled tokens: Y[t] and dX[t] through every row of the token ------------------------------------------
     rng = np.random.default_rng(w.seed)
@@ -155,10 +155,6 @@ def test_full_size(name):
     multi = np.nonzero(nrows_t > 1)[0]
     n_tok = 6 if expert_rows is None else 3
     pick = list(rng.choice(routed, n_tok, replace=False)) + (list(rng.choice(multi, min(4, len(multi)), replace=False)) if len(multi) else [])
-    # RMS of the whole tensors over the routed tokens (unrouted rows are exact zeros)
-    scale = np.sqrt(T / max(1, len(routed)))
-    y_rms = float(out["Y"].float().pow(2).mean().sqrt()) * scale
-    dx_rms = float(out["dX"].float().pow(2).mean().sqrt()) * scale
     y_ref, dx_ref = np.zeros((len(pick), d)), np.zeros((len(pick), d), np.float32)
     for j, t in enumerate(pick):
         dx = np.zeros(d, np.float64)
@@ -175,8 +171,9 @@ def test_full_size(name):
         o.affinity_bwd(X[t:t + 1], R, D, delta[t:t + 1], xnorm[t:t + 1], rnorm, dd, dx32)
         dx_ref[j] = dx32[0]
     idx = torch.from_numpy(np.asarray(pick, dtype=np.int64)).cuda()
-    hz.assert_close_rms(hz.to_np(out["Y"][idx]), y_ref, tol, "Y[sampled tokens]", chain=4, rms=y_rms)
-    hz.assert_close_rms(hz.to_np(out["dX"][idx]), dx_ref, tol, "dX[sampled tokens]", chain=6, rms=dx_rms)
+    # the scale of each comparison is the RMS of the oracle's own rows (all sampled tokens are routed)
+    hz.assert_close_rms(hz.to_np(out["Y"][idx]), y_ref, tol, "Y[sampled tokens]", chain=4)
+    hz.assert_close_rms(hz.to_np(out["dX"][idx]), dx_ref, tol, "dX[sampled tokens]", chain=6)
 
     # ---- sampled hidden units of two other experts: exact slices of the weight gradients ----------------------
     others = [e for e in rng.permutation(E) if e != i and counts[e] > 0][:2]
@@ -197,6 +194,4 @@ def test_full_size(name):
         for nm, ref_slice, chain, take in (("dW1g", s_dW1g[0], 6, lambda a: a[B]),
                                            ("dW1u", s_dW1u[0], 6, lambda a: a[B]),
                                            ("dW2", s_dW2[0], 4, lambda a: a[:, B])):
-            full = hz.to_np(out[nm][e])
-            rms = np.sqrt((full.astype(np.float64) ** 2).mean())
-            hz.assert_close_rms(take(full), ref_slice, tol, f"{nm}[{e}] slice", chain=chain, rms=rms)
+            hz.assert_close_rms(take(hz.to_np(out[nm][e])), ref_slice, tol, f"{nm}[{e}] slice", chain=chain)

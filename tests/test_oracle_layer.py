@@ -276,3 +276,36 @@ def test_oracle_is_thread_count_independent(o32):
     assert np.array_equal(a.Y, b.Y)
     for f in ("dX", "dR", "dW1g", "dW1u", "dW2"):
         assert np.array_equal(getattr(ga, f), getattr(gb, f))
+
+
+def test_storage_grid_composition_reduces_to_the_oracle_without_rounding(o32):
+    """The stage-by-stage composition the GPU tests use as their sharp reference
+    (harness.storage_grid_reference) rounds nothing for an fp32 layer, so it must reproduce the
+    oracle's own forward and backward: same stages, same order, only split at the stored tensors
+    (dXp as two products with the transposed weights, weight gradients expert by expert)."""
+    from tests import harness as hz
+    w = gw.scaled(gw.WORKLOADS["tiny"], T=160, h=48)
+    inp = gw.make_inputs(w)
+    for soft in (False, True):
+        fw = o32.forward(inp["X"], inp["R"], inp["W1g"], inp["W1u"], inp["W2"], D=w.D, k=w.k,
+                         capacity=w.capacity, mode=ob.MODE_TCR, softmax_gate=soft)
+        bw = o32.backward(fw, inp["X"], inp["R"], inp["W1g"], inp["W1u"], inp["W2"], inp["dY"])
+        g = hz.storage_grid_reference(o32, w, inp, fw, softmax_gate=soft)
+        used = fw.route.slot_token >= 0
+        for nm, ref in (("G", fw.G), ("U", fw.U), ("H", fw.H), ("O", fw.O), ("dO", bw.dO), ("dG", bw.dG),
+                        ("dU", bw.dU), ("dXp", bw.dXp)):
+            a, b = getattr(g, nm)[used], ref[used]
+            assert np.max(np.abs(a - b)) <= 2e-6 * np.sqrt((b.astype(np.float64) ** 2).mean()), nm
+        for nm, ref in (("Y", fw.Y), ("dX", bw.dX), ("dR", bw.dR), ("dW1g", bw.dW1g), ("dW1u", bw.dW1u),
+                        ("dW2", bw.dW2), ("dgate", bw.dgate)):
+            a = getattr(g, nm)
+            assert np.max(np.abs(a - ref)) <= 2e-6 * np.sqrt((ref.astype(np.float64) ** 2).mean()), nm
+    # and on a bf16 workload every stored tensor of the composition lies on the bf16 grid
+    wb = gw.scaled(gw.WORKLOADS["small"], T=96, d=128, D=8, E=4, h=64)
+    inp = gw.make_inputs(wb)
+    fw = o32.forward(inp["X"], inp["R"], inp["W1g"], inp["W1u"], inp["W2"], D=wb.D, k=wb.k,
+                     capacity=wb.capacity, mode=ob.MODE_TCR)
+    g = hz.storage_grid_reference(o32, wb, inp, fw)
+    for nm in ("G", "U", "H", "O", "Y", "dO", "dG", "dU", "dXp", "dX", "dW1g", "dW1u", "dW2"):
+        a = getattr(g, nm)
+        assert np.array_equal(a, gw.round_to_bf16(a)), nm
