@@ -14,7 +14,7 @@
  *
  * Layouts: row-major, innermost index contiguous.
  *   X, Y, dY, dX [T,d]      R, dR [E,m] fp32        delta [T,E] fp32      Z [T,m] fp32
- *   W1g, W1u [E,h,d]        W2 [E,d,h]              (gradients: same shape and dtype)
+ *   W1g, W1u [E,h,d]        W2 [E,d,h]              (gradients: same shape; `dtype`, or fp32 with grad_fp32)
  *   Xp, O, dO, dXp [E*C_stride, d]                  G, U, H, dG, dU [E*C_stride, h]
  * C_stride = capacity rounded up to a multiple of 128.  Expert i owns rows
  * [i*C_stride, (i+1)*C_stride); the first counts[i] of them are in use.  Rows from
@@ -32,7 +32,8 @@
  * any launch.  A launch failure maps to ETR_ERR_CUDA.  Device-side problems (a bounded
  * wait in the GEMM pipeline that ran out) never trap: the kernel records a code in
  * etr_stats.error_word, stops issuing work and returns; etr_read_stats reports it as
- * ETR_ERR_TIMEOUT.
+ * ETR_ERR_TIMEOUT.  The bound of those waits is cfg->wait_limit_cycles (default about two
+ * seconds); etr_selftest_bounded_wait exercises the path on its own.
  */
 #ifndef ETR_H_
 #define ETR_H_
@@ -69,11 +70,24 @@ typedef enum { ETR_GEMM_AUTO = 0, ETR_GEMM_SIMT = 1, ETR_GEMM_TCGEN05 = 2, ETR_G
  * read.  The stage calls are unaffected.  ETR_FUSE_AUTO lets the library choose. */
 typedef enum { ETR_FUSE_AUTO = 0, ETR_FUSE_OFF = 1, ETR_FUSE_ON = 2 } etr_fuse;
 
-/* Gate of a selected pair (t, i).  AFFINITY (default): the raw affinity delta_ti ("the affinity
- * matrix is employed as the gating weight").  SOFTMAX: p_ti = exp(delta_ti) / sum_j exp(delta_tj)
+/* Gate of a selected pair (t, i).  AFFINITY (default): the raw affinity delta_ti (the affinity-score
+ * equation of "Cost-Efficient Sparse Expert-Token Affinity", whose matrix the paper also uses as the
+ * gating weight).  SOFTMAX: p_ti = exp(delta_ti) / sum_j exp(delta_tj)
  * over all E experts of the token, the example gate of the general MoE equation; its backward
  * gives every expert of a routed token a gradient (a dense d delta), see etr_gate_softmax_bwd. */
 typedef enum { ETR_GATE_AFFINITY = 0, ETR_GATE_SOFTMAX = 1 } etr_gate;
+
+/* Number of kept candidates set by a threshold on the sum of affinity scores ("Routing Strategy":
+ * the expert chooses its Top-l tokens with l determined by a threshold of the sum of affinity
+ * scores; "Training Strategy": the number of tokens per expert follows an adaptive threshold).  The
+ * paper gives no rule, so this is a reading: walking a candidate list in descending affinity, the
+ * candidate of rank j is kept while the sum of the j-1 affinities before it is still below tau (and
+ * j is within the capacity C, resp. k).  EXPERT applies it to every expert's candidate tokens (both
+ * modes), TOKEN to every token's experts (token choice only: a token then takes 1..k experts and
+ * the unused entries of topk_idx hold -1); the flags combine.  Sums are taken on affinities
+ * quantised to multiples of 2^-32 (round to nearest), as 64-bit integers, so they do not depend on
+ * the order of summation.  tau = +infinity reproduces the plain selection; tau <= 0 keeps nothing. */
+typedef enum { ETR_THRESHOLD_OFF = 0, ETR_THRESHOLD_EXPERT = 1, ETR_THRESHOLD_TOKEN = 2 } etr_threshold;
 
 /* Immutable description of one layer call (host struct, passed by pointer). */
 typedef struct etr_config {
@@ -88,7 +102,16 @@ typedef struct etr_config {
   int32_t gemm_impl;          /* etr_gemm_impl; AUTO = CTA-pair tcgen05 for bf16, SIMT for fp32 */
   int32_t fuse_dispatch;      /* etr_fuse: token rearrangement fused into the GEMM operand fetch */
   int32_t gate_mode;          /* etr_gate: what weighs an expert's output in the combine */
-  int32_t reserved;
+  int32_t grad_fp32;          /* != 0: dW1g, dW1u, dW2 are written as fp32 (same shapes) whatever `dtype` is;
+                                 0: in `dtype`.  The accumulation is fp32 either way. */
+  int32_t weight_dtype;       /* etr_dtype of W1g, W1u, W2.  Must equal `dtype`: the tensor-core
+                                 instruction takes both operands in one 16-bit type, so a layer with
+                                 bf16 activations and fp32 weights has no kernel (ETR_ERR_UNSUPPORTED) */
+  int32_t threshold_mode;     /* etr_threshold flags: selections also cut by a running sum of affinities */
+  float threshold_tau;        /* ETR_THRESHOLD_EXPERT: the sum at which an expert stops taking tokens */
+  float threshold_tau_token;  /* ETR_THRESHOLD_TOKEN: the sum at which a token stops taking experts */
+  int64_t wait_limit_cycles;  /* bound of every device-side wait of the GEMM pipeline, in SM clock
+                                 cycles; 0 = the default, about two seconds */
 } etr_config;
 
 /* Per-call scalars produced and consumed on the device (device struct, 64 bytes). */
@@ -169,7 +192,9 @@ etr_status etr_affinity(const etr_config* cfg, const void* X, const float* R, fl
  * or the batch maximum left in stats by etr_affinity.  Mode: cfg->mode, or from step.
  * Ties go to the lower index.  Kept tokens of an expert are stored in ascending token
  * order.  Fills every member of route and stats->{mode,C,dropped,unrouted,delta_max,
- * rows_total}.  ws: etr_workspace_bytes. */
+ * rows_total} (each is set by the call, not added to: selecting again on the same stats, e.g.
+ * at another step of a sweep, needs no clearing in between; delta_max_key and error_word are
+ * left as they are).  ws: etr_workspace_bytes. */
 etr_status etr_select(const etr_config* cfg, const float* delta, etr_stats* stats,
                       const etr_route* route, void* ws, void* stream);
 
@@ -189,7 +214,9 @@ etr_status etr_select(const etr_config* cfg, const float* delta, etr_stats* stat
  * ends.
  * The call itself allocates and frees nothing.  Its first use on a device looks up the
  * array's device address (once per device, with that device current); make that first call
- * outside any stream capture.
+ * outside any stream capture.  The address is kept for the life of the process: after a
+ * cudaDeviceReset of that device it is stale, and the library must be reloaded before the call
+ * is used there again.
  * All calls share the one array, which keeps whatever the previous call left in it: the
  * selection overwrites every entry it later reads, so nothing needs clearing, but two calls
  * whose kernels overlap on the same GPU (different streams, or threads) race on it — keep
@@ -224,7 +251,8 @@ etr_status etr_combine_bwd(const etr_config* cfg, const etr_route* route, const 
 
 /* dH = dO W2_i;  dG = dH*U*s*(1+G*(1-s)), dU = dH*G*s with s = sigmoid(G);
  * dXp = dG W1g_i + dU W1u_i;  dW2_i = dO^T H;  dW1g_i = dG^T Xp;  dW1u_i = dU^T Xp.
- * Experts with no rows get zero weight gradients. */
+ * Experts with no rows get zero weight gradients.  dW1g, dW1u, dW2 are `dtype`, or fp32 when
+ * cfg->grad_fp32 is set (the fp32 accumulators stored unrounded). */
 etr_status etr_expert_ffn_bwd(const etr_config* cfg, const etr_route* route, const void* dO,
                               const void* Xp, const void* G, const void* U, const void* H,
                               const void* W1g, const void* W1u, const void* W2,
@@ -335,6 +363,15 @@ etr_status etr_layer_step_host_wait(int32_t slot);
 /* Copies the device stats to the host and synchronises the stream.  Returns
  * ETR_ERR_TIMEOUT if a kernel recorded an expired wait. */
 etr_status etr_read_stats(const etr_stats* stats_dev, etr_stats* stats_host, void* stream);
+
+/* Self-test of the bounded device-side wait (the failure path of the GEMM pipeline, which a healthy
+ * run never takes): launches one warp that waits, with the pipeline's own wait routine, on a
+ * barrier nothing will ever arrive on.  After limit_cycles SM clock cycles (1 .. 4e9; 1e5 is about
+ * 50 microseconds) the wait gives up, the kernel writes a code to stats->error_word and returns
+ * normally; etr_read_stats then reports ETR_ERR_TIMEOUT and the stream and context stay usable.
+ * Nothing else is in flight in that kernel: no copy, no tensor memory.  The caller clears
+ * error_word (etr_layer_forward does) before the next ordinary use of `stats`. */
+etr_status etr_selftest_bounded_wait(etr_stats* stats, int64_t limit_cycles, void* stream);
 
 /* Number of kernels launched by this library in the calling process so far. */
 int64_t etr_launch_count(void);

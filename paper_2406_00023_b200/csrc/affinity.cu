@@ -1015,17 +1015,6 @@ static size_t affinity_smem_bytes(int E, int m, int* ldm_out, int* Epad_out) {
   return ((size_t)(Epad + AFF_TB) * ldm + AFF_TB + Epad) * sizeof(float);
 }
 
-static int device_sm_count() {
-  static int n = 0;
-  if (n == 0) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
-    if (n <= 0) n = 148;
-  }
-  return n;
-}
-
 template <class T, int EPL, int TPG>
 static etr_status launch_affinity_warp(const etr_config* c, const void* X, const float* R, float* delta,
                                        float* Z, float* xnorm, float* rnorm, etr_stats* stats,
@@ -1039,7 +1028,7 @@ static etr_status launch_affinity_warp(const etr_config* c, const void* X, const
     if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
       return ETR_ERR_CUDA;
     const int ngroups = ceil_div(c->T, TPG);
-    const int grid = std::min(device_sm_count(), ceil_div(ngroups, nw));
+    const int grid = std::min(current_sm_count(), ceil_div(ngroups, nw));
     ETR_TIME_BEGIN("affinity_fwd_warp_kernel");
     k<<<grid, nw * 32, smem, st>>>((const T*)X, R, delta, Z, xnorm, rnorm, stats, c->T, c->d, c->D,
                                    c->E, m, ldm);
@@ -1085,7 +1074,7 @@ static etr_status launch_score(const etr_config* c, const float* Z, const float*
     if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
       return ETR_ERR_CUDA;
     const int ngroups = ceil_div(c->T, TPG);
-    const int grid = std::min(device_sm_count(), ceil_div(ngroups, nw));
+    const int grid = std::min(current_sm_count(), ceil_div(ngroups, nw));
     ETR_TIME_BEGIN("affinity_score_kernel");
     k<<<grid, nw * 32, smem, st>>>(Z, xnorm, R, delta, rnorm, stats, c->T, c->D, c->E, m, ldm);
     ETR_LAUNCH_CHECK();
@@ -1106,7 +1095,7 @@ static etr_status launch_score_tile(const etr_config* c, const float* Z, const f
   auto k = affinity_score_tile_kernel<EPT>;
   if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
     return ETR_ERR_CUDA;
-  const int grid = std::min(2 * device_sm_count(), ceil_div(c->T, SC_TM));
+  const int grid = std::min(2 * current_sm_count(), ceil_div(c->T, SC_TM));
   ETR_TIME_BEGIN("affinity_score_kernel");
   k<<<grid, 256, smem, st>>>(Z, xnorm, R, delta, rnorm, stats, c->T, c->D, c->E, m, ldm);
   ETR_LAUNCH_CHECK();
@@ -1126,7 +1115,7 @@ static etr_status affinity_forward_split(const etr_config* c, const void* X, con
   if (c->dtype == ETR_BF16) ETR_TRY(launch_pool<__nv_bfloat16>(c, X, Z, xnorm, st));
   else ETR_TRY(launch_pool<float>(c, X, Z, xnorm, st));
   // the tiled form needs a tile of 256 tokens for every SM to pay for its set-up (R and its norms per block)
-  if (c->E <= 64 && m % SC_KC == 0 && ceil_div(c->T, SC_TM) >= device_sm_count()) {
+  if (c->E <= 64 && m % SC_KC == 0 && ceil_div(c->T, SC_TM) >= current_sm_count()) {
     if (c->E <= 16) ETR_TRY(launch_score_tile<2>(c, Z, xnorm, R, delta, rnorm, stats, st, done));
     else if (c->E <= 32) ETR_TRY(launch_score_tile<4>(c, Z, xnorm, R, delta, rnorm, stats, st, done));
     else ETR_TRY(launch_score_tile<8>(c, Z, xnorm, R, delta, rnorm, stats, st, done));

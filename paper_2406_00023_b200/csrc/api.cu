@@ -9,6 +9,8 @@
 
 namespace etr {
 
+static_assert(sizeof(etr_config) == 104 && sizeof(etr_stats) == 64, "layouts the bindings rely on");
+
 static std::atomic<long long> g_launches{0};
 void note_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 
@@ -146,6 +148,13 @@ etr_status etr_validate(const etr_config* c) {
   if (c->gemm_impl < ETR_GEMM_AUTO || c->gemm_impl > ETR_GEMM_TCGEN05_2CTA_WIDE) return ETR_ERR_ARG;
   if (c->fuse_dispatch < ETR_FUSE_AUTO || c->fuse_dispatch > ETR_FUSE_ON) return ETR_ERR_ARG;
   if (c->gate_mode != ETR_GATE_AFFINITY && c->gate_mode != ETR_GATE_SOFTMAX) return ETR_ERR_ARG;
+  if (c->weight_dtype != ETR_F32 && c->weight_dtype != ETR_BF16) return ETR_ERR_ARG;
+  if (c->threshold_mode < 0 || c->threshold_mode > (ETR_THRESHOLD_EXPERT | ETR_THRESHOLD_TOKEN)) return ETR_ERR_ARG;
+  if (c->threshold_mode != ETR_THRESHOLD_OFF && (c->threshold_tau != c->threshold_tau ||
+                                                  c->threshold_tau_token != c->threshold_tau_token))
+    return ETR_ERR_ARG;                                   // NaN thresholds
+  if (c->wait_limit_cycles < 0) return ETR_ERR_ARG;
+  if (c->weight_dtype != c->dtype) return ETR_ERR_UNSUPPORTED;
   if (c->d % c->D != 0 || c->d % 8 != 0 || c->h % 8 != 0) return ETR_ERR_SHAPE;
   if (c->k > c->E || c->E > 256 || c->E > c->d / c->D) return ETR_ERR_SHAPE;
   if ((long long)c->T * c->E >= (1ll << 31)) return ETR_ERR_SHAPE;
@@ -498,6 +507,12 @@ etr_status etr_read_stats(const etr_stats* dev, etr_stats* host, void* stream) {
     return ETR_ERR_CUDA;
   if (cudaStreamSynchronize(st) != cudaSuccess) return ETR_ERR_CUDA;
   return host->error_word ? ETR_ERR_TIMEOUT : ETR_OK;
+}
+
+etr_status etr_selftest_bounded_wait(etr_stats* stats, int64_t limit_cycles, void* stream) {
+  if (stats == nullptr || limit_cycles < 1 || limit_cycles > 4000000000ll) return ETR_ERR_ARG;
+  if (!aligned16(stats)) return ETR_ERR_ALIGN;
+  return tc_wait_selftest(stats, (long long)limit_cycles, (cudaStream_t)stream);
 }
 
 int64_t etr_launch_count(void) { return (int64_t)g_launches.load(); }

@@ -4,6 +4,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "../../include/etr.h"
 
 namespace etr {
@@ -32,6 +34,33 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 inline size_t elem_bytes(int dtype) { return dtype == ETR_BF16 ? 2 : 4; }
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
+inline size_t grad_elem_bytes(const etr_config* c) { return c->grad_fp32 ? 4 : elem_bytes(c->dtype); }
+
+// Opt-in to more than 48 KiB of dynamic shared memory: an attribute of the kernel on ONE device, so
+// it is set once per device (a bit per device ordinal in `done`, one flag word per kernel).
+template <class K>
+inline bool ensure_dyn_smem(K kernel, size_t bytes, std::atomic<unsigned long long>& done) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return false;
+  const unsigned long long bit = 1ull << (dev & 63);
+  if (done.load(std::memory_order_acquire) & bit) return true;
+  if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess)
+    return false;
+  done.fetch_or(bit, std::memory_order_release);
+  return true;
+}
+// Multiprocessor count of the current device (cached per device ordinal).
+inline int current_sm_count() {
+  static std::atomic<int> cache[64];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+  int n = cache[dev & 63].load(std::memory_order_relaxed);
+  if (n <= 0) {
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+    cache[dev & 63].store(n, std::memory_order_relaxed);
+  }
+  return n;
+}
 
 // ---- order-preserving map float -> uint32 (larger float <=> larger key; key 0 is below
 //      every finite float and is used as "not a candidate") --------------------------------
@@ -150,6 +179,7 @@ etr_status tc_ffn_backward(const etr_config* cfg, const etr_route* route, const 
                            void* dXp, void* dW1g, void* dW1u, void* dW2, etr_stats* stats,
                            void* ws, cudaStream_t st);
 size_t tc_workspace_bytes(const etr_config* cfg);
+etr_status tc_wait_selftest(etr_stats* stats, long long limit_cycles, cudaStream_t st);
 bool tc_available();
 
 }  // namespace etr

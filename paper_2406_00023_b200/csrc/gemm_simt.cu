@@ -25,6 +25,7 @@ struct GemmArgs {
   long long out_bs;
   const int32_t* counts;
   int dyn, m_cap;
+  int out_f32;              // STORE: C is fp32 whatever T is (weight gradients with grad_fp32)
 };
 
 __device__ inline float silu_f(float v) { return v / (1.0f + expf(-v)); }
@@ -94,7 +95,8 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(GemmArgs g) {
       if (gn >= g.N) continue;
       const long long o = (long long)e * g.out_bs + (long long)gm * g.ld_out + gn;
       if (EPI == EPI_STORE) {
-        ((T*)g.out0)[o] = from_f32<T>(acc0[i][j]);
+        if (g.out_f32) ((float*)g.out0)[o] = acc0[i][j];
+        else ((T*)g.out0)[o] = from_f32<T>(acc0[i][j]);
       } else if (EPI == EPI_SWIGLU) {
         const float gg = acc0[i][j], uu = acc1[i][j];
         ((T*)g.out0)[o] = from_f32<T>(gg);
@@ -175,6 +177,7 @@ static etr_status ffn_backward_t(const etr_config* c, const etr_route* rt, const
     g.A[0] = {dO, (long long)Cs * d, 1, d};
     g.B[0] = {H, (long long)Cs * h, h, 1};
     g.npair = 1; g.M = d; g.N = h; g.K = 0; g.ld_out = h; g.out_bs = (long long)d * h; g.out0 = dW2;
+    g.out_f32 = c->grad_fp32 != 0;
     ETR_TRY((launch<T, EPI_STORE>(g, E, st)));
   }
   for (int which = 0; which < 2; ++which) {  // dW1[b,c] = sum_r dG[r,b] Xp[r,c]
@@ -184,6 +187,7 @@ static etr_status ffn_backward_t(const etr_config* c, const etr_route* rt, const
     g.B[0] = {Xp, (long long)Cs * d, d, 1};
     g.npair = 1; g.M = h; g.N = d; g.K = 0; g.ld_out = d; g.out_bs = (long long)h * d;
     g.out0 = which ? dW1u : dW1g;
+    g.out_f32 = c->grad_fp32 != 0;
     ETR_TRY((launch<T, EPI_STORE>(g, E, st)));
   }
   return ETR_OK;

@@ -64,6 +64,8 @@ struct TcParams {
   int gather;
   int gather_ld, gather_oob;
   const int32_t* gather_idx;
+  long long wait_limit;  // bound of every mbarrier wait, in SM clock cycles
+  int out_f32;           // plain-store epilogue: out0 is fp32 (weight gradients with grad_fp32)
 };
 
 // ---- PTX wrappers -----------------------------------------------------------------------------
@@ -89,14 +91,15 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 // Bounded wait: false if this or another thread of the CTA gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          long long limit_cycles) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   for (uint32_t it = 1;; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((it & 255u) == 0u) {
       if (*abort_flag) return false;
-      if (clock64() - t0 > TC_WAIT_LIMIT_CYCLES) { *abort_flag = 1; return false; }
+      if (clock64() - t0 > limit_cycles) { *abort_flag = 1; return false; }
     }
   }
 }
@@ -148,13 +151,6 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
   __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
   return *reinterpret_cast<uint32_t*>(&v);
 }
-__device__ __forceinline__ void store32(__nv_bfloat16* dst, const float* v) {
-  uint4* p = reinterpret_cast<uint4*>(dst);
-#pragma unroll
-  for (int q = 0; q < 4; ++q)
-    p[q] = make_uint4(pack_bf16(v[8 * q], v[8 * q + 1]), pack_bf16(v[8 * q + 2], v[8 * q + 3]),
-                      pack_bf16(v[8 * q + 4], v[8 * q + 5]), pack_bf16(v[8 * q + 6], v[8 * q + 7]));
-}
 __device__ __forceinline__ void load32(const __nv_bfloat16* src, float* v) {
   const uint4* p = reinterpret_cast<const uint4*>(src);
 #pragma unroll
@@ -196,9 +192,10 @@ __device__ __forceinline__ void store32_warp(uint8_t* scratch, int lane, int nva
   __syncwarp();
 }
 
-// The same store for a block already packed to bf16 (16 words per lane).
-__device__ __forceinline__ void store32_warp_packed(uint8_t* scratch, int lane, int nvalid, __nv_bfloat16* dst,
-                                                    int ld_out, const uint32_t* w16) {
+// The same turn for 16 raw 32-bit words per lane (64 bytes of a row): a 32 x 32 block already packed
+// to bf16, or half of a 32 x 32 block of fp32.  dst is the first row's address, rows ld_bytes apart.
+__device__ __forceinline__ void store_rows64(uint8_t* scratch, int lane, int nvalid, char* dst,
+                                             long long ld_bytes, const uint32_t* w16) {
   uint4* mine = reinterpret_cast<uint4*>(scratch + lane * TC_SCRATCH_ROW_BYTES);
 #pragma unroll
   for (int q = 0; q < 4; ++q) mine[q] = make_uint4(w16[4 * q], w16[4 * q + 1], w16[4 * q + 2], w16[4 * q + 3]);
@@ -208,9 +205,31 @@ __device__ __forceinline__ void store32_warp_packed(uint8_t* scratch, int lane, 
   for (int i = 0; i < 4; ++i) {
     const int row = (lane >> 2) + 8 * i;
     const uint4 w = *reinterpret_cast<const uint4*>(scratch + row * TC_SCRATCH_ROW_BYTES + sub * 16);
-    if (row < nvalid) *reinterpret_cast<uint4*>(dst + (long long)row * ld_out + sub * 8) = w;
+    if (row < nvalid) *reinterpret_cast<uint4*>(dst + row * ld_bytes + sub * 16) = w;
   }
   __syncwarp();
+}
+__device__ __forceinline__ void store32_warp_packed(uint8_t* scratch, int lane, int nvalid, __nv_bfloat16* dst,
+                                                    int ld_out, const uint32_t* w16) {
+  store_rows64(scratch, lane, nvalid, reinterpret_cast<char*>(dst), 2ll * ld_out, w16);
+}
+// A 32 x 32 block of fp32 accumulators (lane = row, 32 raw words) stored as fp32: two 64-byte halves.
+__device__ __forceinline__ void store32_warp_f32(uint8_t* scratch, int lane, int nvalid, float* dst, int ld_out,
+                                                 const uint32_t* r32) {
+  store_rows64(scratch, lane, nvalid, reinterpret_cast<char*>(dst), 4ll * ld_out, r32);
+  store_rows64(scratch, lane, nvalid, reinterpret_cast<char*>(dst) + 64, 4ll * ld_out, r32 + 16);
+}
+// 32 zeros at element offset `off` of the output (this lane's row of a block with nothing to contract).
+__device__ __forceinline__ void store_zero32(const TcParams& p, long long off) {
+  if (p.out_f32) {
+    float4* q = reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out0) + off);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) q[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+  } else {
+    uint4* q = reinterpret_cast<uint4*>(p.out0 + off);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) q[i] = make_uint4(0, 0, 0, 0);
+  }
 }
 
 // The reverse turn for the saved activations the SwiGLU derivative reads: fetched as 8 rows x
@@ -296,9 +315,13 @@ __device__ __forceinline__ void epilogue_chunks(const TcParams& p, int n0, uint3
       }
     } else {
       tc_wait_ld();
+      if (p.out_f32) {
+        store32_warp_f32(scratch, lane, nvalid, reinterpret_cast<float*>(p.out0) + wbase + 32 * c, p.ld_out, r0);
+      } else {
 #pragma unroll
-      for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r0[i]);
-      store32_warp(scratch, lane, nvalid, p.out0 + wbase + 32 * c, p.ld_out, v);
+        for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r0[i]);
+        store32_warp(scratch, lane, nvalid, p.out0 + wbase + 32 * c, p.ld_out, v);
+      }
     }
   }
 }
@@ -391,7 +414,7 @@ tc_grouped_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_c
       bool ok = true;
       for (int tile = blockIdx.x; ok && tile_coord(p, tile_prefix, s_counts, tile, e_cur, N_TILE_COLS, tc); tile += gridDim.x) {
         for (int kb = 0; kb < tc.kblocks; ++kb) {
-          if (!mbar_wait(empty_bar + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
+          if (!mbar_wait(empty_bar + 8 * stage, phase ^ 1u, abort_flag, p.wait_limit)) { ok = false; break; }
           const uint32_t fb = full_bar + 8 * stage;
           mbar_expect_tx(fb, STAGE_BYTES);
           const bool second = p.k1_blocks > 0 && kb >= p.k1_blocks;
@@ -431,11 +454,11 @@ tc_grouped_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_c
       const uint32_t a_kstep = p.a_mn ? 2048u : 32u, b_kstep = p.b_mn ? 2048u : 32u;
       for (int tile = blockIdx.x; ok && tile_coord(p, tile_prefix, s_counts, tile, e_cur, N_TILE_COLS, tc); tile += gridDim.x) {
         if (tc.kblocks == 0) continue;
-        if (!mbar_wait(tempty_bar + 8 * acc_stage, acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+        if (!mbar_wait(tempty_bar + 8 * acc_stage, acc_phase ^ 1u, abort_flag, p.wait_limit)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc_stage * 256);
         for (int kb = 0; kb < tc.kblocks; ++kb) {
-          if (!mbar_wait(full_bar + 8 * stage, phase, abort_flag)) { ok = false; break; }
+          if (!mbar_wait(full_bar + 8 * stage, phase, abort_flag, p.wait_limit)) { ok = false; break; }
           tc_fence_after();
           const uint32_t sa = tiles_base + stage * STAGE_BYTES;
           const uint32_t sb = sa + 2 * TC_BOX_BYTES;
@@ -470,12 +493,8 @@ tc_grouped_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_c
       const int c_beg = half * NCH;
       const long long obase = (long long)tc.e * p.out_bs + (long long)grow * p.ld_out + tc.n0;
       if (tc.kblocks == 0) {        // nothing to contract: the block of the output is zero
-        if (row_ok) {
-          float z[32];
-#pragma unroll
-          for (int i = 0; i < 32; ++i) z[i] = 0.f;
-          for (int c = c_beg; c < c_beg + NCH && tc.n0 + 32 * c < p.N; ++c) store32(p.out0 + obase + 32 * c, z);
-        }
+        if (row_ok)
+          for (int c = c_beg; c < c_beg + NCH && tc.n0 + 32 * c < p.N; ++c) store_zero32(p, obase + 32 * c);
         continue;
       }
       // SwiGLU derivative: the saved G and U of the first chunk are fetched before the
@@ -487,7 +506,7 @@ tc_grouped_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_c
         load32_warp_issue(p.in0 + wb, p.ld_out, lane, nvalid, pg);
         load32_warp_issue(p.in1 + wb, p.ld_out, lane, nvalid, pu);
       }
-      if (!mbar_wait(tfull_bar + 8 * acc_stage, acc_phase, abort_flag)) { ok = false; break; }
+      if (!mbar_wait(tfull_bar + 8 * acc_stage, acc_phase, abort_flag, p.wait_limit)) { ok = false; break; }
       tc_fence_after();
       const uint32_t taddr = tmem_base + (uint32_t)(acc_stage * 256) + ((uint32_t)(32 * q) << 16);
       epilogue_chunks<EPI, BN>(p, tc.n0, taddr, obase, row_ok, c_beg, NCH, pg, pu, scratch, lane, nvalid);
@@ -561,14 +580,15 @@ __device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t par
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
 }
-__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                                  long long limit_cycles) {
   if (mbar_try_wait_cluster(bar, parity)) return true;
   const long long t0 = clock64();
   for (uint32_t it = 1;; ++it) {
     if (mbar_try_wait_cluster(bar, parity)) return true;
     if ((it & 255u) == 0u) {
       if (*abort_flag) return false;
-      if (clock64() - t0 > TC_WAIT_LIMIT_CYCLES) { *abort_flag = 1; return false; }
+      if (clock64() - t0 > limit_cycles) { *abort_flag = 1; return false; }
     }
   }
 }
@@ -719,7 +739,7 @@ tc_grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap mapA0, const __g
           int4 rows_next = rows_b;
           if (GATHER == 2 && kb + 1 < tc.kblocks)
             rows_next = gather_rows(gidx + (kb + 1) * TC_BK + 4 * (lane & 15), p.gather_oob);
-          if (!mbar_wait_cluster(empty_bar + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
+          if (!mbar_wait_cluster(empty_bar + 8 * stage, phase ^ 1u, abort_flag, p.wait_limit)) { ok = false; break; }
           if (rank == 0 && lane == 0) mbar_expect_tx(full_bar + 8 * stage, 2 * TC2_STAGE_BYTES);
           const uint32_t fb = leader_full + 8 * stage;
           const bool second = TWO_K && kb >= p.k1_blocks;
@@ -762,11 +782,11 @@ tc_grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap mapA0, const __g
       const uint32_t a_kstep = A_MN ? 2048u : 32u, b_kstep = B_MN ? 2048u : 32u;
       for (int tile = pair; ok && tile_coord_pair(p, tile_prefix, s_counts, tile, e_cur, N_TILE_COLS, tc); tile += npairs) {
         if (tc.kblocks == 0) continue;
-        if (!mbar_wait_cluster(tempty_bar + 8 * acc_stage, acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+        if (!mbar_wait_cluster(tempty_bar + 8 * acc_stage, acc_phase ^ 1u, abort_flag, p.wait_limit)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc_stage * 256);
         for (int kb = 0; kb < tc.kblocks; ++kb) {
-          if (!mbar_wait_cluster(full_bar + 8 * stage, phase, abort_flag)) { ok = false; break; }
+          if (!mbar_wait_cluster(full_bar + 8 * stage, phase, abort_flag, p.wait_limit)) { ok = false; break; }
           tc_fence_after();
           const uint32_t sa = tiles_base + stage * TC2_STAGE_BYTES;
           const uint32_t sb = sa + 2 * TC_BOX_BYTES;
@@ -801,12 +821,8 @@ tc_grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap mapA0, const __g
       const int c_beg = half * NCH;
       const long long obase = (long long)tc.e * p.out_bs + (long long)grow * p.ld_out + tc.n0;
       if (tc.kblocks == 0) {
-        if (row_ok) {
-          float z[32];
-#pragma unroll
-          for (int i = 0; i < 32; ++i) z[i] = 0.f;
-          for (int c = c_beg; c < c_beg + NCH && tc.n0 + 32 * c < p.N; ++c) store32(p.out0 + obase + 32 * c, z);
-        }
+        if (row_ok)
+          for (int c = c_beg; c < c_beg + NCH && tc.n0 + 32 * c < p.N; ++c) store_zero32(p, obase + 32 * c);
         continue;
       }
       uint4 pg[4], pu[4];
@@ -816,7 +832,7 @@ tc_grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap mapA0, const __g
         load32_warp_issue(p.in0 + wb, p.ld_out, lane, nvalid, pg);
         load32_warp_issue(p.in1 + wb, p.ld_out, lane, nvalid, pu);
       }
-      if (!mbar_wait_cluster(tfull_bar + 8 * acc_stage, acc_phase, abort_flag)) { ok = false; break; }
+      if (!mbar_wait_cluster(tfull_bar + 8 * acc_stage, acc_phase, abort_flag, p.wait_limit)) { ok = false; break; }
       tc_fence_after();
       const uint32_t taddr = tmem_base + (uint32_t)(acc_stage * 256) + ((uint32_t)(32 * q) << 16);
       epilogue_chunks<EPI, BN>(p, tc.n0, taddr, obase, row_ok, c_beg, NCH, pg, pu, scratch, lane, nvalid);
@@ -954,7 +970,7 @@ tc_grouped_gemm_pair_wide_kernel(const __grid_constant__ CUtensorMap mapA0, cons
           rows_a = m0c < p.M ? gather_rows(p.gather_idx + (size_t)tc.e * p.gather_ld + m0c + 4 * lane, p.gather_oob)
                              : make_int4(p.gather_oob, p.gather_oob, p.gather_oob, p.gather_oob);
         for (int kb = 0; kb < tc.kblocks; ++kb) {
-          if (!mbar_wait_cluster(empty_bar + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
+          if (!mbar_wait_cluster(empty_bar + 8 * stage, phase ^ 1u, abort_flag, p.wait_limit)) { ok = false; break; }
           if (rank == 0 && lane == 0) mbar_expect_tx(full_bar + 8 * stage, 2 * (two ? 6 : 4) * TC_BOX_BYTES);
           const uint32_t fb = leader_full + 8 * stage;
           const bool second = TWO_K && kb >= p.k1_blocks;
@@ -1009,24 +1025,24 @@ tc_grouped_gemm_pair_wide_kernel(const __grid_constant__ CUtensorMap mapA0, cons
       for (int tile = pair; ok && tile_coord_wide(p, tile_prefix, s_counts, tile, e_cur, N_TILE_COLS, tc); tile += npairs) {
         if (tc.kblocks == 0) continue;
         const bool two = tc.n0 + N_TILE_COLS < p.N;
-        if (!mbar_wait_cluster(tempty_bar, acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+        if (!mbar_wait_cluster(tempty_bar, acc_phase ^ 1u, abort_flag, p.wait_limit)) { ok = false; break; }
         tc_fence_after();
         // Lead-in: half 0 of the first K blocks while the epilogue still drains half 1.
         const int lead = two ? min(TCW_LEAD, tc.kblocks) : 0;
         int st = stage;
         uint32_t ph = phase;
         for (int kb = 0; kb < lead; ++kb) {
-          if (!mbar_wait_cluster(full_bar + 8 * st, ph, abort_flag)) { ok = false; break; }
+          if (!mbar_wait_cluster(full_bar + 8 * st, ph, abort_flag, p.wait_limit)) { ok = false; break; }
           tc_fence_after();
           issue(st, 0, kb == 0);
           if (++st == TCW_STAGES) { st = 0; ph ^= 1u; }
         }
         if (!ok) break;
-        if (!mbar_wait_cluster(tempty_bar + 8, acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+        if (!mbar_wait_cluster(tempty_bar + 8, acc_phase ^ 1u, abort_flag, p.wait_limit)) { ok = false; break; }
         tc_fence_after();
         for (int kb = 0; kb < tc.kblocks; ++kb) {
           if (kb >= lead) {
-            if (!mbar_wait_cluster(full_bar + 8 * stage, phase, abort_flag)) { ok = false; break; }
+            if (!mbar_wait_cluster(full_bar + 8 * stage, phase, abort_flag, p.wait_limit)) { ok = false; break; }
             tc_fence_after();
             issue(stage, 0, kb == 0);
           }
@@ -1057,14 +1073,10 @@ tc_grouped_gemm_pair_wide_kernel(const __grid_constant__ CUtensorMap mapA0, cons
       const bool two = tc.n0 + N_TILE_COLS < p.N;
       const long long obase = (long long)tc.e * p.out_bs + (long long)grow * p.ld_out + tc.n0;
       if (tc.kblocks == 0) {
-        if (row_ok) {
-          float z[32];
-#pragma unroll
-          for (int i = 0; i < 32; ++i) z[i] = 0.f;
+        if (row_ok)
           for (int hf = 0; hf < (two ? 2 : 1); ++hf)
             for (int c = c_beg; c < c_beg + NCH && tc.n0 + hf * N_TILE_COLS + 32 * c < p.N; ++c)
-              store32(p.out0 + obase + hf * N_TILE_COLS + 32 * c, z);
-        }
+              store_zero32(p, obase + hf * N_TILE_COLS + 32 * c);
         continue;
       }
       uint4 pg[4], pu[4];
@@ -1074,9 +1086,9 @@ tc_grouped_gemm_pair_wide_kernel(const __grid_constant__ CUtensorMap mapA0, cons
         load32_warp_issue(p.in0 + wb, p.ld_out, lane, nvalid, pg);
         load32_warp_issue(p.in1 + wb, p.ld_out, lane, nvalid, pu);
       }
-      if (!mbar_wait_cluster(tfull_bar, acc_phase, abort_flag)) { ok = false; break; }
+      if (!mbar_wait_cluster(tfull_bar, acc_phase, abort_flag, p.wait_limit)) { ok = false; break; }
       tc_fence_after();
-      if (EPI == TC_EPI_STORE) {
+      if (EPI == TC_EPI_STORE && !p.out_f32) {
         // Plain stores: empty each half into registers (packed bf16) and release it at once;
         // the turn through the scratch and the global stores follow while the MMAs run on.
         static_assert(EPI != TC_EPI_STORE || NCH == 4, "four chunks of 32 columns per warp and half");
@@ -1245,16 +1257,7 @@ static uint32_t make_idesc(int a_mn, int b_mn, int n, int m_instr = TC_BM) {
   return d;
 }
 
-static int sm_count() {
-  static int n = 0;
-  if (n == 0) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
-    if (n <= 0) n = 148;
-  }
-  return n;
-}
+static int sm_count() { return current_sm_count(); }
 
 template <int BN, int EPI>
 static etr_status tc_launch(const char* name, const CUtensorMap& a0, const CUtensorMap& a1,
@@ -1262,12 +1265,8 @@ static etr_status tc_launch(const char* name, const CUtensorMap& a0, const CUten
                             cudaStream_t st) {
   constexpr size_t smem = (size_t)TC_STAGES * (2 + BN / 64) * TC_BOX_BYTES + 1024 + 8 * TC_SCRATCH_BYTES;
   auto k = tc_grouped_gemm_kernel<BN, EPI>;
-  static bool attr_set = false;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-      return ETR_ERR_CUDA;
-    attr_set = true;
-  }
+  static std::atomic<unsigned long long> attr_done{0};      // one bit per device
+  if (!ensure_dyn_smem(k, smem, attr_done)) return ETR_ERR_CUDA;
   p.idesc = make_idesc(p.a_mn, p.b_mn, BN);
   const int grid = max_tiles < sm_count() ? (max_tiles < 1 ? 1 : max_tiles) : sm_count();
   ETR_TIME_BEGIN(name);
@@ -1282,12 +1281,8 @@ static etr_status tc_launch_pair_cfg(const char* name, const CUtensorMap& a0, co
                                  cudaStream_t st) {
   constexpr size_t smem = (size_t)TC2_STAGES * TC2_STAGE_BYTES + 1024 + 8 * TC_SCRATCH_BYTES;
   auto k = tc_grouped_gemm_pair_kernel<EPI, GATHER, CFG>;
-  static bool attr_set = false;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-      return ETR_ERR_CUDA;
-    attr_set = true;
-  }
+  static std::atomic<unsigned long long> attr_done{0};      // one bit per device
+  if (!ensure_dyn_smem(k, smem, attr_done)) return ETR_ERR_CUDA;
   p.idesc = make_idesc(p.a_mn, p.b_mn, 256, 256);
   const int pairs_max = sm_count() / 2;
   const int pairs = max_tiles < pairs_max ? (max_tiles < 1 ? 1 : max_tiles) : pairs_max;
@@ -1313,12 +1308,8 @@ static etr_status tc_launch_pair_wide_cfg(const char* name, const CUtensorMap& a
                                       cudaStream_t st) {
   constexpr size_t smem = (size_t)TCW_STAGES * TCW_STAGE_BYTES + 1024 + 8 * TC_SCRATCH_BYTES;
   auto k = tc_grouped_gemm_pair_wide_kernel<EPI, GATHER, CFG>;
-  static bool attr_set = false;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-      return ETR_ERR_CUDA;
-    attr_set = true;
-  }
+  static std::atomic<unsigned long long> attr_done{0};      // one bit per device
+  if (!ensure_dyn_smem(k, smem, attr_done)) return ETR_ERR_CUDA;
   p.idesc = make_idesc(p.a_mn, p.b_mn, 256, 256);
   const int pairs_max = sm_count() / 2;
   const int pairs = max_tiles < pairs_max ? (max_tiles < 1 ? 1 : max_tiles) : pairs_max;
@@ -1419,6 +1410,12 @@ static etr_status tc_run(TcForm form, const char* name, const CUtensorMap& a0, c
   return tc_launch<256, EPI>(name, a0, a1, b0, b1, p, max_tiles, st);
 }
 
+static TcParams tc_params(const etr_config* c) {
+  TcParams p = {};
+  p.wait_limit = c->wait_limit_cycles > 0 ? (long long)c->wait_limit_cycles : TC_WAIT_LIMIT_CYCLES;
+  return p;
+}
+
 size_t tc_workspace_bytes(const etr_config*) { return 0; }
 bool tc_available() { return true; }
 
@@ -1435,7 +1432,7 @@ etr_status tc_ffn_forward(const etr_config* c, const etr_route* rt, const void* 
   ETR_TRY(make_map(&mH, H, h, Cs, E));
   const int mt = Cs / TC_BM;
   {  // G, U, H = SwiGLU(Xp W1g^T, Xp W1u^T)
-    TcParams p = {};
+    TcParams p = tc_params(c);
     if (Xtok) { p.gather = 1; p.gather_ld = Cs; p.gather_oob = c->T; p.gather_idx = rt->slot_token; }
     p.dual_b = 1; p.M = Cs; p.N = h; p.K = d; p.dyn = TC_DYN_M; p.E = E; p.counts = rt->counts;
     p.out0 = (__nv_bfloat16*)G; p.out1 = (__nv_bfloat16*)U; p.out2 = (__nv_bfloat16*)H;
@@ -1444,7 +1441,7 @@ etr_status tc_ffn_forward(const etr_config* c, const etr_route* rt, const void* 
                                            E * mt * ceil_div(h, 128), st)));
   }
   {  // O = H W2^T
-    TcParams p = {};
+    TcParams p = tc_params(c);
     p.M = Cs; p.N = d; p.K = h; p.dyn = TC_DYN_M; p.E = E; p.counts = rt->counts;
     p.out0 = (__nv_bfloat16*)O; p.out_bs = (long long)Cs * d; p.ld_out = d; p.stats = stats;
     ETR_TRY((tc_run<TC_EPI_STORE>(tc_form_of(c, TC_EPI_STORE, p), "tc_gemm_down", mH, mH, mW2, mW2, p, E * mt * ceil_div(d, 256), st)));
@@ -1469,7 +1466,7 @@ etr_status tc_ffn_backward(const etr_config* c, const etr_route* rt, const void*
   ETR_TRY(make_map(&mW2, W2, h, d, E));
   const int mt = Cs / TC_BM;
   {  // dH = dO W2 (W2 read with its output index contiguous), then dG, dU
-    TcParams p = {};
+    TcParams p = tc_params(c);
     p.b_mn = 1; p.M = Cs; p.N = h; p.K = d; p.dyn = TC_DYN_M; p.E = E; p.counts = rt->counts;
     p.out0 = (__nv_bfloat16*)dG; p.out1 = (__nv_bfloat16*)dU;
     p.in0 = (const __nv_bfloat16*)G; p.in1 = (const __nv_bfloat16*)U;
@@ -1478,7 +1475,7 @@ etr_status tc_ffn_backward(const etr_config* c, const etr_route* rt, const void*
                                             E * mt * ceil_div(h, 256), st)));
   }
   {  // dXp = dG W1g + dU W1u: one contraction over 2h
-    TcParams p = {};
+    TcParams p = tc_params(c);
     p.b_mn = 1; p.k1_blocks = ceil_div(h, TC_BK); p.M = Cs; p.N = d; p.K = 2 * h; p.dyn = TC_DYN_M;
     p.E = E; p.counts = rt->counts;
     p.out0 = (__nv_bfloat16*)dXp; p.out_bs = (long long)Cs * d; p.ld_out = d; p.stats = stats;
@@ -1486,21 +1483,46 @@ etr_status tc_ffn_backward(const etr_config* c, const etr_route* rt, const void*
                                           E * mt * ceil_div(d, 256), st)));
   }
   {  // dW2 = dO^T H: contraction over the expert's rows, both operands MN-major
-    TcParams p = {};
+    TcParams p = tc_params(c);
     p.a_mn = 1; p.b_mn = 1; p.M = d; p.N = h; p.dyn = TC_DYN_K; p.E = E; p.counts = rt->counts;
     p.out0 = (__nv_bfloat16*)dW2; p.out_bs = (long long)d * h; p.ld_out = h; p.stats = stats;
+    p.out_f32 = c->grad_fp32 != 0;
     ETR_TRY((tc_run<TC_EPI_STORE>(tc_form_of(c, TC_EPI_STORE, p), "tc_gemm_dw2", mdO, mdO, mH, mH, p,
                                           E * ceil_div(d, TC_BM) * ceil_div(h, 256), st)));
   }
   for (int which = 0; which < 2; ++which) {  // dW1g = dG^T Xp, dW1u = dU^T Xp
-    TcParams p = {};
+    TcParams p = tc_params(c);
     p.a_mn = 1; p.b_mn = 1; p.M = h; p.N = d; p.dyn = TC_DYN_K; p.E = E; p.counts = rt->counts;
     if (Xtok) { p.gather = 2; p.gather_ld = Cs; p.gather_oob = c->T; p.gather_idx = rt->slot_token; }
     p.out0 = (__nv_bfloat16*)(which ? dW1u : dW1g); p.out_bs = (long long)h * d; p.ld_out = d; p.stats = stats;
+    p.out_f32 = c->grad_fp32 != 0;
     const CUtensorMap& ma = which ? mdU : mdG;
     ETR_TRY((tc_run<TC_EPI_STORE>(tc_form_of(c, TC_EPI_STORE, p), "tc_gemm_dw1", ma, ma, mXp, mXp, p,
                                           E * ceil_div(h, TC_BM) * ceil_div(d, 256), st)));
   }
+  return ETR_OK;
+}
+
+// The pipeline's bounded wait exercised on its own: thread 0 waits on an mbarrier that nothing ever
+// arrives on (no TMA, no tensor memory, nothing in flight), gives up after `limit` cycles and leaves
+// the code 0x7c08 in error_word, exactly as a GEMM kernel would; the kernel then returns normally.
+__global__ void __launch_bounds__(32) tc_wait_selftest_kernel(etr_stats* stats, long long limit) {
+  __shared__ __align__(8) uint64_t bar;
+  __shared__ int abort_flag_s;
+  if (threadIdx.x == 0) {
+    abort_flag_s = 0;
+    mbar_init(smem_u32(&bar), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncwarp();
+  if (threadIdx.x == 0 && !mbar_wait(smem_u32(&bar), 0u, &abort_flag_s, limit))
+    atomicExch(&stats->error_word, 0x7c08);
+}
+
+etr_status tc_wait_selftest(etr_stats* stats, long long limit, cudaStream_t st) {
+  ETR_TIME_BEGIN("tc_wait_selftest_kernel");
+  tc_wait_selftest_kernel<<<1, 32, 0, st>>>(stats, limit);
+  ETR_LAUNCH_CHECK();
   return ETR_OK;
 }
 

@@ -48,6 +48,10 @@ select_token_side_kernel(const float* __restrict__ delta, int32_t* __restrict__ 
     stats->delta_max = dm;
     stats->mode = p.mode;
     stats->C = capacity_from_delta(p, dm);
+    // the CSR kernels that follow on the stream add to these: every selection starts them at zero
+    stats->unrouted = 0;
+    stats->dropped = 0;
+    stats->rows_total = 0;
   }
   for (int tt = warp; tt < SEL_TB; tt += 8) {
     const int t = t0 + tt;
@@ -593,13 +597,8 @@ etr_status select_forward(const etr_config* c, const float* delta, etr_stats* st
   if (c->T >= 8192 && c->T <= 4 * 49152) {     // split each expert's row over a cluster of 4 CTAs
     constexpr int CL = 4;
     const size_t key_bytes = (size_t)((ceil_div(c->T, CL) + SEL_KPT - 1) / SEL_KPT * SEL_KPT) * sizeof(uint32_t);
-    static bool attr_set = false;
-    if (!attr_set) {
-      if (cudaFuncSetAttribute(select_expert_side_cluster_kernel<CL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                               196608) != cudaSuccess)
-        return ETR_ERR_CUDA;
-      attr_set = true;
-    }
+    static std::atomic<unsigned long long> attr_done{0};      // one bit per device
+    if (!ensure_dyn_smem(select_expert_side_cluster_kernel<CL>, 196608, attr_done)) return ETR_ERR_CUDA;
     cudaLaunchConfig_t lc = {};
     lc.gridDim = dim3(c->E * CL);
     lc.blockDim = dim3(1024);
@@ -656,11 +655,14 @@ static void* g_scratch_addr[64] = {};
 
 static etr_status select_scratch_address(void** out) {
   int dev = -1;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return ETR_ERR_CUDA;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { cudaGetLastError(); return ETR_ERR_CUDA; }
   std::lock_guard<std::mutex> lk(g_scratch_mu);
   if (g_scratch_addr[dev] == nullptr) {
     void* p = nullptr;
-    if (cudaGetSymbolAddress(&p, g_select_scratch) != cudaSuccess || p == nullptr) return ETR_ERR_CUDA;
+    if (cudaGetSymbolAddress(&p, g_select_scratch) != cudaSuccess || p == nullptr) {
+      cudaGetLastError();      // the failure is reported by the status; it must not stick to the next launch check
+      return ETR_ERR_CUDA;
+    }
     g_scratch_addr[dev] = p;
   }
   *out = g_scratch_addr[dev];
@@ -673,11 +675,15 @@ extern "C" etr_status etr_select_static(const etr_config* cfg, const float* delt
                                         const etr_route* route, void* stream) {
   using namespace etr;
   ETR_TRY(etr_validate(cfg));
+  // the same argument rules as etr_select
   if (delta == nullptr || stats == nullptr || route == nullptr) return ETR_ERR_ARG;
-  if (!route->topk_idx || !route->counts || !route->slot_token || !route->gate || !route->tok_ptr ||
-      !route->tok_row)
-    return ETR_ERR_ARG;
+  const void* ptrs[6] = {route->topk_idx, route->counts, route->slot_token, route->gate, route->tok_ptr,
+                         route->tok_row};
+  for (const void* q : ptrs)
+    if (q == nullptr) return ETR_ERR_ARG;
   if (!aligned16(delta) || !aligned16(stats)) return ETR_ERR_ALIGN;
+  for (const void* q : ptrs)
+    if (!aligned16(q)) return ETR_ERR_ALIGN;
   if ((unsigned long long)cfg->T * (unsigned long long)cfg->E > ETR_SELECT_STATIC_MAX_ENTRIES ||
       select_workspace_bytes(cfg) > SELECT_STATIC_MAX_BYTES)
     return ETR_ERR_WORKSPACE;

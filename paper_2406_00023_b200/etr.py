@@ -20,6 +20,7 @@ MODE_AUTO, MODE_TCR, MODE_ECR = 0, 1, 2
 GEMM_AUTO, GEMM_SIMT, GEMM_TCGEN05, GEMM_TCGEN05_2CTA, GEMM_TCGEN05_2CTA_WIDE = 0, 1, 2, 3, 4
 FUSE_AUTO, FUSE_OFF, FUSE_ON = 0, 1, 2
 GATE_AFFINITY, GATE_SOFTMAX = 0, 1
+THRESHOLD_OFF, THRESHOLD_EXPERT, THRESHOLD_TOKEN = 0, 1, 2
 
 EXPORTS = [
     "etr_status_string", "etr_validate", "etr_c_stride", "etr_workspace_bytes", "etr_buffers_bytes",
@@ -27,7 +28,7 @@ EXPORTS = [
     "etr_combine_bwd", "etr_expert_ffn_bwd", "etr_dispatch_bwd", "etr_select_bwd", "etr_affinity_bwd",
     "etr_gate_softmax", "etr_gate_softmax_bwd", "etr_affinity_bwd_dense", "etr_load_stats",
     "etr_layer_forward", "etr_layer_backward", "etr_layer_step_host", "etr_layer_step_host_begin",
-    "etr_layer_step_host_wait", "etr_read_stats",
+    "etr_layer_step_host_wait", "etr_read_stats", "etr_selftest_bounded_wait",
     "etr_launch_count", "etr_timing_enable", "etr_timing_collect",
 ]
 
@@ -38,7 +39,9 @@ class Config(C.Structure):
                 ("adaptive", C.c_int32), ("delta_max_override", C.c_float),
                 ("step", C.c_int64), ("switch_step", C.c_int64), ("mode", C.c_int32),
                 ("dtype", C.c_int32), ("gemm_impl", C.c_int32), ("fuse_dispatch", C.c_int32),
-                ("gate_mode", C.c_int32), ("reserved", C.c_int32)]
+                ("gate_mode", C.c_int32), ("grad_fp32", C.c_int32), ("weight_dtype", C.c_int32),
+                ("threshold_mode", C.c_int32), ("threshold_tau", C.c_float),
+                ("threshold_tau_token", C.c_float), ("wait_limit_cycles", C.c_int64)]
 
 
 class Stats(C.Structure):
@@ -126,11 +129,15 @@ def _stream():
 
 def make_config(*, T, d, D, E, k, h, capacity, dtype, mode=MODE_AUTO, step=0, switch_step=0,
                 adaptive=False, c_floor=1, delta_max_override=-1.0, gemm_impl=GEMM_AUTO,
-                fuse_dispatch=0, gate_mode=0) -> Config:
+                fuse_dispatch=0, gate_mode=0, grad_fp32=False, weight_dtype=None, threshold_mode=0,
+                threshold_tau=float("inf"), threshold_tau_token=float("inf"), wait_limit_cycles=0) -> Config:
     return Config(T=T, d=d, D=D, E=E, k=k, h=h, capacity=capacity, c_floor=c_floor,
                   adaptive=int(bool(adaptive)), delta_max_override=float(delta_max_override),
                   step=int(step), switch_step=int(switch_step), mode=int(mode), dtype=int(dtype),
-                  gemm_impl=int(gemm_impl), fuse_dispatch=int(fuse_dispatch), gate_mode=int(gate_mode), reserved=0)
+                  gemm_impl=int(gemm_impl), fuse_dispatch=int(fuse_dispatch), gate_mode=int(gate_mode),
+                  grad_fp32=int(bool(grad_fp32)), weight_dtype=int(dtype if weight_dtype is None else weight_dtype),
+                  threshold_mode=int(threshold_mode), threshold_tau=float(threshold_tau),
+                  threshold_tau_token=float(threshold_tau_token), wait_limit_cycles=int(wait_limit_cycles))
 
 
 def torch_dtype(cfg: Config):
@@ -212,6 +219,12 @@ def read_stats(stats_dev_ptr) -> Stats:
     code = lib().etr_read_stats(_p(stats_dev_ptr), C.byref(s), _stream())
     _check(code, "etr_read_stats")
     return s
+
+
+def selftest_bounded_wait(stats, limit_cycles: int):
+    """Launches the wait self-test: error_word of `stats` becomes non-zero after limit_cycles."""
+    _check(lib().etr_selftest_bounded_wait(_p(stats), C.c_int64(int(limit_cycles)), _stream()),
+           "etr_selftest_bounded_wait")
 
 
 # ---- stage calls (same names as the C ABI) -------------------------------------------------

@@ -23,14 +23,14 @@ def mode_of(w: gw.Workload) -> int:
 
 
 def make_cfg(w: gw.Workload, *, gemm_impl=etr.GEMM_AUTO, delta_max_override=-1.0, mode=None,
-             fuse_dispatch=etr.FUSE_AUTO, gate_mode=etr.GATE_AFFINITY):
+             fuse_dispatch=etr.FUSE_AUTO, gate_mode=etr.GATE_AFFINITY, **extra):
     m = mode_of(w) if mode is None else mode
     return etr.make_config(T=w.T, d=w.d, D=w.D, E=w.E, k=w.k, h=w.h, capacity=w.capacity,
                            dtype=etr.BF16 if w.dtype == "bf16" else etr.F32,
                            mode=etr.MODE_TCR if m == ob.MODE_TCR else etr.MODE_ECR,
                            step=w.step, switch_step=w.switch_step, adaptive=w.adaptive,
                            delta_max_override=delta_max_override, gemm_impl=gemm_impl,
-                           fuse_dispatch=fuse_dispatch, gate_mode=gate_mode)
+                           fuse_dispatch=fuse_dispatch, gate_mode=gate_mode, **extra)
 
 
 def to_dev(a: np.ndarray, w: gw.Workload | None = None, dtype=None):

@@ -1,0 +1,145 @@
+"""Behaviour the C ABI promises besides the numbers of the default path: fp32 weight gradients
+(grad_fp32), a selection that may be repeated on one stats block, and the bounded device-side
+wait, whose expiry must surface as ETR_ERR_TIMEOUT and leave the stream usable."""
+import numpy as np
+import pytest
+import torch
+
+from gen import workloads as gw
+from oracle import binding as ob
+from tests import harness as hz
+from tests.test_gpu_parity import case, override_of, run_select, routes_equal
+
+pytestmark = pytest.mark.gpu
+etr = hz.etr
+
+TC_FORMS = [etr.GEMM_AUTO, etr.GEMM_SIMT, etr.GEMM_TCGEN05, etr.GEMM_TCGEN05_2CTA, etr.GEMM_TCGEN05_2CTA_WIDE]
+
+
+@pytest.mark.parametrize("impl", TC_FORMS)
+@pytest.mark.parametrize("name", ["small_s", "mid_s", "sweep_s_ecr"])
+def test_fp32_weight_gradients(name, impl):
+    """grad_fp32: the three weight gradients leave the accumulators as fp32.  Fed with the
+    oracle's stage inputs on the bf16 grid, what is left is the summation order (fp32 against
+    double) and, for dW1, the kernel's own bf16 store of dG and dU in between; rounded to bf16 they
+    must reproduce the bf16 outputs of the default path bit for bit."""
+    w, inp, o, fw, bw = case(name)
+    dev = hz.upload(w, inp)
+    grid = gw.round_to_bf16
+    dOq, Gq, Uq, Hq = grid(bw.dO), grid(fw.G), grid(fw.U), grid(fw.H)
+    ref = o.expert_ffn_bwd(dOq, fw.Xp, Gq, Uq, Hq, fw.route, inp["W1g"], inp["W1u"], inp["W2"])
+    outs = {}
+    for g32 in (False, True):
+        cfg = hz.make_cfg(w, gemm_impl=impl, grad_fp32=g32)
+        buf = etr.LayerBuffers(cfg)
+        hz.upload_route(buf, fw.route)
+        buf.stats.zero_()
+        etr.dispatch(cfg, dev.X, buf.route, buf.Xp)
+        for nm, a in (("dO", dOq), ("G", Gq), ("U", Uq), ("H", Hq)):
+            getattr(buf, nm).copy_(hz.to_dev(a, w))
+        dt = torch.float32 if g32 else torch.bfloat16
+        dW = [torch.full(t.shape, float("nan"), dtype=dt, device="cuda") for t in (dev.W1g, dev.W1u, dev.W2)]
+        ws = torch.empty(etr.workspace_bytes(cfg), dtype=torch.uint8, device="cuda")
+        etr.expert_ffn_bwd(cfg, buf.route, buf.dO, buf.Xp, buf.G, buf.U, buf.H, dev.W1g, dev.W1u, dev.W2,
+                           buf.dG, buf.dU, buf.dXp, dW[0], dW[1], dW[2], buf.c.stats, ws)
+        assert buf.read_stats().error_word == 0
+        outs[g32] = dW
+    for j, nm in enumerate(("dW1g", "dW1u", "dW2")):
+        got32 = outs[True][j]
+        assert got32.dtype == torch.float32 and not bool(torch.isnan(got32).any())
+        assert torch.equal(got32.to(torch.bfloat16), outs[False][j]), f"{nm}: bf16(fp32 output) != bf16 output"
+    # dW2 = dO^T H from inputs on the grid: only the summation order is left
+    hz.assert_within(hz.to_np(outs[True][2]), ref[5], 2e-5, "dW2 fp32")
+    # dW1 = dG^T Xp with the kernel's stored (bf16) dG, dU: one store on the path
+    hz.assert_close_rms(hz.to_np(outs[True][0]), ref[3], 2e-2, "dW1g fp32", chain=1)
+    hz.assert_close_rms(hz.to_np(outs[True][1]), ref[4], 2e-2, "dW1u fp32", chain=1)
+
+
+def test_layer_with_fp32_weight_gradients():
+    """Whole layer with grad_fp32: the weight gradients lose their final rounding; everything
+    else is bit-identical to the default layer."""
+    w, inp, o, fw, bw = case("small_s")
+    dev = hz.upload(w, inp)
+    res = {}
+    for g32 in (False, True):
+        cfg = hz.make_cfg(w, grad_fp32=g32)
+        buf = etr.LayerBuffers(cfg)
+        dt = torch.float32 if g32 else torch.bfloat16
+        out = dict(Y=torch.empty_like(dev.X), dX=torch.empty_like(dev.X), dR=torch.empty_like(dev.R),
+                   dW1g=torch.empty(dev.W1g.shape, dtype=dt, device="cuda"),
+                   dW1u=torch.empty(dev.W1u.shape, dtype=dt, device="cuda"),
+                   dW2=torch.empty(dev.W2.shape, dtype=dt, device="cuda"))
+        etr.layer_forward(cfg, dev.X, dev.R, dev.W1g, dev.W1u, dev.W2, buf, out["Y"])
+        etr.layer_backward(cfg, dev.X, dev.R, dev.W1g, dev.W1u, dev.W2, dev.dY, buf, out["dX"], out["dR"],
+                           out["dW1g"], out["dW1u"], out["dW2"])
+        torch.cuda.synchronize()
+        assert buf.read_stats().error_word == 0
+        res[g32] = out
+    for k in ("Y", "dX", "dR"):
+        assert torch.equal(res[False][k], res[True][k]), k
+    for k, chain in (("dW1g", 5), ("dW1u", 5), ("dW2", 3)):
+        assert torch.equal(res[True][k].to(torch.bfloat16), res[False][k]), k
+        hz.assert_close_rms(hz.to_np(res[True][k]), getattr(bw, k), 2e-2, k + " fp32", chain=chain)
+
+
+@pytest.mark.parametrize("name", ["small_s", "sweep_s_ecr"])
+def test_select_may_be_repeated_on_one_stats_block(name):
+    """The selection sets every counter it reports: a second selection on the same stats (another
+    step or capacity of a sweep, with delta_max_key left in place by etr_affinity) must give what
+    a selection on fresh stats gives."""
+    w, inp, o, fw, _ = case(name)
+    ov = override_of(name)
+    cfg = hz.make_cfg(w, delta_max_override=ov)
+    buf, first = run_select(w, cfg, fw.delta)
+    assert routes_equal(fw.route, first)
+    ws = torch.empty(etr.workspace_bytes(cfg), dtype=torch.uint8, device="cuda")
+    # again, and then once more with the other mode and a smaller capacity, never clearing stats
+    etr.select(cfg, buf.delta, buf.c.stats, buf.route, ws)
+    assert routes_equal(fw.route, hz.route_from_buffers(buf, cfg))
+    other = ob.MODE_ECR if hz.mode_of(w) == ob.MODE_TCR else ob.MODE_TCR
+    w2 = gw.scaled(w, cf=w.cf / 2, adaptive=False)
+    cfg2 = hz.make_cfg(w2, mode=other)
+    buf2 = etr.LayerBuffers(cfg2)
+    buf2.delta.copy_(buf.delta)
+    buf2.stats.copy_(buf.stats)                   # carries the first selection's counters
+    etr.select(cfg2, buf2.delta, buf2.c.stats, buf2.route, ws)
+    ref2 = o.select(fw.delta, w.k, other, w2.capacity, w2.C_stride)
+    assert routes_equal(ref2, hz.route_from_buffers(buf2, cfg2))
+    etr.select_static(cfg2, buf2.delta, buf2.c.stats, buf2.route)
+    assert routes_equal(ref2, hz.route_from_buffers(buf2, cfg2))
+
+
+def test_bounded_wait_expires_as_a_status_and_the_stream_stays_usable():
+    """The failure path of the GEMM pipeline without a failure: a one-warp kernel waits, with the
+    pipeline's wait routine and a limit of 1e5 cycles (about 50 microseconds), on a barrier nothing
+    arrives on.  The kernel must return by itself, etr_read_stats must report ETR_ERR_TIMEOUT, and
+    an ordinary layer call on the same stream and buffers must then pass as usual."""
+    w, inp, o, fw, bw = case("small_s")
+    cfg = hz.make_cfg(w)
+    dev = hz.upload(w, inp)
+    buf = etr.LayerBuffers(cfg)
+    buf.stats.zero_()
+    t0 = torch.cuda.Event(enable_timing=True)
+    t1 = torch.cuda.Event(enable_timing=True)
+    t0.record()
+    etr.selftest_bounded_wait(buf.c.stats, 100_000)
+    t1.record()
+    with pytest.raises(etr.EtrError) as e:
+        buf.read_stats()
+    assert e.value.code == etr.ERR_TIMEOUT
+    assert int(buf.stats[6].item()) == 0x7c08
+    assert t0.elapsed_time(t1) < 50.0, "the wait did not end near its limit"
+    with pytest.raises(etr.EtrError) as e:
+        etr.selftest_bounded_wait(buf.c.stats, 0)
+    assert e.value.code == etr.ERR_ARG
+    # the next ordinary call: same stream, same buffers; etr_layer_forward clears the stats
+    Y = torch.empty_like(dev.X)
+    etr.layer_forward(cfg, dev.X, dev.R, dev.W1g, dev.W1u, dev.W2, buf, Y)
+    st = buf.read_stats()
+    assert st.error_word == 0
+    hz.assert_close_rms(hz.to_np(Y), fw.Y, 2e-2, "Y after an expired wait", chain=4)
+    # a limit passed through the config reaches the GEMM kernels; a generous one changes nothing
+    cfg_l = hz.make_cfg(w, wait_limit_cycles=2_000_000_000)
+    Y2 = torch.empty_like(dev.X)
+    etr.layer_forward(cfg_l, dev.X, dev.R, dev.W1g, dev.W1u, dev.W2, buf, Y2)
+    assert buf.read_stats().error_word == 0 and torch.equal(Y, Y2)

@@ -34,9 +34,16 @@ def _affinities(w, seed):
     return (torch.randn(w.T, w.E, generator=g, device="cuda") / np.sqrt(w.d)).contiguous()
 
 
+# T = 3000: one CTA per expert; T = 12000: each expert's keys split over a cluster of four CTAs;
+# T = 65536 with E = 64 fills the fixed array to its last entry (the largest problem accepted).
+SHAPES = [dict(T=3000), dict(T=12000), dict(T=65536, E=64, d=4096, D=16)]
+
+
+@pytest.mark.parametrize("shape", SHAPES, ids=lambda s: f"T{s['T']}")
 @pytest.mark.parametrize("mode", [etr.MODE_TCR, etr.MODE_ECR])
-def test_select_static_matches_select_on_two_calls_in_a_row(mode):
-    w = gw.scaled(gw.WORKLOADS["small"], T=3000)
+def test_select_static_matches_select_on_two_calls_in_a_row(mode, shape):
+    w = gw.scaled(gw.WORKLOADS["small"], **shape)
+    assert w.T * w.E <= etr.SELECT_STATIC_MAX_ENTRIES
     cfg = etr.make_config(T=w.T, d=w.d, D=w.D, E=w.E, k=w.k, h=w.h, capacity=w.capacity,
                           dtype=etr.BF16, mode=mode)
     ws = torch.empty(etr.workspace_bytes(cfg), dtype=torch.uint8, device="cuda")
@@ -68,4 +75,11 @@ def test_select_static_rejects_problems_beyond_its_fixed_scratch():
     with pytest.raises(etr.EtrError) as e:
         etr.select_static(too_big, dummy, dummy, route)
     assert e.value.code == etr.ERR_WORKSPACE
+    assert etr.launch_count() == n0
+    # the same argument rules as etr_select: a route pointer off its 16-byte alignment is refused
+    ok = etr.make_config(T=3000, d=1024, D=8, E=16, k=2, h=2816, capacity=469, dtype=etr.BF16, mode=etr.MODE_ECR)
+    bad_route = etr.Route(*([dummy.data_ptr()] * 5 + [dummy.data_ptr() + 4]))
+    with pytest.raises(etr.EtrError) as e:
+        etr.select_static(ok, dummy, dummy, bad_route)
+    assert e.value.code == etr.ERR_ALIGN
     assert etr.launch_count() == n0
