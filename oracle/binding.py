@@ -112,6 +112,26 @@ class Oracle:
         r.dropped, r.unrouted = int(dropped[0]), int(unrouted[0])
         return r
 
+    def select_thresholded(self, delta, k, mode, C, C_stride, threshold_mode, tau_expert=float("inf"),
+                           tau_token=float("inf")):
+        """select() with the cut by a running sum of affinities (bit 0: expert side, bit 1: token side)."""
+        delta = self.arr(delta)
+        T, E = delta.shape
+        r = SimpleNamespace(
+            topk_idx=np.empty((T, k), np.int32), counts=np.empty(E, np.int32),
+            slot_token=np.empty(E * C_stride, np.int32), gate=np.empty(E * C_stride, self.np),
+            tok_ptr=np.empty(T + 1, np.int32), tok_row=np.full(E * C_stride, -1, np.int32),
+            C=int(C), C_stride=int(C_stride), mode=int(mode), E=E, T=T, k=k)
+        dropped = np.zeros(1, np.int32)
+        unrouted = np.zeros(1, np.int32)
+        f = self._f("select_thresholded")
+        f.argtypes = [ctypes.c_int] * 7 + [ctypes.c_double] * 2 + [ctypes.c_void_p] * 9
+        f(T, E, k, int(mode), int(C), int(C_stride), int(threshold_mode), float(tau_expert), float(tau_token),
+          _p(delta), _p(r.topk_idx), _p(r.counts), _p(r.slot_token), _p(r.gate), _p(r.tok_ptr), _p(r.tok_row),
+          _p(dropped), _p(unrouted))
+        r.dropped, r.unrouted = int(dropped[0]), int(unrouted[0])
+        return r
+
     def dispatch(self, X, route):
         X = self.arr(X)
         d = X.shape[1]
@@ -243,7 +263,7 @@ class Oracle:
     # -- the whole layer: the stages above in order ---------------------------------------
     def forward(self, X, R, W1g, W1u, W2, *, D, k, capacity, C_stride=None, mode=None, step=0,
                 switch_step=0, adaptive=False, c_floor=1, delta_max_override=-1.0, route=None,
-                softmax_gate=False):
+                softmax_gate=False, threshold_mode=0, tau_expert=float("inf"), tau_token=float("inf")):
         d = X.shape[1]
         E = R.shape[0]
         if C_stride is None:
@@ -254,7 +274,10 @@ class Oracle:
                 mode = mode_for_step(step, switch_step)
             dstar = float(dmax) if delta_max_override < 0 else float(delta_max_override)
             C = capacity_bound(d, E, capacity, c_floor, adaptive, dstar)
-            route = self.select(delta, k, mode, C, C_stride)
+            if threshold_mode:
+                route = self.select_thresholded(delta, k, mode, C, C_stride, threshold_mode, tau_expert, tau_token)
+            else:
+                route = self.select(delta, k, mode, C, C_stride)
             gate = route.gate
         else:  # frozen selection: gates re-read from this call's affinities
             gate = np.zeros(E * route.C_stride, self.np)

@@ -27,7 +27,9 @@
 // threshold), the source of delta_max (batch maximum), the clamp of C_min into
 // [c_floor, capacity], and the raw-affinity gate; the paper under-specifies these.  The
 // softmax-gate variant and the load statistics are pinned by library softmax / autograd, finite
-// differences and closed forms.
+// differences and closed forms.  The threshold on the sum of affinity scores (select_thresholded)
+// is a reading of a rule the paper names without stating: parity unpinned as a reading, the
+// function pinned by brute force over prefixes, its two limits and monotonicity.
 #pragma once
 #include <algorithm>
 #include <cmath>
@@ -141,6 +143,95 @@ void select(int T, int E, int k, int mode, int C, int C_stride, const S* delta,
       return delta[(size_t)a * E + i] > delta[(size_t)b * E + i];
     });
     const int n = std::min<int>(C, (int)cand.size());
+    std::vector<int32_t> keep(cand.begin(), cand.begin() + n);
+    std::sort(keep.begin(), keep.end());
+    counts[i] = n;
+    kept += n;
+    for (int p = 0; p < n; ++p) {
+      const size_t r = (size_t)i * C_stride + p;
+      slot_token[r] = keep[p];
+      gate[r] = delta[(size_t)keep[p] * E + i];
+      rows_of[keep[p]].push_back((int32_t)r);
+    }
+  }
+  int32_t un = 0, pos = 0;
+  for (int t = 0; t < T; ++t) {
+    tok_ptr[t] = pos;
+    for (int32_t r : rows_of[t]) tok_row[pos++] = r;
+    if (rows_of[t].empty()) ++un;
+  }
+  tok_ptr[T] = pos;
+  if (dropped) *dropped = (int32_t)(n_cand - kept);
+  if (unrouted) *unrouted = un;
+}
+
+// ---- selection with a threshold on the sum of affinity scores ------------------------------
+// "Routing Strategy" says that the number l of tokens an expert takes "is determined by a
+// threshold of the sum of affinity scores", and "Training Strategy" that the number of tokens per
+// expert follows an adaptive threshold; neither gives the rule.  The reading implemented here
+// (parity unpinned as a reading; the function itself is pinned by brute force over prefixes, by
+// its limits tau = +infinity and tau <= first score, and by monotonicity in tau):
+//
+//   walk a candidate list in descending affinity (ties: lower index first); the candidate of
+//   rank j (1-based) is kept while j is within the cap (C for an expert's tokens, k for a
+//   token's experts) and the sum of the j-1 affinities before it is still below tau.
+//
+// threshold_mode bit 0 (expert side): applied to every expert's candidate tokens, in both modes.
+// threshold_mode bit 1 (token side): applied to every token's Top-k experts in token choice, so a
+// token takes between 0 and k experts; topk_idx holds -1 in the unused places.
+// The sums are taken on affinities quantised to multiples of 2^-32, q(delta) = round-to-nearest
+// (delta * 2^32), as 64-bit integers, and tau is quantised the same way, so that the decision does
+// not depend on the order of summation; both sides of a parity test take it in this arithmetic.
+inline int64_t quantise_affinity(double v) {
+  const double s = v * 4294967296.0;
+  if (!(s < 9.2e18)) return std::numeric_limits<int64_t>::max();       // +infinity (or NaN): never reached
+  if (s < -9.2e18) return std::numeric_limits<int64_t>::min();
+  return (int64_t)std::llrint(s);
+}
+
+template <class S>
+void select_thresholded(int T, int E, int k, int mode, int C, int C_stride, int threshold_mode,
+                        double tau_expert, double tau_token, const S* delta, int32_t* topk_idx,
+                        int32_t* counts, int32_t* slot_token, S* gate, int32_t* tok_ptr,
+                        int32_t* tok_row, int32_t* dropped, int32_t* unrouted) {
+  const bool cut_expert = (threshold_mode & 1) != 0, cut_token = (threshold_mode & 2) != 0;
+  const int64_t tq_expert = quantise_affinity(tau_expert), tq_token = quantise_affinity(tau_token);
+  std::vector<std::vector<int32_t>> L(E);
+  long n_cand = 0;
+  for (int t = 0; t < T; ++t) {
+    if (mode == MODE_TCR) {
+      std::vector<int32_t> order(E);
+      std::iota(order.begin(), order.end(), 0);
+      const S* row = delta + (size_t)t * E;
+      std::stable_sort(order.begin(), order.end(),
+                       [row](int32_t a, int32_t b) { return row[a] > row[b]; });
+      int64_t sum_before = 0;
+      for (int j = 0; j < k; ++j) {
+        const bool keep = !cut_token || sum_before < tq_token;
+        topk_idx[(size_t)t * k + j] = keep ? order[j] : -1;
+        if (keep) { L[order[j]].push_back(t); ++n_cand; }
+        sum_before += quantise_affinity((double)row[order[j]]);
+      }
+    } else {
+      for (int j = 0; j < k; ++j) topk_idx[(size_t)t * k + j] = -1;
+      for (int i = 0; i < E; ++i) L[i].push_back(t);
+      n_cand += E;
+    }
+  }
+  for (size_t r = 0; r < (size_t)E * C_stride; ++r) { slot_token[r] = -1; gate[r] = (S)0; }
+  std::vector<std::vector<int32_t>> rows_of(T);
+  long kept = 0;
+  for (int i = 0; i < E; ++i) {
+    std::vector<int32_t>& cand = L[i];              // ascending token id by construction
+    std::stable_sort(cand.begin(), cand.end(), [delta, E, i](int32_t a, int32_t b) {
+      return delta[(size_t)a * E + i] > delta[(size_t)b * E + i];
+    });
+    int n = 0;
+    int64_t sum_before = 0;
+    while (n < (int)cand.size() && n < C && (!cut_expert || sum_before < tq_expert)) {
+      sum_before += quantise_affinity((double)delta[(size_t)cand[n] * E + i]);
+      ++n;
+    }
     std::vector<int32_t> keep(cand.begin(), cand.begin() + n);
     std::sort(keep.begin(), keep.end());
     counts[i] = n;

@@ -20,6 +20,13 @@ using namespace etr_oracle;
     select<S>(T, E, k, mode, C, C_stride, delta, topk_idx, counts, slot_token, gate, tok_ptr,        \
               tok_row, dropped, unrouted);                                                           \
   }                                                                                                  \
+  extern "C" void etr_oracle_select_thresholded_##SUF(                                               \
+      int T, int E, int k, int mode, int C, int C_stride, int threshold_mode, double tau_expert,     \
+      double tau_token, const S* delta, int32_t* topk_idx, int32_t* counts, int32_t* slot_token,     \
+      S* gate, int32_t* tok_ptr, int32_t* tok_row, int32_t* dropped, int32_t* unrouted) {            \
+    select_thresholded<S>(T, E, k, mode, C, C_stride, threshold_mode, tau_expert, tau_token, delta,  \
+                          topk_idx, counts, slot_token, gate, tok_ptr, tok_row, dropped, unrouted);  \
+  }                                                                                                  \
   extern "C" void etr_oracle_dispatch_##SUF(int E, int C_stride, int d, const S* X,                  \
                                             const int32_t* slot_token, S* Xp) {                      \
     dispatch<S>(E, C_stride, d, X, slot_token, Xp);                                                  \

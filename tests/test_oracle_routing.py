@@ -305,3 +305,120 @@ def test_select_reductions(o32):
     # expert choice with C = T: every pair selected
     rt = o32.select(delta, w.k, ob.MODE_ECR, w.T, 512)
     assert np.all(rt.counts == w.T) and np.all(np.diff(rt.tok_ptr) == w.E)
+
+
+# ------------------------------------------ threshold on the sum of affinity scores ------------
+# The rule ("Routing Strategy": the number of tokens an expert takes follows a threshold of the sum
+# of affinity scores) is pinned without restating its loop: by exhaustive search over prefix
+# lengths in exact rational arithmetic, by its two limits, by a closed form on constant scores and
+# by monotonicity in tau.
+
+ROUTE_FIELDS = ("topk_idx", "counts", "slot_token", "gate", "tok_ptr", "tok_row")
+
+
+def same_route(a, b):
+    return all(np.array_equal(getattr(a, f), getattr(b, f)) for f in ROUTE_FIELDS) and \
+        a.dropped == b.dropped and a.unrouted == b.unrouted
+
+
+@pytest.mark.parametrize("mode", [ob.MODE_TCR, ob.MODE_ECR])
+@pytest.mark.parametrize("flags", [1, 2, 3])
+def test_threshold_at_infinity_is_the_plain_selection(o32, mode, flags):
+    delta = (rand((300, 8), 21) / 16).astype(np.float32)
+    for C in (1, 17, 300):
+        assert same_route(o32.select(delta, 2, mode, C, 384),
+                          o32.select_thresholded(delta, 2, mode, C, 384, flags))
+
+
+@pytest.mark.parametrize("mode", [ob.MODE_TCR, ob.MODE_ECR])
+def test_threshold_below_the_first_score_keeps_one_and_nonpositive_keeps_none(o32, mode):
+    delta = np.abs(rand((200, 6), 22) / 8).astype(np.float32) + np.float32(0.01)      # all positive
+    plain1 = o32.select(delta, 2, mode, 1, 128)              # capacity 1: each expert's best candidate
+    tiny = o32.select_thresholded(delta, 2, mode, 50, 128, 1, tau_expert=1e-6)
+    assert np.array_equal(tiny.counts, plain1.counts) and np.array_equal(tiny.slot_token, plain1.slot_token)
+    for tau in (0.0, -1.0):
+        none = o32.select_thresholded(delta, 2, mode, 50, 128, 1, tau_expert=tau)
+        assert np.all(none.counts == 0) and none.unrouted == 200 and none.tok_ptr[-1] == 0
+    # token side: a token whose first affinity already reaches tau takes that expert only
+    one = o32.select_thresholded(delta, 3, ob.MODE_TCR, 200, 256, 2, tau_token=1e-6)
+    top = o32.select(delta, 1, ob.MODE_TCR, 200, 256)
+    assert np.array_equal(one.topk_idx[:, 0], top.topk_idx[:, 0]) and np.all(one.topk_idx[:, 1:] == -1)
+    assert np.array_equal(one.counts, top.counts) and np.array_equal(one.slot_token, top.slot_token)
+
+
+@pytest.mark.parametrize("seed", range(6))
+@pytest.mark.parametrize("mode", [ob.MODE_TCR, ob.MODE_ECR])
+def test_threshold_bruteforce_over_prefixes(o64, mode, seed):
+    """Scores are multiples of 1/64, so sums are exact both as 2^-32 integers and as fractions.
+    For every expert, among all prefix lengths n of its candidate list in (score descending, token
+    ascending) order, the answer is the longest n <= C all of whose proper prefixes (lengths
+    0..n-1) sum to less than tau."""
+    from fractions import Fraction
+    rng = np.random.default_rng(100 + seed)
+    T, E, k, C = 12, 3, 2, 7
+    delta = rng.integers(-20, 40, size=(T, E)) / 64.0
+    tau = Fraction(int(rng.integers(1, 200)), 64)
+    got = o64.select_thresholded(delta, k, mode, C, 128, 1, tau_expert=float(tau))
+    plain = o64.select(delta, k, mode, T, 128)               # no cut: each expert's full candidate list
+    for i in range(E):
+        cand = plain.slot_token[i * 128:i * 128 + plain.counts[i]]
+        order = sorted(cand, key=lambda t: (-delta[t, i], t))
+        best = 0
+        for n in range(0, min(C, len(order)) + 1):
+            sums = [sum((Fraction(delta[t, i]) for t in order[:j]), Fraction(0)) for j in range(n)]
+            if all(s < tau for s in sums):
+                best = n
+        assert got.counts[i] == best
+        assert sorted(order[:best]) == list(got.slot_token[i * 128:i * 128 + best])
+
+
+def test_threshold_closed_form_on_constant_scores(o32):
+    """All affinities equal to a = 1/8: an expert keeps min(C, T, ceil(tau / a)) tokens, lowest ids first."""
+    T, E, C = 40, 4, 30
+    delta = np.full((T, E), 0.125, np.float32)
+    for tau, want in ((0.1, 1), (0.125, 1), (0.126, 2), (1.0, 8), (1.01, 9), (3.75, 30), (100.0, 30)):
+        r = o32.select_thresholded(delta, 2, ob.MODE_ECR, C, 128, 1, tau_expert=tau)
+        assert np.all(r.counts == want), (tau, r.counts)
+        assert np.array_equal(r.slot_token[:want], np.arange(want))
+    # token side, k = 4 experts of affinity 1/8 each: ceil(tau / a) experts, capped by k
+    for tau, want in ((0.125, 1), (0.2, 2), (0.4, 4), (9.0, 4)):
+        r = o32.select_thresholded(delta, 4, ob.MODE_TCR, T, 128, 2, tau_token=tau)
+        assert np.all((r.topk_idx >= 0).sum(1) == want)
+        assert np.array_equal(r.topk_idx[0, :want], np.arange(want))
+
+
+@pytest.mark.parametrize("mode", [ob.MODE_TCR, ob.MODE_ECR])
+def test_threshold_is_monotone_and_keeps_a_prefix(o32, mode):
+    delta = (rand((500, 8), 23) / 12).astype(np.float32)     # mixed signs
+    C, Cs = 90, 128
+    prev = None
+    full = o32.select(delta, 2, mode, 500, 512)
+    for tau in (0.05, 0.3, 1.0, 2.5, 6.0, 1e9):
+        r = o32.select_thresholded(delta, 2, mode, C, Cs, 1, tau_expert=tau)
+        assert np.all(r.counts <= C)
+        for i in range(8):
+            kept = set(r.slot_token[i * Cs:i * Cs + r.counts[i]])
+            cand = full.slot_token[i * 512:i * 512 + full.counts[i]]
+            order = sorted(cand, key=lambda t: (-delta[t, i], t))
+            assert kept == set(order[:r.counts[i]])          # a prefix of the ranked candidates
+            if prev is not None:
+                assert prev[i] <= kept                       # grows with tau
+        prev = [set(r.slot_token[i * Cs:i * Cs + r.counts[i]]) for i in range(8)]
+    assert same_route(r, o32.select(delta, 2, mode, C, Cs))  # a huge tau is no cut at all
+
+
+def test_threshold_sum_does_not_depend_on_float_summation_order(o32):
+    """Scores whose float sum depends on the order (1/3-like values of mixed size): the decision is
+    taken on 2^-32 integers, so it equals the one computed with Python integers."""
+    rng = np.random.default_rng(9)
+    T = 4000
+    delta = (rng.random((T, 1)) * 0.3 + 1e-4).astype(np.float32)
+    tau = 57.123
+    r = o32.select_thresholded(delta, 1, ob.MODE_ECR, T, 4096, 1, tau_expert=tau)
+    q = [int(round(float(v) * 2 ** 32)) for v in delta[:, 0]]          # exact: float * 2^32 is an integer or a dyadic
+    order = sorted(range(T), key=lambda t: (-q[t], t))
+    tq, s, n = int(round(tau * 2 ** 32)), 0, 0
+    while n < T and s < tq:
+        s += q[order[n]]
+        n += 1
+    assert r.counts[0] == n
