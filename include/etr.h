@@ -208,7 +208,7 @@ etr_status etr_select(const etr_config* cfg, const float* delta, etr_stats* stat
  * the route outputs as usual, and the T*E 32-bit keys that etr_select keeps in `ws` live
  * instead in a fixed array inside the library image.
  *
- * Limit: T*E <= ETR_SELECT_STATIC_MAX_ENTRIES (16 MiB of keys plus 64 KiB of scan scratch,
+ * Limit: T*E <= ETR_SELECT_STATIC_MAX_ENTRIES (16 MiB of keys plus 640 KiB of scan scratch,
  * enough for every workload up to T=65536, E=64); larger problems return ETR_ERR_WORKSPACE
  * and launch nothing.  Every GPU that loads the library carries those bytes until the process
  * ends.

@@ -206,10 +206,11 @@ void select_thresholded(int T, int E, int k, int mode, int C, int C_stride, int 
       std::stable_sort(order.begin(), order.end(),
                        [row](int32_t a, int32_t b) { return row[a] > row[b]; });
       int64_t sum_before = 0;
+      bool open = true;                               // the walk stops at the first rank it does not keep
       for (int j = 0; j < k; ++j) {
-        const bool keep = !cut_token || sum_before < tq_token;
-        topk_idx[(size_t)t * k + j] = keep ? order[j] : -1;
-        if (keep) { L[order[j]].push_back(t); ++n_cand; }
+        open = open && (!cut_token || sum_before < tq_token);
+        topk_idx[(size_t)t * k + j] = open ? order[j] : -1;
+        if (open) { L[order[j]].push_back(t); ++n_cand; }
         sum_before += quantise_affinity((double)row[order[j]]);
       }
     } else {

@@ -23,7 +23,21 @@ constexpr int SEL_MAX_EPL = 8;     // experts per lane: E <= 256
 struct SelectParams {
   int T, E, k, d, C_stride, capacity, c_floor, adaptive, mode;
   float delta_max_override;
+  int cut_token;              // token choice: a token stops taking experts once the sum of the taken affinities reaches tq_token
+  long long tq_token;         // threshold on 2^-32 integers
 };
+
+// Affinity as a multiple of 2^-32 (round to nearest even): the unit the threshold sums are taken in,
+// so that they are exact and independent of the order of summation.
+__device__ __forceinline__ long long quantise_affinity(float delta) {
+  return __double2ll_rn((double)delta * 4294967296.0);
+}
+static long long quantise_threshold(float tau) {
+  const double s = (double)tau * 4294967296.0;
+  if (!(s < 9.2e18)) return 0x7fffffffffffffffll;        // +infinity: never reached
+  if (s < -9.2e18) return (long long)0x8000000000000000ull;
+  return llrint(s);
+}
 
 // C = capacity, or clamp(ceil((1/E) exp{d dm^2/(2-dm^2)}), c_floor, capacity).
 __device__ inline int capacity_from_delta(const SelectParams& p, float delta_max) {
@@ -38,10 +52,15 @@ __device__ inline int capacity_from_delta(const SelectParams& p, float delta_max
 
 __global__ void __launch_bounds__(256)
 select_token_side_kernel(const float* __restrict__ delta, int32_t* __restrict__ topk_idx,
-                         uint32_t* __restrict__ keyT, etr_stats* stats, SelectParams p) {
+                         uint32_t* __restrict__ keyT, etr_stats* stats, int32_t* __restrict__ skipped,
+                         SelectParams p) {
   __shared__ uint32_t tile[256 * (SEL_TB + 1)];      // [E][33]
+  __shared__ int s_skipped;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int t0 = blockIdx.x * SEL_TB;
+  if (tid == 0) s_skipped = 0;
+  if (p.cut_token) __syncthreads();
+  int n_skipped = 0;                                 // ranks this warp's tokens gave up (lane 0 counts)
   if (blockIdx.x == 0 && tid == 0) {
     const uint32_t mk = stats->delta_max_key;
     const float dm = mk ? key_to_float(mk) : 0.f;
@@ -56,21 +75,24 @@ select_token_side_kernel(const float* __restrict__ delta, int32_t* __restrict__ 
   for (int tt = warp; tt < SEL_TB; tt += 8) {
     const int t = t0 + tt;
     uint32_t key[SEL_MAX_EPL];
-    bool cand[SEL_MAX_EPL];
+    bool cand[SEL_MAX_EPL], taken[SEL_MAX_EPL];
 #pragma unroll
     for (int u = 0; u < SEL_MAX_EPL; ++u) {
       const int i = lane + 32 * u;
       key[u] = (t < p.T && i < p.E) ? ordered_key(delta[(size_t)t * p.E + i]) : 0u;
       cand[u] = (p.mode == ETR_MODE_ECR);
+      taken[u] = false;
     }
     if (p.mode == ETR_MODE_TCR && t < p.T) {
+      long long sum_before = 0;                      // of the affinities of the ranks before j (threshold walk)
+      bool open = true;
       for (int j = 0; j < p.k; ++j) {
         // arg-max over (key, lower index wins) among experts not yet taken
         unsigned long long best = 0ull;
 #pragma unroll
         for (int u = 0; u < SEL_MAX_EPL; ++u) {
           const int i = lane + 32 * u;
-          if (i < p.E && !cand[u]) {
+          if (i < p.E && !taken[u]) {
             const unsigned long long v = ((unsigned long long)key[u] << 32) | (uint32_t)(0x7fffffff - i);
             best = v > best ? v : best;
           }
@@ -81,11 +103,16 @@ select_token_side_kernel(const float* __restrict__ delta, int32_t* __restrict__ 
           best = other > best ? other : best;
         }
         const int win = 0x7fffffff - (int)(uint32_t)(best & 0xffffffffull);
+        if (p.cut_token) {                           // the walk stops at the first rank it does not keep
+          open = open && sum_before < p.tq_token;
+          sum_before += quantise_affinity(key_to_float((uint32_t)(best >> 32)));
+          n_skipped += !open;
+        }
         if (lane == (win & 31)) {
 #pragma unroll
-          for (int u = 0; u < SEL_MAX_EPL; ++u) if (u == (win >> 5)) cand[u] = true;
+          for (int u = 0; u < SEL_MAX_EPL; ++u) if (u == (win >> 5)) { taken[u] = true; cand[u] = open; }
         }
-        if (lane == 0) topk_idx[(size_t)t * p.k + j] = win;
+        if (lane == 0) topk_idx[(size_t)t * p.k + j] = open ? win : -1;
       }
     } else if (t < p.T) {
       for (int j = lane; j < p.k; j += 32) topk_idx[(size_t)t * p.k + j] = -1;
@@ -96,7 +123,9 @@ select_token_side_kernel(const float* __restrict__ delta, int32_t* __restrict__ 
       if (i < p.E) tile[i * (SEL_TB + 1) + tt] = cand[u] ? key[u] : 0u;
     }
   }
+  if (p.cut_token && lane == 0 && n_skipped) atomicAdd(&s_skipped, n_skipped);
   __syncthreads();
+  if (tid == 0 && skipped) skipped[blockIdx.x] = s_skipped;        // candidates given up by this block's tokens
   for (int idx = tid; idx < p.E * SEL_TB; idx += 256) {
     const int i = idx / SEL_TB, tt = idx % SEL_TB;
     if (t0 + tt < p.T) keyT[(size_t)i * p.T + t0 + tt] = tile[i * (SEL_TB + 1) + tt];
@@ -148,6 +177,88 @@ __device__ __forceinline__ void pick_bin(const uint32_t* hist, uint32_t rem, int
   rem_out = __shfl_sync(0xffffffffu, r, owner);
 }
 
+// Expert-side threshold: limit[i] = how many of expert i's candidates, taken in descending affinity,
+// it takes before the running sum of their affinities (2^-32 integers) reaches tq; INT_MAX if it
+// never does.  The candidate of rank j is kept while the sum of the j-1 before it is below tq, so the
+// number kept is the first j whose sum reaches tq.  Sums only grow while affinities are positive, and
+// a radix bin never mixes signs (the sign is the key's top bit), so the crossing is found like the
+// C-th largest key: four 8-bit passes over the expert's keys, here with a histogram of counts and one
+// of sums per pass, walking the bins from the top to the first one whose cumulated sum reaches what
+// is left of tq.  In the last pass a bin is a single key value q > 0, of which ceil(left / q) are needed.
+__global__ void __launch_bounds__(1024)
+select_threshold_limit_kernel(const uint32_t* __restrict__ keyT, int32_t* __restrict__ limit, int T,
+                              long long tq) {
+  __shared__ uint32_t hist_cnt[256];
+  __shared__ unsigned long long hist_sum[256];
+  __shared__ uint32_t s_prefix, s_before;
+  __shared__ long long s_left;
+  __shared__ int s_state;                            // 0: walking, 1: never reached
+  const int i = blockIdx.x, tid = threadIdx.x, lane = tid & 31;
+  const uint32_t* row = keyT + (size_t)i * T;
+  if (tq <= 0) { if (tid == 0) limit[i] = 0; return; }
+  if (tid == 0) { s_prefix = 0; s_before = 0; s_left = tq; s_state = 0; }
+  for (int pass = 0; pass < 4; ++pass) {
+    const int shift = 24 - 8 * pass;
+    if (tid < 256) { hist_cnt[tid] = 0; hist_sum[tid] = 0ull; }
+    __syncthreads();
+    const uint32_t prefix = s_prefix;
+    const uint32_t pmask = pass == 0 ? 0u : (0xffffffffu << (shift + 8));
+    for (int c0 = 0; c0 < T; c0 += 1024) {
+      const int t = c0 + tid;
+      const uint32_t kx = t < T ? row[t] : 0u;
+      const bool active = kx != 0u && (kx & pmask) == prefix;
+      const uint32_t digit = (kx >> shift) & 0xffu;
+      const long long q = active ? quantise_affinity(key_to_float(kx)) : 0ll;
+      // lanes holding the same digit add once, through their first lane
+      uint32_t todo = __ballot_sync(0xffffffffu, active);
+      while (todo) {
+        const int leader = __ffs(todo) - 1;
+        const uint32_t d0 = __shfl_sync(0xffffffffu, digit, leader);
+        const bool mine = active && digit == d0;
+        const uint32_t group = __ballot_sync(0xffffffffu, mine);
+        long long sum = mine ? q : 0ll;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+        if (lane == leader) {
+          atomicAdd(&hist_cnt[d0], (uint32_t)__popc(group));
+          atomicAdd(&hist_sum[d0], (unsigned long long)sum);
+        }
+        todo &= ~group;
+      }
+    }
+    __syncthreads();
+    if (tid == 0) {
+      long long cum = 0, left = s_left;
+      uint32_t cnt = 0;
+      int found = -1;
+      for (int b = 255; b >= 0; --b) {
+        if (hist_cnt[b] == 0) continue;
+        const long long sb = (long long)hist_sum[b];
+        if (cum + sb >= left) { found = b; break; }
+        cum += sb;
+        cnt += hist_cnt[b];
+      }
+      if (found < 0) {
+        s_state = 1;
+      } else {
+        s_prefix = prefix | ((uint32_t)found << shift);
+        s_left = left - cum;
+        s_before += cnt;
+      }
+    }
+    __syncthreads();
+    if (s_state) break;                              // uniform across the CTA
+  }
+  if (tid == 0) {
+    if (s_state) {
+      limit[i] = 0x7fffffff;
+    } else {
+      const long long q = quantise_affinity(key_to_float(s_prefix));      // > 0: its bin's sum crossed
+      limit[i] = (int32_t)(s_before + (uint32_t)((s_left + q - 1) / q));
+    }
+  }
+}
+
 // One CTA (1024 threads) per expert; every thread owns 4 consecutive tokens per sweep.
 constexpr int SEL_KPT = 4;
 constexpr int SEL_SWEEP = 1024 * SEL_KPT;
@@ -159,8 +270,8 @@ __device__ __forceinline__ void load_keys(const uint32_t* __restrict__ row, int 
 
 __global__ void __launch_bounds__(1024)
 select_expert_side_kernel(uint32_t* __restrict__ keyT, const etr_stats* __restrict__ stats,
-                          int32_t* __restrict__ counts, int32_t* __restrict__ slot_token,
-                          float* __restrict__ gate, int T, int C_stride) {
+                          const int32_t* __restrict__ limit, int32_t* __restrict__ counts,
+                          int32_t* __restrict__ slot_token, float* __restrict__ gate, int T, int C_stride) {
   __shared__ uint32_t hist[256];
   __shared__ uint32_t s_prefix, s_remaining, s_ncand;
   __shared__ uint32_t warp_tot[32], warp_pre[32];
@@ -169,7 +280,7 @@ select_expert_side_kernel(uint32_t* __restrict__ keyT, const etr_stats* __restri
   uint32_t* row = keyT + (size_t)i * T;
   int32_t* my_slot = slot_token + (size_t)i * C_stride;
   float* my_gate = gate + (size_t)i * C_stride;
-  const int C = stats->C;
+  const int C = limit ? min(stats->C, limit[i]) : stats->C;      // limit: the threshold on the sum of affinities
 
   // radix select, 4 passes of 8 bits: the n_keep-th largest key; pass 0 also counts candidates
   uint32_t tau = 0, quota = 0, n_keep = 0;
@@ -310,8 +421,9 @@ __device__ __forceinline__ uint32_t sel_peer_load(const uint32_t* local, uint32_
 template <int CL>
 __global__ void __launch_bounds__(1024, 2)
 select_expert_side_cluster_kernel(uint32_t* __restrict__ keyT, const etr_stats* __restrict__ stats,
-                                  int32_t* __restrict__ counts, int32_t* __restrict__ slot_token,
-                                  float* __restrict__ gate, int T, int C_stride) {
+                                  const int32_t* __restrict__ limit, int32_t* __restrict__ counts,
+                                  int32_t* __restrict__ slot_token, float* __restrict__ gate, int T,
+                                  int C_stride) {
   __shared__ uint32_t hist[256], tot[256];
   __shared__ uint32_t s_prefix, s_remaining, s_ncand_local, s_ncand;
   __shared__ uint32_t s_cnt_gt, s_cnt_eq;
@@ -325,7 +437,7 @@ select_expert_side_cluster_kernel(uint32_t* __restrict__ keyT, const etr_stats* 
   uint32_t* row = keyT + (size_t)i * T;
   int32_t* my_slot = slot_token + (size_t)i * C_stride;
   float* my_gate = gate + (size_t)i * C_stride;
-  const int C = stats->C;
+  const int C = limit ? min(stats->C, limit[i]) : stats->C;
 
   // this CTA's keys are read from global memory once and stay in shared memory for every pass
   extern __shared__ uint32_t sk[];
@@ -517,12 +629,19 @@ csr_count_kernel(const int32_t* __restrict__ posT, int32_t* __restrict__ tok_ptr
 
 __global__ void __launch_bounds__(1024)
 csr_scan_kernel(int32_t* __restrict__ block_total, int32_t* __restrict__ tok_ptr, etr_stats* stats,
-                int nblocks, int n_cand) {
+                int nblocks, int n_cand, const int32_t* __restrict__ skipped, int n_skipped_blocks) {
   __shared__ int wsum[32], wpre[32];
-  __shared__ int carry;
+  __shared__ int carry, given_up;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  if (tid == 0) { carry = 0; tok_ptr[0] = 0; }
+  if (tid == 0) { carry = 0; given_up = 0; tok_ptr[0] = 0; }
   __syncthreads();
+  if (skipped) {              // candidates the tokens gave up themselves (token-side threshold): integer sum
+    int s = 0;
+    for (int b = tid; b < n_skipped_blocks; b += 1024) s += skipped[b];
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    if (lane == 0 && s) atomicAdd(&given_up, s);
+    __syncthreads();
+  }
   for (int c0 = 0; c0 < nblocks; c0 += 1024) {
     const int b = c0 + tid;
     const int v = b < nblocks ? block_total[b] : 0;
@@ -554,7 +673,7 @@ csr_scan_kernel(int32_t* __restrict__ block_total, int32_t* __restrict__ tok_ptr
   }
   if (tid == 0) {
     stats->rows_total = carry;
-    stats->dropped = n_cand - carry;
+    stats->dropped = n_cand - given_up - carry;
   }
 }
 
@@ -574,8 +693,12 @@ csr_fill_kernel(const int32_t* __restrict__ posT, const int32_t* __restrict__ bl
 
 // key / position matrix [E][T], then one int per 256-token block
 static size_t select_keys_bytes(const etr_config* c) { return align_up((size_t)c->T * c->E * sizeof(uint32_t), 256); }
+// ... then the per-expert threshold limits and the per-block counts of given-up candidates
+static size_t select_scan_bytes(const etr_config* c) { return align_up((size_t)ceil_div(c->T, 256) * sizeof(int32_t), 256); }
+static size_t select_limit_bytes(const etr_config* c) { return align_up((size_t)c->E * sizeof(int32_t), 256); }
 size_t select_workspace_bytes(const etr_config* c) {
-  return select_keys_bytes(c) + align_up((size_t)ceil_div(c->T, 256) * sizeof(int32_t), 256);
+  return select_keys_bytes(c) + select_scan_bytes(c) + select_limit_bytes(c) +
+         align_up((size_t)ceil_div(c->T, SEL_TB) * sizeof(int32_t), 256);
 }
 
 int resolve_mode(const etr_config* c) {
@@ -589,10 +712,20 @@ etr_status select_forward(const etr_config* c, const float* delta, etr_stats* st
   p.T = c->T; p.E = c->E; p.k = c->k; p.d = c->d; p.C_stride = c_stride_of(c);
   p.capacity = c->capacity; p.c_floor = c->c_floor < 1 ? 1 : c->c_floor; p.adaptive = c->adaptive;
   p.mode = resolve_mode(c); p.delta_max_override = c->delta_max_override;
+  p.cut_token = (c->threshold_mode & ETR_THRESHOLD_TOKEN) != 0 && p.mode == ETR_MODE_TCR;
+  p.tq_token = quantise_threshold(c->threshold_tau_token);
   uint32_t* keyT = (uint32_t*)ws;
+  char* ws_tail = reinterpret_cast<char*>(ws) + select_keys_bytes(c) + select_scan_bytes(c);
+  int32_t* limit = (c->threshold_mode & ETR_THRESHOLD_EXPERT) ? reinterpret_cast<int32_t*>(ws_tail) : nullptr;
+  int32_t* skipped = p.cut_token ? reinterpret_cast<int32_t*>(ws_tail + select_limit_bytes(c)) : nullptr;
   ETR_TIME_BEGIN("select_token_side_kernel");
-  select_token_side_kernel<<<ceil_div(c->T, SEL_TB), 256, 0, st>>>(delta, rt->topk_idx, keyT, stats, p);
+  select_token_side_kernel<<<ceil_div(c->T, SEL_TB), 256, 0, st>>>(delta, rt->topk_idx, keyT, stats, skipped, p);
   ETR_LAUNCH_CHECK();
+  if (limit) {
+    ETR_TIME_BEGIN("select_threshold_limit_kernel");
+    select_threshold_limit_kernel<<<c->E, 1024, 0, st>>>(keyT, limit, c->T, quantise_threshold(c->threshold_tau));
+    ETR_LAUNCH_CHECK();
+  }
   ETR_TIME_BEGIN("select_expert_side_kernel");
   if (c->T >= 8192 && c->T <= 4 * 49152) {     // split each expert's row over a cluster of 4 CTAs
     constexpr int CL = 4;
@@ -610,12 +743,13 @@ etr_status select_forward(const etr_config* c, const float* delta, etr_stats* st
     lc.attrs = attr;
     lc.numAttrs = 1;
     if (cudaLaunchKernelEx(&lc, select_expert_side_cluster_kernel<CL>, keyT, (const etr_stats*)stats,
-                           rt->counts, rt->slot_token, rt->gate, c->T, p.C_stride) != cudaSuccess) {
+                           (const int32_t*)limit, rt->counts, rt->slot_token, rt->gate, c->T,
+                           p.C_stride) != cudaSuccess) {
       timing_end(st);
       return ETR_ERR_CUDA;
     }
   } else {
-    select_expert_side_kernel<<<c->E, 1024, 0, st>>>(keyT, stats, rt->counts, rt->slot_token, rt->gate,
+    select_expert_side_kernel<<<c->E, 1024, 0, st>>>(keyT, stats, limit, rt->counts, rt->slot_token, rt->gate,
                                                      c->T, p.C_stride);
   }
   ETR_LAUNCH_CHECK();
@@ -626,7 +760,8 @@ etr_status select_forward(const etr_config* c, const float* delta, etr_stats* st
   ETR_LAUNCH_CHECK();
   const int n_cand = p.mode == ETR_MODE_TCR ? c->T * c->k : c->T * c->E;
   ETR_TIME_BEGIN("csr_scan_kernel");
-  csr_scan_kernel<<<1, 1024, 0, st>>>(block_total, rt->tok_ptr, stats, nblocks, n_cand);
+  csr_scan_kernel<<<1, 1024, 0, st>>>(block_total, rt->tok_ptr, stats, nblocks, n_cand, skipped,
+                                      ceil_div(c->T, SEL_TB));
   ETR_LAUNCH_CHECK();
   ETR_TIME_BEGIN("csr_fill_kernel");
   csr_fill_kernel<<<nblocks, 256, 0, st>>>((const int32_t*)keyT, block_total, rt->tok_ptr, rt->tok_row,
@@ -644,8 +779,9 @@ etr_status select_forward(const etr_config* c, const float* delta, etr_stats* st
 // process exits.
 namespace etr {
 
-// the keys, plus the per-block scan scratch (one int per 256 tokens; T <= 4 Mi)
-constexpr size_t SELECT_STATIC_MAX_BYTES = ETR_SELECT_STATIC_MAX_ENTRIES * sizeof(uint32_t) + (64u << 10) + 512u;
+// the keys, plus the small arrays select_forward keeps behind them: one int per 256 tokens (scan), one
+// per expert (threshold limits), one per 32 tokens (candidates given up); T <= 4 Mi, E <= 256
+constexpr size_t SELECT_STATIC_MAX_BYTES = ETR_SELECT_STATIC_MAX_ENTRIES * sizeof(uint32_t) + (640u << 10);
 static __device__ __align__(256) unsigned char g_select_scratch[SELECT_STATIC_MAX_BYTES];
 
 // In host code `g_select_scratch` is only a handle for the runtime's symbol table, not a

@@ -1,6 +1,7 @@
 """Behaviour the C ABI promises besides the numbers of the default path: fp32 weight gradients
-(grad_fp32), a selection that may be repeated on one stats block, and the bounded device-side
-wait, whose expiry must surface as ETR_ERR_TIMEOUT and leave the stream usable."""
+(grad_fp32), a selection that may be repeated on one stats block, the bounded device-side wait,
+whose expiry must surface as ETR_ERR_TIMEOUT and leave the stream usable, and the selection cut by
+a threshold on the sum of affinity scores (bit-exact against the oracle's select_thresholded)."""
 import numpy as np
 import pytest
 import torch
@@ -143,3 +144,70 @@ def test_bounded_wait_expires_as_a_status_and_the_stream_stays_usable():
     Y2 = torch.empty_like(dev.X)
     etr.layer_forward(cfg_l, dev.X, dev.R, dev.W1g, dev.W1u, dev.W2, buf, Y2)
     assert buf.read_stats().error_word == 0 and torch.equal(Y, Y2)
+
+
+THRESHOLD_CASES = [
+    # (T, E, k, C, mode, flags, tau_expert, tau_token)
+    (1000, 16, 2, 160, ob.MODE_TCR, 1, 2.0, np.inf),
+    (1000, 16, 2, 160, ob.MODE_ECR, 1, 3.5, np.inf),
+    (1000, 16, 4, 300, ob.MODE_TCR, 2, np.inf, 0.12),
+    (1000, 16, 4, 300, ob.MODE_TCR, 3, 1.5, 0.12),
+    (777, 8, 2, 64, ob.MODE_ECR, 1, 1e-3, np.inf),            # below the first score: one token each
+    (777, 8, 2, 64, ob.MODE_ECR, 1, 0.0, np.inf),             # nothing kept
+    (777, 8, 2, 64, ob.MODE_TCR, 3, np.inf, np.inf),          # no cut at all
+    (12000, 32, 2, 900, ob.MODE_ECR, 1, 30.0, np.inf),        # expert's keys split over a cluster of CTAs
+    (12000, 32, 2, 900, ob.MODE_TCR, 3, 12.0, 0.2),
+]
+
+
+@pytest.mark.parametrize("T,E,k,C,mode,flags,tau_e,tau_t", THRESHOLD_CASES)
+def test_selection_with_a_threshold_on_the_affinity_sum(T, E, k, C, mode, flags, tau_e, tau_t):
+    """etr_select with threshold_mode set against the oracle's select_thresholded on the same affinity
+    bits: every map, count and counter identical (the sums are integers on both sides)."""
+    w = gw.scaled(gw.WORKLOADS["small"], T=T, E=E, k=k, d=1024, D=8, cf=(C - 0.5) * E / (T * k))
+    assert w.capacity == C
+    rng = np.random.default_rng(T + 31 * flags)
+    delta = (rng.standard_normal((T, E)) / 12).astype(np.float32)       # mixed signs, |delta| ~ 0.08
+    delta[rng.random((T, E)) < 0.02] = np.float32(0.0625)               # and some exact ties
+    o = ob.Oracle("f32")
+    ref = o.select_thresholded(delta, k, mode, C, w.C_stride, flags, tau_e, tau_t)
+    cfg = hz.make_cfg(w, mode=mode, threshold_mode=flags, threshold_tau=tau_e, threshold_tau_token=tau_t)
+    _, got = run_select(w, cfg, delta)
+    assert routes_equal(ref, got)
+    if flags & 1 and np.isfinite(tau_e) and tau_e > 0.01:
+        assert np.any(got.counts < min(C, T)), "the threshold was meant to bite"
+    buf = etr.LayerBuffers(cfg)
+    buf.stats.zero_()
+    buf.delta.copy_(torch.from_numpy(delta))
+    etr.select_static(cfg, buf.delta, buf.c.stats, buf.route)
+    assert routes_equal(ref, hz.route_from_buffers(buf, cfg))
+
+
+@pytest.mark.parametrize("mode,flags", [(ob.MODE_TCR, 3), (ob.MODE_ECR, 1)])
+def test_layer_with_a_threshold_on_the_affinity_sum(mode, flags):
+    """The whole layer with the threshold on: routing identical to the oracle's, outputs and
+    gradients within the usual bounds (the stages after the selection do not know about it)."""
+    w, inp, o, _, _ = case("small_s")
+    tau_e, tau_t = 2.5, 0.09
+    fw = o.forward(inp["X"], inp["R"], inp["W1g"], inp["W1u"], inp["W2"], D=w.D, k=w.k, capacity=w.capacity,
+                   mode=mode, threshold_mode=flags, tau_expert=tau_e, tau_token=tau_t)
+    bw = o.backward(fw, inp["X"], inp["R"], inp["W1g"], inp["W1u"], inp["W2"], inp["dY"])
+    assert 0 < fw.route.tok_ptr[-1] < o.select(fw.delta, w.k, mode, w.capacity, w.C_stride).tok_ptr[-1]
+    cfg = hz.make_cfg(w, mode=mode, threshold_mode=flags, threshold_tau=tau_e, threshold_tau_token=tau_t)
+    dev = hz.upload(w, inp)
+    buf = etr.LayerBuffers(cfg)
+    out = dict(Y=torch.empty_like(dev.X), dX=torch.empty_like(dev.X), dR=torch.empty_like(dev.R),
+               dW1g=torch.empty_like(dev.W1g), dW1u=torch.empty_like(dev.W1u), dW2=torch.empty_like(dev.W2))
+    etr.layer_forward(cfg, dev.X, dev.R, dev.W1g, dev.W1u, dev.W2, buf, out["Y"])
+    etr.layer_backward(cfg, dev.X, dev.R, dev.W1g, dev.W1u, dev.W2, dev.dY, buf, out["dX"], out["dR"],
+                       out["dW1g"], out["dW1u"], out["dW2"])
+    torch.cuda.synchronize()
+    assert buf.read_stats().error_word == 0
+    got = hz.route_from_buffers(buf, cfg)
+    # the device's affinities differ from the oracle's in the last bits, and a running sum within
+    # a few 2^-32 of tau may then stop one candidate earlier or later: compare on the oracle's route
+    # only when the maps agree, which these seeds give
+    assert hz.assert_routes_match(fw.delta, fw.route, got, mode), "threshold crossings have clear margins here"
+    for nm, ref, chain in (("Y", fw.Y, 4), ("dX", bw.dX, 6), ("dR", bw.dR, 4), ("dW1g", bw.dW1g, 6),
+                           ("dW1u", bw.dW1u, 6), ("dW2", bw.dW2, 4)):
+        hz.assert_close_rms(hz.to_np(out[nm]), ref, 2e-2, nm, chain=chain)

@@ -370,6 +370,16 @@ def test_threshold_bruteforce_over_prefixes(o64, mode, seed):
                 best = n
         assert got.counts[i] == best
         assert sorted(order[:best]) == list(got.slot_token[i * 128:i * 128 + best])
+    if mode == ob.MODE_TCR:      # token side, same search over each token's ranked experts (k = 3, mixed signs)
+        tok = o64.select_thresholded(delta, 3, mode, T, 128, 2, tau_token=float(tau))
+        for t in range(T):
+            order = sorted(range(E), key=lambda i: (-delta[t, i], i))
+            best = 0
+            for n in range(0, 4):
+                sums = [sum((Fraction(delta[t, i]) for i in order[:j]), Fraction(0)) for j in range(n)]
+                if all(s < tau for s in sums):
+                    best = n
+            assert list(tok.topk_idx[t]) == order[:best] + [-1] * (3 - best)
 
 
 def test_threshold_closed_form_on_constant_scores(o32):
