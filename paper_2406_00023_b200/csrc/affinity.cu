@@ -730,6 +730,80 @@ affinity_bwd_dx_kernel(const T* __restrict__ X, const float* __restrict__ R,
 constexpr int DXC_MAX_TOKENS = 16;
 constexpr int DXC_ROWS = 512;          // row entries held in shared memory; later ones are read in place
 
+// cz and beta of every routed token of a chunk (phase 2 of the chunked dX kernels), for the pooled
+// columns j = tid, tid + 256, ...  The chunk's staged row entries are walked as ONE flat list, eight at
+// a time: the eight R values a thread needs are requested together before any is used, so a chunk
+// costs a few rounds of L2 latency instead of one per token and entry.  Within a token the entries
+// are still added in list order (same sums, bit for bit, as a loop per token).  Entries beyond the
+// staged ones (DXC_ROWS) are read in place.
+__device__ __forceinline__ void dx_chunk_cz(float* __restrict__ cz, float* __restrict__ s_beta,
+                                            const int* __restrict__ s_ptr, const int* __restrict__ s_exp,
+                                            const float* __restrict__ s_w, const float* __restrict__ s_dg,
+                                            const float* __restrict__ s_dl, const float* __restrict__ s_a,
+                                            const float* __restrict__ R, const float* __restrict__ rnorm,
+                                            const float* __restrict__ delta, const float* __restrict__ dgate,
+                                            const int32_t* __restrict__ tok_row, int base, int staged_max,
+                                            int nt, int m, int E, int C_stride, int t0, float sqD, int D,
+                                            int tid) {
+  for (int j = tid; j < m; j += 256) {
+    int tl = 0;
+    while (tl < nt && s_ptr[tl + 1] == s_ptr[tl]) ++tl;              // first routed token
+    float acc = 0.f, beta = 0.f;
+    const int total = s_ptr[nt] - base;
+    const int staged = min(total, staged_max);
+    for (int e0 = 0; e0 < staged; e0 += 8) {
+      float rv[8];
+#pragma unroll
+      for (int b = 0; b < 8; ++b) {
+        const int e = e0 + b;
+        const int i = e < staged ? s_exp[e] : -1;
+        rv[b] = i >= 0 ? R[(size_t)i * m + j] : 0.f;
+      }
+#pragma unroll
+      for (int b = 0; b < 8; ++b) {
+        const int e = e0 + b;
+        if (e >= staged) break;
+        while (s_ptr[tl + 1] - base <= e) {                          // the entry opens a later token: close this one
+          const float a = s_a[tl];
+          cz[(size_t)tl * m + j] = acc;
+          if (j == 0) s_beta[tl] = a != 0.f ? beta / (a * a) : 0.f;
+          acc = 0.f; beta = 0.f;
+          ++tl;
+          while (s_ptr[tl + 1] == s_ptr[tl]) ++tl;
+        }
+        if (s_exp[e] >= 0 && s_a[tl] != 0.f) {
+          beta = fmaf(s_dg[e], s_dl[e], beta);
+          acc = fmaf(s_w[e], rv[b], acc);
+        }
+      }
+    }
+    // entries that did not fit the staged lists, token by token
+    while (tl < nt) {
+      const int beg = max(s_ptr[tl] - base, staged), end = s_ptr[tl + 1] - base;
+      const float a = s_a[tl];
+      if (a != 0.f) {
+        for (int q = beg; q < end; ++q) {
+          const int r = tok_row[base + q];
+          const int i = r / C_stride;
+          const float b = rnorm[i];
+          if (b == 0.f) continue;
+          const float dg = dgate[r];
+          beta = fmaf(dg, delta[(size_t)(t0 + tl) * E + i], beta);
+          acc = fmaf(dg * sqD / (a * b) / (float)D, R[(size_t)i * m + j], acc);
+        }
+      }
+      if (s_ptr[tl + 1] > s_ptr[tl]) {
+        cz[(size_t)tl * m + j] = acc;
+        if (j == 0) s_beta[tl] = a != 0.f ? beta / (a * a) : 0.f;
+      }
+      acc = 0.f; beta = 0.f;
+      ++tl;
+    }
+  }
+}
+
+
+
 template <class T, int NV, bool GROUP8>
 __global__ void __launch_bounds__(256, 4)
 affinity_bwd_dx_chunk_kernel(const T* __restrict__ X, const float* __restrict__ R,
@@ -769,36 +843,8 @@ affinity_bwd_dx_chunk_kernel(const T* __restrict__ X, const float* __restrict__ 
     s_w[e] = dg * sqD / (a * b) / (float)D;
   }
   __syncthreads();
-  for (int it = tid; it < nt * m; it += 256) {
-    const int tl = it / m, j = it - tl * m;
-    const int beg = s_ptr[tl] - base, end = s_ptr[tl + 1] - base;
-    if (beg == end) continue;
-    const float a = s_a[tl];
-    float acc = 0.f, beta = 0.f;
-    if (a != 0.f) {
-      for (int q = beg; q < end; ++q) {
-        int i;
-        float w, dg, dl;
-        if (q < DXC_ROWS) {
-          i = s_exp[q]; w = s_w[q]; dg = s_dg[q]; dl = s_dl[q];
-        } else {
-          const int r = tok_row[base + q];
-          i = r / C_stride;
-          const float b = rnorm[i];
-          dg = dgate[r];
-          dl = delta[(size_t)(t0 + tl) * E + i];
-          w = dg * sqD / (a * b) / (float)D;
-          if (b == 0.f) i = -1;
-        }
-        if (i < 0) continue;
-        beta = fmaf(dg, dl, beta);
-        acc = fmaf(w, R[(size_t)i * m + j], acc);
-      }
-      beta /= (a * a);
-    }
-    cz[it] = acc;
-    if (j == 0) s_beta[tl] = beta;
-  }
+  dx_chunk_cz(cz, s_beta, s_ptr, s_exp, s_w, s_dg, s_dl, s_a, R, rnorm, delta, dgate, tok_row, base,
+              DXC_ROWS, nt, m, E, C_stride, t0, sqD, D, tid);
   __syncthreads();
   const int vpt = d / 8 / NV;                      // threads per token
   for (int wi = tid; wi < nt * vpt; wi += 256) {
@@ -1175,7 +1221,8 @@ template <class T>
 static etr_status launch_bwd_dx(const etr_config* c, const void* X, const float* R, const float* delta,
                                 const float* xnorm, const float* rnorm, const etr_route* rt,
                                 const float* dgate, const float* ddelta, const void* dXp_fused, void* dX,
-                                size_t smem, cudaStream_t st) {
+                                etr_stats* stats, size_t smem, cudaStream_t st) {
+  (void)stats;
   const int m = c->d / c->D, Cs = c_stride_of(c), grid = ceil_div(c->T, 8);
   auto launch = [&](auto k, const char* name) -> etr_status {
     if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
@@ -1188,12 +1235,12 @@ static etr_status launch_bwd_dx(const etr_config* c, const void* X, const float*
   // chunked form of the fused kernel: as many tokens per block as keep cz within 48 KiB (at most 16)
   int tpb = DXC_MAX_TOKENS;
   while (tpb > 2 && (size_t)tpb * m * sizeof(float) > 48 * 1024) tpb /= 2;
+  int d_shift = 0;
+  while ((1 << d_shift) < c->D) ++d_shift;
+  const bool group8 = c->D >= 8 && (1 << d_shift) == c->D;
   if (dXp_fused && !ddelta && (size_t)tpb * m * sizeof(float) <= 48 * 1024) {
     const size_t csm = (size_t)tpb * m * sizeof(float);
     ETR_TIME_BEGIN("affinity_bwd_dx_fused_kernel");
-    int d_shift = 0;
-    while ((1 << d_shift) < c->D) ++d_shift;
-    const bool group8 = c->D >= 8 && (1 << d_shift) == c->D;
     auto go = [&](auto k) {
       k<<<ceil_div(c->T, tpb), 256, csm, st>>>((const T*)X, R, delta, xnorm, rnorm, rt->tok_ptr, rt->tok_row, dgate,
                                                (const T*)dXp_fused, (T*)dX, c->T, c->d, c->D, c->E, m, Cs, tpb,
@@ -1223,15 +1270,16 @@ static etr_status launch_bwd_dx(const etr_config* c, const void* X, const float*
 etr_status affinity_backward(const etr_config* c, const void* X, const float* R, const float* delta,
                              const float* Z, const float* xnorm, const float* rnorm,
                              const etr_route* rt, const float* dgate, const float* ddelta,
-                             const void* dXp_fused, void* dX, float* dR, void* ws, cudaStream_t st) {
+                             const void* dXp_fused, void* dX, float* dR, void* ws, etr_stats* stats,
+                             cudaStream_t st) {
   const int m = c->d / c->D, Cs = c_stride_of(c);
   const int nch = ddelta ? ceil_div(c->T, DR_DENSE_TOKENS) : Cs / DR_CHUNK;
   if (m > 256 * DR_MAXJ) return ETR_ERR_UNSUPPORTED;
   const size_t smem = (size_t)8 * m * sizeof(float);
   if (smem > 200 * 1024) return ETR_ERR_UNSUPPORTED;
   ETR_TRY((c->dtype == ETR_BF16
-               ? launch_bwd_dx<__nv_bfloat16>(c, X, R, delta, xnorm, rnorm, rt, dgate, ddelta, dXp_fused, dX, smem, st)
-               : launch_bwd_dx<float>(c, X, R, delta, xnorm, rnorm, rt, dgate, ddelta, dXp_fused, dX, smem, st)));
+               ? launch_bwd_dx<__nv_bfloat16>(c, X, R, delta, xnorm, rnorm, rt, dgate, ddelta, dXp_fused, dX, stats, smem, st)
+               : launch_bwd_dx<float>(c, X, R, delta, xnorm, rnorm, rt, dgate, ddelta, dXp_fused, dX, stats, smem, st)));
   float* part = (float*)ws;
   if (ddelta) {
     ETR_TIME_BEGIN("affinity_bwd_dr_dense_partial_kernel");

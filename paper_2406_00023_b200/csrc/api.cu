@@ -288,7 +288,7 @@ etr_status etr_affinity_bwd(const etr_config* c, const void* X, const float* R, 
   ETR_TRY(etr_validate(c));
   ETR_TRY(check_ptrs({X, R, delta, Z, xnorm, rnorm, dgate, dX, dR, ws}));
   ETR_TRY(check_route(route));
-  return affinity_backward(c, X, R, delta, Z, xnorm, rnorm, route, dgate, nullptr, nullptr, dX, dR, ws,
+  return affinity_backward(c, X, R, delta, Z, xnorm, rnorm, route, dgate, nullptr, nullptr, dX, dR, ws, nullptr,
                            (cudaStream_t)stream);
 }
 
@@ -316,7 +316,7 @@ etr_status etr_affinity_bwd_dense(const etr_config* c, const void* X, const floa
   ETR_TRY(etr_validate(c));
   ETR_TRY(check_ptrs({X, R, delta, Z, xnorm, rnorm, ddelta, dX, dR, ws}));
   ETR_TRY(check_route(route));
-  return affinity_backward(c, X, R, delta, Z, xnorm, rnorm, route, nullptr, ddelta, nullptr, dX, dR, ws,
+  return affinity_backward(c, X, R, delta, Z, xnorm, rnorm, route, nullptr, ddelta, nullptr, dX, dR, ws, nullptr,
                            (cudaStream_t)stream);
 }
 
@@ -375,7 +375,7 @@ etr_status etr_layer_backward(const etr_config* c, const void* X, const float* R
     ddelta = b->ddelta;
   }
   return affinity_backward(c, X, R, b->delta, b->Z, b->xnorm, b->rnorm, &b->route, b->dgate, ddelta,
-                           b->dXp, dX, dR, b->ws, (cudaStream_t)stream);
+                           b->dXp, dX, dR, b->ws, b->stats, (cudaStream_t)stream);
 }
 
 // Side streams and events for the host-buffer step (host-side objects, created once per device).

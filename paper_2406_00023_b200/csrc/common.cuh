@@ -135,6 +135,49 @@ __device__ inline float warp_sum(float v) {
   return v;
 }
 
+// ---- shared-memory barriers (mbarrier) and the bounded wait every pipeline of the library uses ----
+// A wait never spins forever: after limit_cycles SM clock cycles it sets the CTA's abort flag and
+// returns false; the kernel then stops issuing work, records a code in etr_stats.error_word and
+// returns (the host reads it as ETR_ERR_TIMEOUT).
+constexpr long long ETR_WAIT_LIMIT_CYCLES = 4000000000ll;   // about two seconds
+
+#ifdef __CUDACC__
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait: false if this or another thread of the CTA gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          long long limit_cycles) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  for (uint32_t it = 1;; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((it & 255u) == 0u) {
+      if (*abort_flag) return false;
+      if (clock64() - t0 > limit_cycles) { *abort_flag = 1; return false; }
+    }
+  }
+}
+#endif
+
 // ---- stage entry points, one translation unit each ------------------------------------------
 etr_status affinity_forward(const etr_config* c, const void* X, const float* R, float* delta,
                             float* Z, float* xnorm, float* rnorm, etr_stats* stats, cudaStream_t st);
@@ -142,7 +185,8 @@ size_t affinity_bwd_workspace_bytes(const etr_config* c);
 etr_status affinity_backward(const etr_config* c, const void* X, const float* R, const float* delta,
                              const float* Z, const float* xnorm, const float* rnorm,
                              const etr_route* rt, const float* dgate, const float* ddelta,
-                             const void* dXp_fused, void* dX, float* dR, void* ws, cudaStream_t st);
+                             const void* dXp_fused, void* dX, float* dR, void* ws, etr_stats* stats,
+                             cudaStream_t st);
 // softmax-gate variant and load statistics (gate.cu)
 etr_status gate_softmax_forward(const etr_config* c, const float* delta, const etr_route* rt, float* lse,
                                 cudaStream_t st);

@@ -37,7 +37,7 @@ constexpr int TC_BK = 64;
 constexpr int TC_STAGES = 4;
 constexpr int TC_THREADS = 320;        // TMA warp, MMA warp, 8 epilogue warps
 constexpr uint32_t TC_BOX_BYTES = 64 * 64 * 2;
-constexpr long long TC_WAIT_LIMIT_CYCLES = 4000000000ll;   // about two seconds
+constexpr long long TC_WAIT_LIMIT_CYCLES = ETR_WAIT_LIMIT_CYCLES;
 
 enum { TC_EPI_STORE = 0, TC_EPI_SWIGLU = 1, TC_EPI_DSWIGLU = 2 };
 enum { TC_DYN_M = 1, TC_DYN_K = 2 };
@@ -68,41 +68,7 @@ struct TcParams {
   int out_f32;           // plain-store epilogue: out0 is fp32 (weight gradients with grad_fp32)
 };
 
-// ---- PTX wrappers -----------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t smem_u32(const void* p) {
-  return (uint32_t)__cvta_generic_to_shared(p);
-}
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-  return ok != 0;
-}
-// Bounded wait: false if this or another thread of the CTA gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                          long long limit_cycles) {
-  if (mbar_try_wait(bar, parity)) return true;
-  const long long t0 = clock64();
-  for (uint32_t it = 1;; ++it) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if ((it & 255u) == 0u) {
-      if (*abort_flag) return false;
-      if (clock64() - t0 > limit_cycles) { *abort_flag = 1; return false; }
-    }
-  }
-}
+// ---- PTX wrappers (mbarrier helpers and the bounded wait: common.cuh) ---------------------------
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0,
                                             int c1, int c2) {
   asm volatile(

@@ -107,6 +107,20 @@ def test_tokens_kept_by_every_expert_overflow_the_staged_row_lists(dtype):
     assert np.all(np.diff(got.tok_ptr) == w.E)
 
 
+@pytest.mark.parametrize("d,D,dtype", [(2048, 16, "bf16"), (2048, 4, "bf16"), (2048, 8, "f32"), (4096, 32, "bf16"),
+                                       (8192, 64, "bf16")])
+def test_fused_dx_at_wide_hidden_sizes(d, D, dtype):
+    """Hidden sizes of 2048, 4096 and 8192 in the fused dX kernel (whole 4 to 16 KiB rows per token and
+    row of dXp), power-of-two and generic group sizes, a ragged last chunk of tokens (T = 215 =
+    13 * 16 + 7), and expert choice with C = T / 4, which gives tokens anything from no row (zeros,
+    X not read) to the rows of most of the 16 experts, so that one chunk's flat list of row entries
+    crosses many token boundaries."""
+    w = gw.scaled(W["small"], T=215, d=d, D=D, E=16, h=64, cf=2.0, dtype=dtype)
+    fw, got, out = layer_vs_oracle(w, gw.make_inputs(w), ob.MODE_ECR)
+    n = np.diff(got.tok_ptr)
+    assert n.min() == 0 and n.max() >= 6 and n.sum() > 3 * w.T
+
+
 @pytest.mark.parametrize("E,dtype", [(16, "bf16"), (32, "f32"), (64, "bf16")])
 def test_affinity_with_a_score_tile_for_every_sm(E, dtype):
     """38100 tokens: at least one 256-token tile per SM, which is when the score kernel takes its

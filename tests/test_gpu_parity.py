@@ -28,6 +28,8 @@ CASES = {
     "tiny_ecr": gw.scaled(W["tiny"], name="tiny_ecr", mode="ecr", cf=1.0),
     "small_s": gw.scaled(W["small"], name="small_s", T=1000, d=512, D=8, E=16, h=320),
     "mid_s": gw.scaled(W["mid"], name="mid_s", T=1536, d=512, D=8, E=8, h=384, n_clusters=8),
+    # d = 2048: 4 KiB token rows and 256 pooled columns, as in the mid and sweep workloads
+    "mid_w": gw.scaled(W["mid"], name="mid_w", T=1500, d=2048, D=8, E=8, h=128, n_clusters=32),
     "sweep_s_tcr": gw.scaled(W["sweep"], name="sweep_s_tcr", T=2048, d=1024, D=16, E=16, h=256,
                              n_clusters=16, step=600),
     "sweep_s_ecr": gw.scaled(W["sweep"], name="sweep_s_ecr", T=2048, d=1024, D=16, E=16, h=256,
@@ -443,7 +445,7 @@ def test_pipelined_host_steps_match_the_layer_calls():
         etr.layer_step_host_wait(etr.HostSlot(cfg, etr.HOST_SLOTS))
 
 
-@pytest.mark.parametrize("name", ["tiny", "small_s", "mid_s"])
+@pytest.mark.parametrize("name", ["tiny", "small_s", "mid_s", "mid_w"])
 def test_stage_calls_compose_to_the_layer_calls(name):
     """The ten stage entry points called one by one give what etr_layer_forward/backward give.
     Only dX may differ, by one rounding: the layer call fuses the dispatch backward into the
@@ -479,7 +481,7 @@ def test_stage_calls_compose_to_the_layer_calls(name):
 
 
 @pytest.mark.parametrize("gate", ["affinity", "softmax"])
-@pytest.mark.parametrize("name", ["small_s", "mid_s", "sweep_s_tcr", "sweep_s_ecr"])
+@pytest.mark.parametrize("name", ["small_s", "mid_s", "mid_w", "sweep_s_tcr", "sweep_s_ecr"])
 def test_parity_with_the_storage_grid_modelled(name, gate):
     """The sharp version of the value comparison, with no exceptions: every stored activation and
     every output and gradient of the layer against the oracle's stages composed with the same
