@@ -69,6 +69,13 @@ typedef enum { ETR_GEMM_AUTO = 0, ETR_GEMM_SIMT = 1, ETR_GEMM_TCGEN05 = 2, ETR_G
  * row gathers (four rows per request, named by slot_token), and buf->Xp is neither written nor
  * read.  The stage calls are unaffected.  ETR_FUSE_AUTO lets the library choose. */
 typedef enum { ETR_FUSE_AUTO = 0, ETR_FUSE_OFF = 1, ETR_FUSE_ON = 2 } etr_fuse;
+/* fuse_combine: in etr_layer_forward on the tensor-core path with Top-1 token choice (k = 1, the
+ * routing of the paper's efficiency runs) every token has at most one row, so the gate-weighted sum
+ * of the general MoE equation has a single term and the down GEMM's epilogue writes gate * O straight
+ * to the token's row of Y; the combine kernel does not run (tokens without a row get their zeros from
+ * a small fill kernel).  Same bits as the separate combine.  AUTO and ON enable it wherever that
+ * condition holds, OFF never; with k >= 2 or expert choice a token's rows lie in different experts'
+ * tiles and the sum stays in etr_combine, whose fixed order keeps the result deterministic. */
 
 /* Gate of a selected pair (t, i).  AFFINITY (default): the raw affinity delta_ti (the affinity-score
  * equation of "Cost-Efficient Sparse Expert-Token Affinity", whose matrix the paper also uses as the
@@ -112,6 +119,8 @@ typedef struct etr_config {
   float threshold_tau_token;  /* ETR_THRESHOLD_TOKEN: the sum at which a token stops taking experts */
   int64_t wait_limit_cycles;  /* bound of every device-side wait of the GEMM pipeline, in SM clock
                                  cycles; 0 = the default, about two seconds */
+  int32_t fuse_combine;       /* etr_fuse: the combine folded into the down GEMM's epilogue (see below) */
+  int32_t reserved0;
 } etr_config;
 
 /* Per-call scalars produced and consumed on the device (device struct, 64 bytes). */

@@ -9,7 +9,7 @@
 
 namespace etr {
 
-static_assert(sizeof(etr_config) == 104 && sizeof(etr_stats) == 64, "layouts the bindings rely on");
+static_assert(sizeof(etr_config) == 112 && sizeof(etr_stats) == 64, "layouts the bindings rely on");
 
 static std::atomic<long long> g_launches{0};
 void note_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
@@ -49,6 +49,12 @@ static bool use_tc(const etr_config* c) {
 // Token rearrangement fused into the GEMM operand fetch (layer calls, tensor-core path only).
 static bool fuse_dispatch(const etr_config* c) {
   return use_tc(c) && c->fuse_dispatch == ETR_FUSE_ON;
+}
+
+// Combine folded into the down GEMM's epilogue (layer calls, tensor-core path): only where it is exact,
+// Top-1 token choice, in which a token has at most one row and its output needs no sum.
+static bool fuse_combine(const etr_config* c) {
+  return use_tc(c) && c->fuse_combine != ETR_FUSE_OFF && c->k == 1 && resolve_mode(c) == ETR_MODE_TCR;
 }
 
 static etr_status check_ptrs(std::initializer_list<const void*> ps) {
@@ -147,6 +153,7 @@ etr_status etr_validate(const etr_config* c) {
   if (c->mode < ETR_MODE_AUTO || c->mode > ETR_MODE_ECR) return ETR_ERR_ARG;
   if (c->gemm_impl < ETR_GEMM_AUTO || c->gemm_impl > ETR_GEMM_TCGEN05_2CTA_WIDE) return ETR_ERR_ARG;
   if (c->fuse_dispatch < ETR_FUSE_AUTO || c->fuse_dispatch > ETR_FUSE_ON) return ETR_ERR_ARG;
+  if (c->fuse_combine < ETR_FUSE_AUTO || c->fuse_combine > ETR_FUSE_ON) return ETR_ERR_ARG;
   if (c->gate_mode != ETR_GATE_AFFINITY && c->gate_mode != ETR_GATE_SOFTMAX) return ETR_ERR_ARG;
   if (c->weight_dtype != ETR_F32 && c->weight_dtype != ETR_BF16) return ETR_ERR_ARG;
   if (c->threshold_mode < 0 || c->threshold_mode > (ETR_THRESHOLD_EXPERT | ETR_THRESHOLD_TOKEN)) return ETR_ERR_ARG;
@@ -229,7 +236,7 @@ etr_status etr_expert_ffn(const etr_config* c, const etr_route* route, const voi
   ETR_TRY(check_route(route));
   if (use_tc(c)) {
     ETR_TRY(check_ptrs({stats, ws}));
-    return tc_ffn_forward(c, route, Xp, nullptr, W1g, W1u, W2, G, U, H, O, stats, ws, (cudaStream_t)stream);
+    return tc_ffn_forward(c, route, Xp, nullptr, W1g, W1u, W2, G, U, H, O, stats, ws, nullptr, (cudaStream_t)stream);
   }
   return simt_ffn_forward(c, route, Xp, W1g, W1u, W2, G, U, H, O, (cudaStream_t)stream);
 }
@@ -339,16 +346,23 @@ etr_status etr_layer_forward(const etr_config* c, const void* X, const float* R,
   ETR_TRY(etr_affinity(c, X, R, b->delta, b->Z, b->xnorm, b->rnorm, b->stats, stream));
   ETR_TRY(etr_select(c, b->delta, b->stats, &b->route, b->ws, stream));
   if (c->gate_mode == ETR_GATE_SOFTMAX) ETR_TRY(etr_gate_softmax(c, b->delta, &b->route, b->lse, stream));
-  if (fuse_dispatch(c)) {       // the first GEMM gathers its rows from X: no Xp
+  const bool fc = fuse_combine(c);
+  if (fc) {                     // Top-1: Y is written by the down GEMM's epilogue; tokens without a row get zeros here
+    ETR_TRY(check_ptrs({Y}));
+    ETR_TRY(zero_unrouted_rows(c, &b->route, Y, (cudaStream_t)stream));
+  }
+  if (fuse_dispatch(c) || fc) {
+    const bool fd = fuse_dispatch(c);      // the first GEMM gathers its rows from X: no Xp
     ETR_TRY(check_ptrs({X, W1g, W1u, W2, b->G, b->U, b->H, b->O, b->ws}));
-    ETR_TRY(tc_ffn_forward(c, &b->route, nullptr, X, W1g, W1u, W2, b->G, b->U, b->H, b->O, b->stats, b->ws,
-                           (cudaStream_t)stream));
+    if (!fd) ETR_TRY(etr_dispatch(c, X, &b->route, b->Xp, stream));
+    ETR_TRY(tc_ffn_forward(c, &b->route, fd ? nullptr : b->Xp, fd ? X : nullptr, W1g, W1u, W2, b->G, b->U, b->H,
+                           b->O, b->stats, b->ws, fc ? Y : nullptr, (cudaStream_t)stream));
   } else {
     ETR_TRY(etr_dispatch(c, X, &b->route, b->Xp, stream));
     ETR_TRY(etr_expert_ffn(c, &b->route, b->Xp, W1g, W1u, W2, b->G, b->U, b->H, b->O, b->stats, b->ws,
                            stream));
   }
-  return etr_combine(c, &b->route, b->O, Y, stream);
+  return fc ? ETR_OK : etr_combine(c, &b->route, b->O, Y, stream);
 }
 
 etr_status etr_layer_backward(const etr_config* c, const void* X, const float* R, const void* W1g,

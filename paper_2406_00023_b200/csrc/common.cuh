@@ -216,7 +216,10 @@ etr_status simt_ffn_backward(const etr_config* cfg, const etr_route* route, cons
 // through route->slot_token and Xp is not read (may be nullptr).
 etr_status tc_ffn_forward(const etr_config* cfg, const etr_route* route, const void* Xp, const void* X_tokens,
                           const void* W1g, const void* W1u, const void* W2, void* G, void* U,
-                          void* H, void* O, etr_stats* stats, void* ws, cudaStream_t st);
+                          void* H, void* O, etr_stats* stats, void* ws, void* Y_top1, cudaStream_t st);
+// Y_top1 != nullptr (Top-1 token choice only): the down GEMM's epilogue also writes gate * O of every
+// row in use to the row of its token in Y; rows of tokens without a row are not touched.
+etr_status zero_unrouted_rows(const etr_config* c, const etr_route* rt, void* Y, cudaStream_t st);
 etr_status tc_ffn_backward(const etr_config* cfg, const etr_route* route, const void* dO,
                            const void* Xp, const void* X_tokens, const void* G, const void* U, const void* H,
                            const void* W1g, const void* W1u, const void* W2, void* dG, void* dU,

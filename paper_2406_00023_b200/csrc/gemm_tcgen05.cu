@@ -64,6 +64,10 @@ struct TcParams {
   int gather;
   int gather_ld, gather_oob;
   const int32_t* gather_idx;
+  // Combine folded into the plain-store epilogue (Top-1 token choice: a token has at most one row, so
+  // its output is that row times its gate and needs no sum): besides out0, row r of expert e also goes,
+  // scaled, to row sc_tok[e*M + r] of sc_out (skipped where the slot holds -1).  sc_out == nullptr: off.
+  const int32_t* sc_tok; const float* sc_gate; __nv_bfloat16* sc_out; int sc_ld;
   long long wait_limit;  // bound of every mbarrier wait, in SM clock cycles
   int out_f32;           // plain-store epilogue: out0 is fp32 (weight gradients with grad_fp32)
 };
@@ -185,6 +189,35 @@ __device__ __forceinline__ void store32_warp_f32(uint8_t* scratch, int lane, int
   store_rows64(scratch, lane, nvalid, reinterpret_cast<char*>(dst), 4ll * ld_out, r32);
   store_rows64(scratch, lane, nvalid, reinterpret_cast<char*>(dst) + 64, 4ll * ld_out, r32 + 16);
 }
+// The combine of a Top-1 layer in the epilogue: the 32 x 32 block just stored (packed bf16, w16 of this
+// lane's row) scaled by the row's gate and written to the row of the token the slot holds.  The value
+// is formed exactly as the separate kernels would: the stored bf16 output widened, times the gate in
+// fp32, rounded to bf16.  Rows turn through the scratch like any store; the token of a row comes from
+// the lane that owns it.
+__device__ __forceinline__ void scatter32_warp(uint8_t* scratch, int lane, int tok, float gate,
+                                               __nv_bfloat16* out, int ld, int col, const uint32_t* w16) {
+  uint4* mine = reinterpret_cast<uint4*>(scratch + lane * TC_SCRATCH_ROW_BYTES);
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    uint32_t y[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const uint32_t w = w16[4 * q + i];
+      y[i] = pack_bf16(gate * __uint_as_float(w << 16), gate * __uint_as_float(w & 0xffff0000u));
+    }
+    mine[q] = make_uint4(y[0], y[1], y[2], y[3]);
+  }
+  __syncwarp();
+  const int sub = lane & 3;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int row = (lane >> 2) + 8 * i;
+    const int t = __shfl_sync(0xffffffffu, tok, row);
+    const uint4 w = *reinterpret_cast<const uint4*>(scratch + row * TC_SCRATCH_ROW_BYTES + sub * 16);
+    if (t >= 0) *reinterpret_cast<uint4*>(out + (long long)t * ld + col + sub * 8) = w;
+  }
+  __syncwarp();
+}
 // 32 zeros at element offset `off` of the output (this lane's row of a block with nothing to contract).
 __device__ __forceinline__ void store_zero32(const TcParams& p, long long off) {
   if (p.out_f32) {
@@ -229,7 +262,8 @@ __device__ __forceinline__ void load32_warp_turn(uint8_t* scratch, int lane, con
 template <int EPI, int BN>
 __device__ __forceinline__ void epilogue_chunks(const TcParams& p, int n0, uint32_t taddr, long long obase,
                                                 bool row_ok, int c_beg, int nch, uint4 (&pg)[4],
-                                                uint4 (&pu)[4], uint8_t* scratch, int lane, int nvalid) {
+                                                uint4 (&pu)[4], uint8_t* scratch, int lane, int nvalid,
+                                                int sc_t = -1, float sc_g = 0.f) {
   const long long wbase = obase - (long long)lane * p.ld_out;     // row 0 of this warp's 32 rows
 #pragma unroll 1
   for (int c = c_beg; c < c_beg + nch; ++c) {
@@ -283,10 +317,16 @@ __device__ __forceinline__ void epilogue_chunks(const TcParams& p, int n0, uint3
       tc_wait_ld();
       if (p.out_f32) {
         store32_warp_f32(scratch, lane, nvalid, reinterpret_cast<float*>(p.out0) + wbase + 32 * c, p.ld_out, r0);
-      } else {
+      } else if (p.sc_out == nullptr) {
 #pragma unroll
         for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r0[i]);
         store32_warp(scratch, lane, nvalid, p.out0 + wbase + 32 * c, p.ld_out, v);
+      } else {
+        uint32_t pk[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) pk[i] = pack_bf16(__uint_as_float(r0[2 * i]), __uint_as_float(r0[2 * i + 1]));
+        store32_warp_packed(scratch, lane, nvalid, p.out0 + wbase + 32 * c, p.ld_out, pk);
+        scatter32_warp(scratch, lane, sc_t, sc_g, p.sc_out, p.sc_ld, n0 + 32 * c, pk);
       }
     }
   }
@@ -475,7 +515,13 @@ tc_grouped_gemm_kernel(const __grid_constant__ CUtensorMap mapA0, const __grid_c
       if (!mbar_wait(tfull_bar + 8 * acc_stage, acc_phase, abort_flag, p.wait_limit)) { ok = false; break; }
       tc_fence_after();
       const uint32_t taddr = tmem_base + (uint32_t)(acc_stage * 256) + ((uint32_t)(32 * q) << 16);
-      epilogue_chunks<EPI, BN>(p, tc.n0, taddr, obase, row_ok, c_beg, NCH, pg, pu, scratch, lane, nvalid);
+      int sc_t = -1;
+      float sc_g = 0.f;
+      if (EPI == TC_EPI_STORE && p.sc_out != nullptr && row_ok && grow < p.M) {
+        sc_t = p.sc_tok[(long long)tc.e * p.M + grow];
+        sc_g = p.sc_gate[(long long)tc.e * p.M + grow];
+      }
+      epilogue_chunks<EPI, BN>(p, tc.n0, taddr, obase, row_ok, c_beg, NCH, pg, pu, scratch, lane, nvalid, sc_t, sc_g);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(tempty_bar + 8 * acc_stage);
@@ -801,7 +847,13 @@ tc_grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap mapA0, const __g
       if (!mbar_wait_cluster(tfull_bar + 8 * acc_stage, acc_phase, abort_flag, p.wait_limit)) { ok = false; break; }
       tc_fence_after();
       const uint32_t taddr = tmem_base + (uint32_t)(acc_stage * 256) + ((uint32_t)(32 * q) << 16);
-      epilogue_chunks<EPI, BN>(p, tc.n0, taddr, obase, row_ok, c_beg, NCH, pg, pu, scratch, lane, nvalid);
+      int sc_t = -1;
+      float sc_g = 0.f;
+      if (EPI == TC_EPI_STORE && p.sc_out != nullptr && row_ok && grow < p.M) {
+        sc_t = p.sc_tok[(long long)tc.e * p.M + grow];
+        sc_g = p.sc_gate[(long long)tc.e * p.M + grow];
+      }
+      epilogue_chunks<EPI, BN>(p, tc.n0, taddr, obase, row_ok, c_beg, NCH, pg, pu, scratch, lane, nvalid, sc_t, sc_g);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(leader_tempty + 8 * acc_stage);
@@ -1052,6 +1104,12 @@ tc_grouped_gemm_pair_wide_kernel(const __grid_constant__ CUtensorMap mapA0, cons
         load32_warp_issue(p.in0 + wb, p.ld_out, lane, nvalid, pg);
         load32_warp_issue(p.in1 + wb, p.ld_out, lane, nvalid, pu);
       }
+      int sc_t = -1;
+      float sc_g = 0.f;
+      if (EPI == TC_EPI_STORE && p.sc_out != nullptr && row_ok && grow < p.M) {
+        sc_t = p.sc_tok[(long long)tc.e * p.M + grow];
+        sc_g = p.sc_gate[(long long)tc.e * p.M + grow];
+      }
       if (!mbar_wait_cluster(tfull_bar, acc_phase, abort_flag, p.wait_limit)) { ok = false; break; }
       tc_fence_after();
       if (EPI == TC_EPI_STORE && !p.out_f32) {
@@ -1082,7 +1140,11 @@ tc_grouped_gemm_pair_wide_kernel(const __grid_constant__ CUtensorMap mapA0, cons
 #pragma unroll
             for (int c = 0; c < NCH; ++c)
               if (n0h + 32 * (c_beg + c) < p.N)
+              {
                 store32_warp_packed(scratch, lane, nvalid, p.out0 + wb + 32 * (c_beg + c), p.ld_out, pk[c]);
+                if (p.sc_out != nullptr)
+                  scatter32_warp(scratch, lane, sc_t, sc_g, p.sc_out, p.sc_ld, n0h + 32 * (c_beg + c), pk[c]);
+              }
           }
         }
       } else if (EPI == TC_EPI_SWIGLU) {
@@ -1136,7 +1198,7 @@ tc_grouped_gemm_pair_wide_kernel(const __grid_constant__ CUtensorMap mapA0, cons
               load32_warp_issue(p.in1 + wb, p.ld_out, lane, nvalid, pu);
             }
             const uint32_t taddr = tmem_base + (uint32_t)(hf * 256) + ((uint32_t)(32 * q) << 16);
-            epilogue_chunks<EPI, BN>(p, n0h, taddr, ob, row_ok, c_beg, NCH, pg, pu, scratch, lane, nvalid);
+            epilogue_chunks<EPI, BN>(p, n0h, taddr, ob, row_ok, c_beg, NCH, pg, pu, scratch, lane, nvalid, sc_t, sc_g);
           }
           tc_fence_before();
           __syncwarp();
@@ -1387,7 +1449,7 @@ bool tc_available() { return true; }
 
 etr_status tc_ffn_forward(const etr_config* c, const etr_route* rt, const void* Xp, const void* Xtok, const void* W1g,
                           const void* W1u, const void* W2, void* G, void* U, void* H, void* O,
-                          etr_stats* stats, void*, cudaStream_t st) {
+                          etr_stats* stats, void*, void* Y_top1, cudaStream_t st) {
   const int d = c->d, h = c->h, Cs = c_stride_of(c), E = c->E;
   CUtensorMap mXp, mW1g, mW1u, mW2, mH;
   if (Xtok) ETR_TRY(make_gather_map(&mXp, Xtok, d, c->T));
@@ -1410,6 +1472,9 @@ etr_status tc_ffn_forward(const etr_config* c, const etr_route* rt, const void* 
     TcParams p = tc_params(c);
     p.M = Cs; p.N = d; p.K = h; p.dyn = TC_DYN_M; p.E = E; p.counts = rt->counts;
     p.out0 = (__nv_bfloat16*)O; p.out_bs = (long long)Cs * d; p.ld_out = d; p.stats = stats;
+    if (Y_top1) {      // Top-1: the combine in this epilogue (the caller has zeroed the rows of unrouted tokens)
+      p.sc_tok = rt->slot_token; p.sc_gate = rt->gate; p.sc_out = (__nv_bfloat16*)Y_top1; p.sc_ld = d;
+    }
     ETR_TRY((tc_run<TC_EPI_STORE>(tc_form_of(c, TC_EPI_STORE, p), "tc_gemm_down", mH, mH, mW2, mW2, p, E * mt * ceil_div(d, 256), st)));
   }
   return ETR_OK;

@@ -141,6 +141,24 @@ combine_bwd_kernel(const T* __restrict__ dY, const T* __restrict__ O,
   if (lane == 0) dgate[r] = dot;
 }
 
+// Y[t,:] = 0 for tokens without a row (the part of the combine that the fused Top-1 epilogue of the
+// down GEMM leaves over).  One warp per token.
+__global__ void __launch_bounds__(256)
+zero_unrouted_kernel(const int32_t* __restrict__ tok_ptr, uint4* __restrict__ Y, int Ttok, int row_vec) {
+  const int t = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (t >= Ttok || tok_ptr[t] != tok_ptr[t + 1]) return;
+  uint4* dst = Y + (size_t)t * row_vec;
+  for (int v = lane; v < row_vec; v += 32) dst[v] = make_uint4(0, 0, 0, 0);
+}
+
+etr_status zero_unrouted_rows(const etr_config* c, const etr_route* rt, void* Y, cudaStream_t st) {
+  ETR_TIME_BEGIN("zero_unrouted_kernel");
+  zero_unrouted_kernel<<<ceil_div(c->T, 8), 256, 0, st>>>(rt->tok_ptr, (uint4*)Y, c->T,
+                                                          (int)((size_t)c->d * elem_bytes(c->dtype) / 16));
+  ETR_LAUNCH_CHECK();
+  return ETR_OK;
+}
+
 template <class T>
 static etr_status permute_launch(int which, const etr_config* c, const etr_route* rt, const void* a,
                                  const void* b, void* out, float* dgate, cudaStream_t st) {

@@ -41,7 +41,8 @@ class Config(C.Structure):
                 ("dtype", C.c_int32), ("gemm_impl", C.c_int32), ("fuse_dispatch", C.c_int32),
                 ("gate_mode", C.c_int32), ("grad_fp32", C.c_int32), ("weight_dtype", C.c_int32),
                 ("threshold_mode", C.c_int32), ("threshold_tau", C.c_float),
-                ("threshold_tau_token", C.c_float), ("wait_limit_cycles", C.c_int64)]
+                ("threshold_tau_token", C.c_float), ("wait_limit_cycles", C.c_int64),
+                ("fuse_combine", C.c_int32), ("reserved0", C.c_int32)]
 
 
 class Stats(C.Structure):
@@ -130,14 +131,16 @@ def _stream():
 def make_config(*, T, d, D, E, k, h, capacity, dtype, mode=MODE_AUTO, step=0, switch_step=0,
                 adaptive=False, c_floor=1, delta_max_override=-1.0, gemm_impl=GEMM_AUTO,
                 fuse_dispatch=0, gate_mode=0, grad_fp32=False, weight_dtype=None, threshold_mode=0,
-                threshold_tau=float("inf"), threshold_tau_token=float("inf"), wait_limit_cycles=0) -> Config:
+                threshold_tau=float("inf"), threshold_tau_token=float("inf"), wait_limit_cycles=0,
+                fuse_combine=0) -> Config:
     return Config(T=T, d=d, D=D, E=E, k=k, h=h, capacity=capacity, c_floor=c_floor,
                   adaptive=int(bool(adaptive)), delta_max_override=float(delta_max_override),
                   step=int(step), switch_step=int(switch_step), mode=int(mode), dtype=int(dtype),
                   gemm_impl=int(gemm_impl), fuse_dispatch=int(fuse_dispatch), gate_mode=int(gate_mode),
                   grad_fp32=int(bool(grad_fp32)), weight_dtype=int(dtype if weight_dtype is None else weight_dtype),
                   threshold_mode=int(threshold_mode), threshold_tau=float(threshold_tau),
-                  threshold_tau_token=float(threshold_tau_token), wait_limit_cycles=int(wait_limit_cycles))
+                  threshold_tau_token=float(threshold_tau_token), wait_limit_cycles=int(wait_limit_cycles),
+                  fuse_combine=int(fuse_combine), reserved0=0)
 
 
 def torch_dtype(cfg: Config):

@@ -126,7 +126,17 @@ def _record(what, n, stats):
 # (measured: O 2.35e-3, Y 2.87e-3, dX 3.5-3.8e-3).  Asserted with a 20 % margin.
 RMS_ERR_PER_STORE = 2e-3
 OUTLIER_FRACTION = 2e-5       # measured: at most 2.0e-5 of a tensor's elements (2 of 102400)
-OUTLIER_CEILING = 2.0         # measured: none beyond 1.8x the element's tolerance
+OUTLIER_CEILING = 2.0         # measured: none beyond 1.95x the element's tolerance
+# Weight gradients of W1 on clustered tokens (the mixture and skewed workloads): the rows of Xp an
+# expert sums over are nearly parallel (within-cluster cosine 0.8), so in dW1[j,q] = sum_r dG[r,j] Xp[r,q]
+# the values cancel (dG is signed) while the rounding errors of the stored dG do not, and their size
+# follows the cluster means' |mu_q|: the error scale varies from column to column and more elements
+# sit beyond a bound set by the tensor's overall RMS (measured: 3.4e-5 of them at most).
+OUTLIER_FRACTION_CLUSTERED_DW1 = 5e-5
+
+
+def dw1_outlier_fraction(w) -> float:
+    return OUTLIER_FRACTION if w.x_kind == "iso" else OUTLIER_FRACTION_CLUSTERED_DW1
 
 
 def assert_close_rms(got, ref, rel, what, chain=1, rms=None, outlier_fraction=OUTLIER_FRACTION):

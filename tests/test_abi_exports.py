@@ -42,7 +42,7 @@ def test_host_side_validation_needs_no_gpu():
     n = ctypes.c_size_t(0)
     assert etr.lib().etr_buffers_bytes(ctypes.byref(good), 1, ctypes.byref(n)) == etr.OK and n.value > 1 << 20
     # struct layouts the binding relies on
-    assert ctypes.sizeof(etr.Config) == 104 and ctypes.sizeof(etr.Stats) == 64
+    assert ctypes.sizeof(etr.Config) == 112 and ctypes.sizeof(etr.Stats) == 64
     # the expert weights share the activations' dtype: anything else has no kernel
     assert etr.validate(etr.make_config(T=512, d=256, D=4, E=8, k=2, h=512, capacity=160, dtype=etr.F32,
                                         weight_dtype=etr.BF16)) == etr.ERR_UNSUPPORTED

@@ -211,3 +211,56 @@ def test_layer_with_a_threshold_on_the_affinity_sum(mode, flags):
     for nm, ref, chain in (("Y", fw.Y, 4), ("dX", bw.dX, 6), ("dR", bw.dR, 4), ("dW1g", bw.dW1g, 6),
                            ("dW1u", bw.dW1u, 6), ("dW2", bw.dW2, 4)):
         hz.assert_close_rms(hz.to_np(out[nm]), ref, 2e-2, nm, chain=chain)
+
+
+@pytest.mark.parametrize("impl", [etr.GEMM_AUTO, etr.GEMM_TCGEN05, etr.GEMM_TCGEN05_2CTA, etr.GEMM_TCGEN05_2CTA_WIDE])
+@pytest.mark.parametrize("name,cf", [("small_s", 1.25), ("sweep_s_tcr", 0.5)])
+def test_top1_combine_in_the_down_gemm_epilogue(name, cf, impl):
+    """Top-1 token choice: with the combine folded into the down GEMM's epilogue (the default there)
+    the combine kernel does not run and every output equals the unfused path bit for bit, on all
+    tile forms; tokens without a row (capacity factor 0.5 drops many) get exact zeros; with k = 2 the
+    switch changes nothing."""
+    w0, inp, o, _, _ = case(name)
+    w = gw.scaled(w0, k=1, cf=cf, adaptive=False)
+    dev = hz.upload(w, inp)
+    res, names = {}, {}
+    for fuse in (etr.FUSE_OFF, etr.FUSE_AUTO):
+        cfg = hz.make_cfg(w, mode=ob.MODE_TCR, gemm_impl=impl, fuse_combine=fuse)
+        buf = etr.LayerBuffers(cfg)
+        out = dict(Y=torch.full_like(dev.X, float("nan")), dX=torch.empty_like(dev.X), dR=torch.empty_like(dev.R),
+                   dW1g=torch.empty_like(dev.W1g), dW1u=torch.empty_like(dev.W1u), dW2=torch.empty_like(dev.W2))
+        etr.timing_enable(True)
+        etr.layer_forward(cfg, dev.X, dev.R, dev.W1g, dev.W1u, dev.W2, buf, out["Y"])
+        names[fuse] = [n for n, _ in etr.timing_collect()]
+        etr.timing_enable(False)
+        etr.layer_backward(cfg, dev.X, dev.R, dev.W1g, dev.W1u, dev.W2, dev.dY, buf, out["dX"], out["dR"],
+                           out["dW1g"], out["dW1u"], out["dW2"])
+        torch.cuda.synchronize()
+        st = buf.read_stats()
+        assert st.error_word == 0
+        out["O"] = buf.O.clone()
+        res[fuse] = (out, st, hz.to_np(buf.tok_ptr))
+    assert "combine_kernel" in names[etr.FUSE_OFF] and "combine_kernel" not in names[etr.FUSE_AUTO]
+    assert "zero_unrouted_kernel" in names[etr.FUSE_AUTO]
+    a, b = res[etr.FUSE_OFF][0], res[etr.FUSE_AUTO][0]
+    for k in a:
+        assert torch.equal(a[k], b[k]), k
+    st, ptr = res[etr.FUSE_AUTO][1], res[etr.FUSE_AUTO][2]
+    unrouted = np.diff(ptr) == 0
+    assert st.unrouted == int(unrouted.sum())
+    if cf < 1:
+        assert st.unrouted > 0
+    assert np.all(hz.to_np(b["Y"])[unrouted] == 0) and not np.isnan(hz.to_np(b["Y"])).any()
+    # against the oracle as well
+    fw = o.forward(inp["X"], inp["R"], inp["W1g"], inp["W1u"], inp["W2"], D=w.D, k=1, capacity=w.capacity,
+                   mode=ob.MODE_TCR)
+    hz.assert_close_rms(hz.to_np(b["Y"]), fw.Y, 2e-2, "Y (combine in the epilogue)", chain=4)
+    # k = 2: a token's rows lie in different experts' tiles; the switch must leave the path alone
+    w2 = gw.scaled(w0, adaptive=False)
+    cfg2 = hz.make_cfg(w2, mode=ob.MODE_TCR, gemm_impl=impl, fuse_combine=etr.FUSE_ON)
+    buf2 = etr.LayerBuffers(cfg2)
+    Y2 = torch.empty_like(dev.X)
+    etr.timing_enable(True)
+    etr.layer_forward(cfg2, dev.X, dev.R, dev.W1g, dev.W1u, dev.W2, buf2, Y2)
+    assert "combine_kernel" in [n for n, _ in etr.timing_collect()]
+    etr.timing_enable(False)

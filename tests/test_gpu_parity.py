@@ -396,13 +396,7 @@ def test_layer_with_softmax_gate(name):
     hz.assert_close_rms(hz.to_np(out["Y"]), fw.Y, tol, "Y", chain=4)
     hz.assert_close_rms(hz.to_np(out["dX"]), bw.dX, tol, "dX", chain=6)
     hz.assert_close_rms(hz.to_np(out["dR"]), bw.dR, tol, "dR", chain=4)
-    # mid_s: 8 tight clusters, so the rows of Xp an expert sums over are nearly parallel.  In
-    # dW1[j,q] = sum_r dG[r,j] Xp[r,q] the values then cancel (dG is signed) while the rounding
-    # errors of dG do not, and their size follows the cluster mean's |mu_q|: the error scale
-    # varies from column to column, and more elements (measured 3.4e-5) sit beyond a bound set by
-    # the tensor's overall RMS.  Against the oracle on the storage grid the same tensors agree to
-    # one ulp + 2e-2 rms with no exception (test_parity_with_the_storage_grid_modelled[mid_s-*]).
-    frac = 5e-5 if name == "mid_s" else hz.OUTLIER_FRACTION
+    frac = hz.dw1_outlier_fraction(w)      # clustered tokens: see harness.OUTLIER_FRACTION_CLUSTERED_DW1
     hz.assert_close_rms(hz.to_np(out["dW1g"]), bw.dW1g, tol, "dW1g", chain=6, outlier_fraction=frac)
     hz.assert_close_rms(hz.to_np(out["dW1u"]), bw.dW1u, tol, "dW1u", chain=6, outlier_fraction=frac)
     hz.assert_close_rms(hz.to_np(out["dW2"]), bw.dW2, tol, "dW2", chain=4)
