@@ -84,10 +84,10 @@ typedef enum { ETR_FUSE_AUTO = 0, ETR_FUSE_OFF = 1, ETR_FUSE_ON = 2 } etr_fuse;
  * gives every expert of a routed token a gradient (a dense d delta), see etr_gate_softmax_bwd. */
 typedef enum { ETR_GATE_AFFINITY = 0, ETR_GATE_SOFTMAX = 1 } etr_gate;
 
-/* Number of kept candidates set by a threshold on the sum of affinity scores ("Routing Strategy":
- * the expert chooses its Top-l tokens with l determined by a threshold of the sum of affinity
- * scores; "Training Strategy": the number of tokens per expert follows an adaptive threshold).  The
- * paper gives no rule, so this is a reading: walking a candidate list in descending affinity, the
+/* Number of kept candidates limited by the accumulated affinity ("Routing Strategy", the sentence
+ * that introduces the expert-side equation: how many tokens an expert takes depends on the sum of
+ * their affinity scores; "Training Strategy": that number adapts during training).  The paper gives
+ * no rule, so this is a reading: walking a candidate list in descending affinity, the
  * candidate of rank j is kept while the sum of the j-1 affinities before it is still below tau (and
  * j is within the capacity C, resp. k).  EXPERT applies it to every expert's candidate tokens (both
  * modes), TOKEN to every token's experts (token choice only: a token then takes 1..k experts and

@@ -166,9 +166,10 @@ void select(int T, int E, int k, int mode, int C, int C_stride, const S* delta,
 }
 
 // ---- selection with a threshold on the sum of affinity scores ------------------------------
-// "Routing Strategy" says that the number l of tokens an expert takes "is determined by a
-// threshold of the sum of affinity scores", and "Training Strategy" that the number of tokens per
-// expert follows an adaptive threshold; neither gives the rule.  The reading implemented here
+// In "Routing Strategy" (the sentence that introduces the expert-side equation) the number l of
+// tokens an expert takes depends on how large the accumulated affinity of its tokens has become,
+// and "Training Strategy" says this number adapts during training; neither passage gives the rule.
+// The reading implemented here
 // (parity unpinned as a reading; the function itself is pinned by brute force over prefixes, by
 // its limits tau = +infinity and tau <= first score, and by monotonicity in tau):
 //

@@ -308,8 +308,9 @@ def test_select_reductions(o32):
 
 
 # ------------------------------------------ threshold on the sum of affinity scores ------------
-# The rule ("Routing Strategy": the number of tokens an expert takes follows a threshold of the sum
-# of affinity scores) is pinned without restating its loop: by exhaustive search over prefix
+# The rule (a reading of the sentence that introduces the expert-side equation of "Routing
+# Strategy": an expert stops taking tokens once their accumulated affinity is large enough) is
+# pinned without restating its loop: by exhaustive search over prefix
 # lengths in exact rational arithmetic, by its two limits, by a closed form on constant scores and
 # by monotonicity in tau.
 
