@@ -21,7 +21,9 @@ The backward pass uses the same two row exchanges with the roles swapped (d O ro
 Everything here is tensor plumbing on `torch.distributed` (gloo on CPU tensors in the tests, NCCL on
 CUDA tensors in deployment); the arithmetic of each rank stays in the library's kernels.  No kernel
 ever reads another GPU's memory: rows are copied into this rank's own buffers before any is used.
-This module is covered by two-rank CPU tests; it has not run on several GPUs.
+Covered by a two-rank CPU test of the exchanges against the oracle and by a GPU test in which two
+ranks share one GPU (`ExpertParallelLayer`, exchanges over gloo); it has not run on several GPUs, so
+it has no performance figure.
 """
 from __future__ import annotations
 
@@ -32,8 +34,23 @@ import torch.distributed as dist
 
 
 def _a2a(out, inp, out_splits, in_splits, group):
+    if inp.is_cuda and dist.get_backend(group) == "gloo":     # gloo moves host memory: stage through it
+        o = torch.empty(out.shape, dtype=out.dtype)
+        dist.all_to_all_single(o, inp.cpu(), list(out_splits), list(in_splits), group=group)
+        out.copy_(o)
+        return out
     dist.all_to_all_single(out, inp, list(out_splits), list(in_splits), group=group)
     return out
+
+
+def _all_reduce(t, op, group):
+    if t.is_cuda and dist.get_backend(group) == "gloo":
+        h = t.cpu()
+        dist.all_reduce(h, op=op, group=group)
+        t.copy_(h)
+    else:
+        dist.all_reduce(t, op=op, group=group)
+    return t
 
 
 def exchange_affinities(delta_local: torch.Tensor, group=None):
@@ -48,7 +65,7 @@ def exchange_affinities(delta_local: torch.Tensor, group=None):
     n = T_local * E_local
     _a2a(recv.view(-1), send.view(-1), [n] * W, [n] * W, group)
     dmax = delta_local.max().reshape(1).clone()
-    dist.all_reduce(dmax, op=dist.ReduceOp.MAX, group=group)
+    _all_reduce(dmax, dist.ReduceOp.MAX, group)
     return recv.view(W * T_local, E_local), dmax[0]
 
 
@@ -63,6 +80,7 @@ class ExchangePlan:
     want_rows: list          # [W] int64 tensors: row ids in this rank's [E_local * C_stride] buffers
     send_tokens: list        # [W] int64 tensors: local token ids to send to each rank
     send_gates: list         # [W] float tensors: gate of each of those rows
+    send_rows: list          # [W] int64 tensors: the row each of them fills in the destination's buffers
     rows_in: list            # splits of rows received by the expert side, per source rank
     rows_out: list           # splits of rows sent by the token side, per destination rank
 
@@ -84,10 +102,12 @@ def build_plan(slot_token: torch.Tensor, gate: torch.Tensor, T_local: int, group
     ask_gate = torch.cat([gate[r] for r in want_rows])
     got_tok = torch.empty(sum(rows_out), dtype=torch.int64, device=slot_token.device)
     got_gate = torch.empty(sum(rows_out), dtype=gate.dtype, device=gate.device)
+    got_row = torch.empty(sum(rows_out), dtype=torch.int64, device=slot_token.device)
     _a2a(got_tok, ask_tok, rows_out, rows_in, group)
     _a2a(got_gate, ask_gate, rows_out, rows_in, group)
+    _a2a(got_row, torch.cat(want_rows), rows_out, rows_in, group)
     return ExchangePlan(W, rank, T_local, want_rows, list(got_tok.split(rows_out)),
-                        list(got_gate.split(rows_out)), rows_in, rows_out)
+                        list(got_gate.split(rows_out)), list(got_row.split(rows_out)), rows_in, rows_out)
 
 
 def dispatch_rows(plan: ExchangePlan, X_local: torch.Tensor, n_buffer_rows: int, group=None) -> torch.Tensor:
@@ -151,3 +171,93 @@ def combine_local(plan: ExchangePlan, rows_back: torch.Tensor, accumulate_dtype=
             Y[tok_s[sel]] += part_s[sel]
         off += n
     return Y
+
+
+def with_unit_gates(plan: ExchangePlan) -> ExchangePlan:
+    """The same plan with every gate 1: `combine_local` then is the plain sum of a token's rows
+    (the dispatch backward, d X[t] = sum of the token's rows of d Xp)."""
+    return ExchangePlan(plan.world, plan.rank, plan.T_local, plan.want_rows, plan.send_tokens,
+                        [torch.ones_like(g) for g in plan.send_gates], plan.send_rows, plan.rows_in,
+                        plan.rows_out)
+
+
+class ExpertParallelLayer:
+    """Forward and backward of the layer with the experts spread over the ranks of `group`, expert
+    choice, fixed capacity: the per-rank arithmetic runs in the library's kernels (affinity, selection,
+    expert FFN and their backward forms through the C ABI), the exchanges in the functions above.
+
+    Every rank passes its T_local tokens, the full expert embeddings R [E, m] and the weights of its
+    own experts [E_local, ...].  The adaptive capacity bound needs the batch maximum of the affinities
+    over all ranks, which `exchange_affinities` returns; here the capacity is the caller's number."""
+
+    def __init__(self, *, T_local, d, D, E, h, capacity, group=None, device="cuda"):
+        from . import etr
+        self.etr, self.group = etr, group
+        self.W, self.rank = dist.get_world_size(group), dist.get_rank(group)
+        assert E % self.W == 0
+        self.T_local, self.T, self.E, self.E_local, self.d, self.D, self.h = T_local, T_local * self.W, E, E // self.W, d, D, h
+        # the local tokens against all experts (S1 and the dense router backward)
+        self.cfg_tok = etr.make_config(T=T_local, d=d, D=D, E=E, k=1, h=h, capacity=capacity, dtype=etr.BF16,
+                                       mode=etr.MODE_ECR, gate_mode=etr.GATE_SOFTMAX)
+        # the local experts over all tokens (S3, S5 and their backward)
+        self.cfg_own = etr.make_config(T=self.T, d=d, D=D, E=self.E_local, k=1, h=h, capacity=capacity,
+                                       dtype=etr.BF16, mode=etr.MODE_ECR)
+        self.own = etr.LayerBuffers(self.cfg_own, device=device)
+        self.rows = self.E_local * etr.c_stride(self.cfg_own)
+        f32 = dict(dtype=torch.float32, device=device)
+        m = d // D
+        self.delta = torch.empty(T_local, E, **f32)
+        self.Z = torch.empty(T_local, m, **f32)
+        self.xnorm, self.rnorm = torch.empty(T_local, **f32), torch.empty(E, **f32)
+        self.stats_tok = torch.zeros(16, dtype=torch.int32, device=device)
+        self.ws_tok = torch.empty(etr.workspace_bytes(self.cfg_tok), dtype=torch.uint8, device=device)
+        self.ws_own = torch.empty(etr.workspace_bytes(self.cfg_own), dtype=torch.uint8, device=device)
+
+    def forward(self, X, R, W1g, W1u, W2):
+        etr, own = self.etr, self.own
+        self.stats_tok.zero_()
+        etr.affinity(self.cfg_tok, X, R, self.delta, self.Z, self.xnorm, self.rnorm, self.stats_tok)
+        delta_own, self.delta_max = exchange_affinities(self.delta, self.group)
+        own.delta.copy_(delta_own)
+        own.stats.zero_()
+        etr.select(self.cfg_own, own.delta, own.c.stats, own.route, self.ws_own)
+        self.plan = build_plan(own.slot_token, own.gate, self.T_local, self.group)
+        own.Xp.copy_(dispatch_rows(self.plan, X, self.rows, self.group))
+        etr.expert_ffn(self.cfg_own, own.route, own.Xp, W1g, W1u, W2, own.G, own.U, own.H, own.O, own.c.stats,
+                       self.ws_own)
+        self.O_back = return_rows(self.plan, own.O, self.group)
+        return combine_local(self.plan, self.O_back).to(X.dtype)
+
+    def backward(self, X, R, W1g, W1u, W2, dY):
+        """Returns dX [T_local, d], dR [E, m] (summed over the ranks) and the weight gradients of the local
+        experts."""
+        etr, own, plan = self.etr, self.own, self.plan
+        send_tok = torch.cat(plan.send_tokens)
+        gates = torch.cat(plan.send_gates)
+        dY_rows = dY[send_tok].float()
+        own.dO.copy_(scatter_rows_to_experts(plan, (dY_rows * gates[:, None]).to(dY.dtype), self.rows, self.group))
+        dgate_rows = (dY_rows * self.O_back.float()).sum(1)
+        dW1g, dW1u, dW2 = torch.empty_like(W1g), torch.empty_like(W1u), torch.empty_like(W2)
+        etr.expert_ffn_bwd(self.cfg_own, own.route, own.dO, own.Xp, own.G, own.U, own.H, W1g, W1u, W2, own.dG,
+                           own.dU, own.dXp, dW1g, dW1u, dW2, own.c.stats, self.ws_own)
+        dX = combine_local(with_unit_gates(plan), return_rows(plan, own.dXp, self.group)).to(dY.dtype)
+        # router gradient of the local tokens: d delta is non-zero on the token's selected pairs
+        Cs = self.rows // self.E_local
+        expert = torch.cat([q * self.E_local + torch.div(r, Cs, rounding_mode="floor")
+                            for q, r in enumerate(plan.send_rows)])
+        ddelta = torch.zeros_like(self.delta)
+        ddelta[send_tok, expert] = dgate_rows
+        n_rows = torch.zeros(self.T_local, dtype=torch.int32, device=dY.device)
+        n_rows.index_add_(0, send_tok, torch.ones_like(send_tok, dtype=torch.int32))
+        tok_ptr = torch.zeros(self.T_local + 1, dtype=torch.int32, device=dY.device)
+        tok_ptr[1:] = torch.cumsum(n_rows, 0)
+        spare = torch.zeros(max(int(tok_ptr[-1]), 4), dtype=torch.int32, device=dY.device)
+        route = etr.Route(spare.data_ptr(), spare.data_ptr(), spare.data_ptr(), spare.data_ptr(),
+                          tok_ptr.data_ptr(), spare.data_ptr())          # only tok_ptr is read: which tokens have rows
+        dR = torch.empty_like(R)
+        etr.affinity_bwd_dense(self.cfg_tok, X, R, self.delta, self.Z, self.xnorm, self.rnorm, route, ddelta, dX,
+                               dR, self.ws_tok)
+        _all_reduce(dR, dist.ReduceOp.SUM, self.group)
+        st = etr.read_stats(own.c.stats)
+        assert st.error_word == 0
+        return dX, dR, dW1g, dW1u, dW2

@@ -86,8 +86,10 @@ def _rank_main(rank, world, port, q):
         dgate = ep.scatter_rows_to_experts(plan, dgate_rows, El * Cs)[:, 0]
         assert np.allclose(dgate.numpy(), bw.dgate[rows], rtol=1e-12, atol=1e-300)
         dXp_back = ep.return_rows(plan, t(np.ascontiguousarray(bw.dXp[rows])))
-        ones = ep.ExchangePlan(plan.world, plan.rank, plan.T_local, plan.want_rows, plan.send_tokens,
-                               [torch.ones_like(g) for g in plan.send_gates], plan.rows_in, plan.rows_out)
+        for qq in range(world):          # the token side knows which buffer row each of its rows fills
+            own_rows = np.arange(qq * El * Cs, (qq + 1) * El * Cs)[plan.send_rows[qq].numpy()]
+            assert np.array_equal(fw.route.slot_token[own_rows], plan.send_tokens[qq].numpy() + rank * Tl)
+        ones = ep.with_unit_gates(plan)
         dX_ffn = ep.combine_local(ones, dXp_back, torch.float64)
         assert np.allclose(dX_ffn.numpy(), bw.dX_ffn[tok], rtol=1e-14, atol=1e-300)
         q.put((rank, "ok", sum(plan.rows_in), sum(plan.rows_out)))
