@@ -183,6 +183,21 @@ etr_status etr_buffers_bytes(const etr_config* cfg, int with_host_staging, size_
 etr_status etr_buffers_bind(const etr_config* cfg, int with_host_staging, void* base, size_t bytes,
                             etr_buffers* out);
 
+/* The same carving as plain numbers, for callers that place the buffers themselves: C_stride, the
+ * size of the block, and the byte offset of every etr_buffers member from a 256-byte aligned base
+ * (members a config does not use have offset 0 and size 0: the host staging without
+ * with_host_staging, lse and ddelta without the softmax gate).  etr_buffers_bind(base) equals
+ * base + these offsets. */
+typedef struct etr_layout_info {
+  int32_t C_stride;
+  int32_t reserved;
+  size_t total_bytes, ws_bytes;
+  size_t stats, topk_idx, counts, slot_token, gate, tok_ptr, tok_row;
+  size_t delta, Z, xnorm, rnorm, Xp, G, U, H, O, dO, dG, dU, dXp, dgate, ws;
+  size_t X_dev, dY_dev, Y_dev, dX_dev, lse, ddelta;
+} etr_layout_info;
+etr_status etr_layout(const etr_config* cfg, int with_host_staging, etr_layout_info* out);
+
 /* ---- forward stages ---------------------------------------------------------------- */
 
 /* GrAP pooling and cosine affinity ("Cost-Efficient Sparse Expert-Token Affinity": the
@@ -372,6 +387,8 @@ etr_status etr_layer_step_host_wait(int32_t slot);
 /* Copies the device stats to the host and synchronises the stream.  Returns
  * ETR_ERR_TIMEOUT if a kernel recorded an expired wait. */
 etr_status etr_read_stats(const etr_stats* stats_dev, etr_stats* stats_host, void* stream);
+/* The same call under the name the status word suggests. */
+etr_status etr_read_status(const etr_stats* stats_dev, etr_stats* stats_host, void* stream);
 
 /* Self-test of the bounded device-side wait (the failure path of the GEMM pipeline, which a healthy
  * run never takes): launches one warp that waits, with the pipeline's own wait routine, on a

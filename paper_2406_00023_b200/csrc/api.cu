@@ -204,6 +204,30 @@ etr_status etr_buffers_bind(const etr_config* c, int with_host_staging, void* ba
   return ETR_OK;
 }
 
+etr_status etr_layout(const etr_config* c, int with_host_staging, etr_layout_info* out) {
+  if (out == nullptr) return ETR_ERR_ARG;
+  ETR_TRY(etr_validate(c));
+  etr_buffers b;
+  size_t total = 0;
+  char* const base = reinterpret_cast<char*>(uintptr_t(256));      // any aligned non-null base: only differences are kept
+  carve(c, with_host_staging, base, &b, &total);
+  auto off = [&](const void* p) -> size_t { return p ? (size_t)(reinterpret_cast<const char*>(p) - base) : 0; };
+  memset(out, 0, sizeof(*out));
+  out->C_stride = c_stride_of(c);
+  out->total_bytes = total;
+  out->ws_bytes = b.ws_bytes;
+  out->stats = off(b.stats);
+  out->topk_idx = off(b.route.topk_idx); out->counts = off(b.route.counts); out->slot_token = off(b.route.slot_token);
+  out->gate = off(b.route.gate); out->tok_ptr = off(b.route.tok_ptr); out->tok_row = off(b.route.tok_row);
+  out->delta = off(b.delta); out->Z = off(b.Z); out->xnorm = off(b.xnorm); out->rnorm = off(b.rnorm);
+  out->Xp = off(b.Xp); out->G = off(b.G); out->U = off(b.U); out->H = off(b.H); out->O = off(b.O);
+  out->dO = off(b.dO); out->dG = off(b.dG); out->dU = off(b.dU); out->dXp = off(b.dXp); out->dgate = off(b.dgate);
+  out->ws = off(b.ws);
+  out->X_dev = off(b.X_dev); out->dY_dev = off(b.dY_dev); out->Y_dev = off(b.Y_dev); out->dX_dev = off(b.dX_dev);
+  out->lse = off(b.lse); out->ddelta = off(b.ddelta);
+  return ETR_OK;
+}
+
 etr_status etr_affinity(const etr_config* c, const void* X, const float* R, float* delta, float* Z,
                         float* xnorm, float* rnorm, etr_stats* stats, void* stream) {
   ETR_TRY(etr_validate(c));
@@ -527,6 +551,10 @@ etr_status etr_selftest_bounded_wait(etr_stats* stats, int64_t limit_cycles, voi
   if (stats == nullptr || limit_cycles < 1 || limit_cycles > 4000000000ll) return ETR_ERR_ARG;
   if (!aligned16(stats)) return ETR_ERR_ALIGN;
   return tc_wait_selftest(stats, (long long)limit_cycles, (cudaStream_t)stream);
+}
+
+etr_status etr_read_status(const etr_stats* dev, etr_stats* host, void* stream) {
+  return etr_read_stats(dev, host, stream);
 }
 
 int64_t etr_launch_count(void) { return (int64_t)g_launches.load(); }

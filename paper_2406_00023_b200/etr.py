@@ -24,7 +24,7 @@ THRESHOLD_OFF, THRESHOLD_EXPERT, THRESHOLD_TOKEN = 0, 1, 2
 
 EXPORTS = [
     "etr_status_string", "etr_validate", "etr_c_stride", "etr_workspace_bytes", "etr_buffers_bytes",
-    "etr_buffers_bind", "etr_affinity", "etr_select", "etr_select_static", "etr_dispatch", "etr_expert_ffn", "etr_combine",
+    "etr_buffers_bind", "etr_layout", "etr_read_status", "etr_affinity", "etr_select", "etr_select_static", "etr_dispatch", "etr_expert_ffn", "etr_combine",
     "etr_combine_bwd", "etr_expert_ffn_bwd", "etr_dispatch_bwd", "etr_select_bwd", "etr_affinity_bwd",
     "etr_gate_softmax", "etr_gate_softmax_bwd", "etr_affinity_bwd_dense", "etr_load_stats",
     "etr_layer_forward", "etr_layer_backward", "etr_layer_step_host", "etr_layer_step_host_begin",
@@ -62,6 +62,14 @@ class Buffers(C.Structure):
                                           "dO", "dG", "dU", "dXp", "dgate", "ws")] + \
                [("ws_bytes", C.c_size_t)] + \
                [(n, C.c_void_p) for n in ("X_dev", "dY_dev", "Y_dev", "dX_dev", "lse", "ddelta")]
+
+
+class LayoutInfo(C.Structure):
+    _fields_ = [("C_stride", C.c_int32), ("reserved", C.c_int32)] + \
+               [(n, C.c_size_t) for n in ("total_bytes", "ws_bytes", "stats", "topk_idx", "counts", "slot_token",
+                                          "gate", "tok_ptr", "tok_row", "delta", "Z", "xnorm", "rnorm", "Xp", "G",
+                                          "U", "H", "O", "dO", "dG", "dU", "dXp", "dgate", "ws", "X_dev", "dY_dev",
+                                          "Y_dev", "dX_dev", "lse", "ddelta")]
 
 
 class EtrError(RuntimeError):
@@ -153,6 +161,13 @@ def validate(cfg: Config) -> int:
 
 def c_stride(cfg: Config) -> int:
     return lib().etr_c_stride(C.byref(cfg))
+
+
+def layout(cfg: Config, host_staging: bool = False) -> LayoutInfo:
+    """Offsets of every buffer inside the block etr_buffers_bind carves."""
+    out = LayoutInfo()
+    _check(lib().etr_layout(C.byref(cfg), int(host_staging), C.byref(out)), "etr_layout")
+    return out
 
 
 def workspace_bytes(cfg: Config) -> int:

@@ -46,3 +46,26 @@ def test_host_side_validation_needs_no_gpu():
     # the expert weights share the activations' dtype: anything else has no kernel
     assert etr.validate(etr.make_config(T=512, d=256, D=4, E=8, k=2, h=512, capacity=160, dtype=etr.F32,
                                         weight_dtype=etr.BF16)) == etr.ERR_UNSUPPORTED
+
+
+def test_layout_gives_the_offsets_bind_uses():
+    from paper_2406_00023_b200 import etr
+    for staging, gate in ((0, etr.GATE_AFFINITY), (1, etr.GATE_SOFTMAX)):
+        cfg = etr.make_config(T=512, d=256, D=4, E=8, k=2, h=512, capacity=160, dtype=etr.BF16, gate_mode=gate)
+        lay = etr.layout(cfg, bool(staging))
+        n = ctypes.c_size_t(0)
+        assert etr.lib().etr_buffers_bytes(ctypes.byref(cfg), staging, ctypes.byref(n)) == etr.OK
+        assert lay.total_bytes == n.value and lay.C_stride == 256 and lay.ws_bytes == etr.workspace_bytes(cfg)
+        base = 1 << 20                                   # binding only computes addresses: no memory is touched
+        b = etr.Buffers()
+        assert etr.lib().etr_buffers_bind(ctypes.byref(cfg), staging, ctypes.c_void_p(base),
+                                          ctypes.c_size_t(n.value), ctypes.byref(b)) == etr.OK
+        for name in ("delta", "Z", "xnorm", "rnorm", "Xp", "G", "U", "H", "O", "dO", "dG", "dU", "dXp", "dgate", "ws"):
+            assert getattr(b, name) == base + getattr(lay, name), name
+            assert getattr(lay, name) % 256 == 0
+        assert b.route.slot_token == base + lay.slot_token and b.route.tok_row == base + lay.tok_row
+        assert b.stats == base + lay.stats
+        if staging:
+            assert b.X_dev == base + lay.X_dev and b.lse == base + lay.lse and lay.ddelta > lay.lse > 0
+        else:
+            assert lay.X_dev == 0 and lay.lse == 0 and not b.X_dev
