@@ -135,7 +135,9 @@ __device__ __forceinline__ void load32(const __nv_bfloat16* src, float* v) {
   }
 }
 
-struct TileCoord { int e, m0, n0, kblocks, m_lim; };
+// last_kk: 16-wide MMA steps of the last K block that hold rows in use (contractions over an expert's
+// rows: the steps beyond multiply pad rows, which are zero, and are skipped)
+struct TileCoord { int e, m0, n0, kblocks, m_lim, last_kk; };
 
 // Warp-cooperative store of a 32-row x 32-column bf16 block whose row `lane` is held by lane
 // `lane` as 32 floats.  Written directly, every store instruction would touch 32 rows with 16
@@ -346,10 +348,12 @@ __device__ __forceinline__ bool tile_coord(const TcParams& p, const int* tile_pr
   if (p.dyn == TC_DYN_M) {
     mt_count = (min(n_e, p.M) + TC_BM - 1) / TC_BM;
     tc.kblocks = (p.K + TC_BK - 1) / TC_BK;
+    tc.last_kk = TC_BK / 16;
     tc.m_lim = mt_count * TC_BM;
   } else {
     mt_count = (p.M + TC_BM - 1) / TC_BM;
     tc.kblocks = (n_e + TC_BK - 1) / TC_BK;
+    tc.last_kk = n_e > 0 ? ((n_e - 1) % TC_BK) / 16 + 1 : TC_BK / 16;
     tc.m_lim = p.M;
   }
   tc.e = e_cur;
@@ -654,10 +658,12 @@ __device__ __forceinline__ bool tile_coord_pair(const TcParams& p, const int* ti
   if (p.dyn == TC_DYN_M) {
     mt_count = (min(n_e, p.M) + 255) / 256;
     tc.kblocks = (p.K + TC_BK - 1) / TC_BK;
+    tc.last_kk = TC_BK / 16;
     tc.m_lim = (min(n_e, p.M) + TC_BM - 1) / TC_BM * TC_BM;
   } else {
     mt_count = (p.M + 255) / 256;
     tc.kblocks = (n_e + TC_BK - 1) / TC_BK;
+    tc.last_kk = n_e > 0 ? ((n_e - 1) % TC_BK) / 16 + 1 : TC_BK / 16;
     tc.m_lim = p.M;
   }
   tc.e = e_cur;
@@ -797,7 +803,13 @@ tc_grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap mapA0, const __g
         if (!mbar_wait_cluster(tempty_bar + 8 * acc_stage, acc_phase ^ 1u, abort_flag, p.wait_limit)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc_stage * 256);
-        for (int kb = 0; kb < tc.kblocks; ++kb) {
+        // A contraction over the expert's rows (operand modes 3, or the generic form) ends in a K block
+        // whose last 16-wide steps may hold pad rows only: that block is peeled off the loop and runs
+        // just the steps with rows in use (the skipped ones would add zeros).  The loop itself stays
+        // free of the test: anything extra in it shows in the GEMM time.
+        constexpr bool PEEL = CFG < 0 || CFG == 3;
+        const int nloop = PEEL ? tc.kblocks - 1 : tc.kblocks;
+        for (int kb = 0; kb < nloop; ++kb) {
           if (!mbar_wait_cluster(full_bar + 8 * stage, phase, abort_flag, p.wait_limit)) { ok = false; break; }
           tc_fence_after();
           const uint32_t sa = tiles_base + stage * TC2_STAGE_BYTES;
@@ -809,6 +821,22 @@ tc_grouped_gemm_pair_kernel(const __grid_constant__ CUtensorMap mapA0, const __g
             tc_mma_pair(d_tmem, ad, bd, p.idesc, (kb > 0 || kk > 0) ? 1u : 0u);
           }
           tc_commit_pair(empty_bar + 8 * stage);      // frees the stage in both CTAs
+          if (++stage == TC2_STAGES) { stage = 0; phase ^= 1u; }
+        }
+        if (PEEL && ok) {
+          if (!mbar_wait_cluster(full_bar + 8 * stage, phase, abort_flag, p.wait_limit)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sa = tiles_base + stage * TC2_STAGE_BYTES;
+          const uint32_t sb = sa + 2 * TC_BOX_BYTES;
+#pragma unroll
+          for (int kk = 0; kk < TC_BK / 16; ++kk) {
+            if (kk < tc.last_kk) {
+              const uint64_t ad = make_smem_desc(sa + kk * a_kstep, a_lbo, 1024u);
+              const uint64_t bd = make_smem_desc(sb + kk * b_kstep, b_lbo, 1024u);
+              tc_mma_pair(d_tmem, ad, bd, p.idesc, (nloop > 0 || kk > 0) ? 1u : 0u);
+            }
+          }
+          tc_commit_pair(empty_bar + 8 * stage);
           if (++stage == TC2_STAGES) { stage = 0; phase ^= 1u; }
         }
         if (!ok) break;
@@ -900,10 +928,12 @@ __device__ __forceinline__ bool tile_coord_wide(const TcParams& p, const int* ti
   if (p.dyn == TC_DYN_M) {
     mt_count = (min(n_e, p.M) + 255) / 256;
     tc.kblocks = (p.K + TC_BK - 1) / TC_BK;
+    tc.last_kk = TC_BK / 16;
     tc.m_lim = (min(n_e, p.M) + TC_BM - 1) / TC_BM * TC_BM;
   } else {
     mt_count = (p.M + 255) / 256;
     tc.kblocks = (n_e + TC_BK - 1) / TC_BK;
+    tc.last_kk = n_e > 0 ? ((n_e - 1) % TC_BK) / 16 + 1 : TC_BK / 16;
     tc.m_lim = p.M;
   }
   tc.e = e_cur;
