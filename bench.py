@@ -39,10 +39,10 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # under profiles/ (absent: not captured for the current version of that kernel).
 NCU_TRAFFIC_BYTES = {}
 # tc_grouped_gemm_pair_kernel and its wide form: measured on the mid workload, all 7 launches of one step
-# (profiles/tc_grouped_gemm_pair_kernels_mid_ncu_full.md): 3670.4 MB of DRAM traffic against 3799.7 MB
+# (profiles/tc_grouped_gemm_pair_kernels_mid_ncu_full.md): 3674.3 MB of DRAM traffic against 3799.7 MB
 # of algorithmic bytes (part of the output is still in L2 when a kernel ends).  The large workload is
 # too big for a multi-pass capture, so its traffic is this ratio times its own algorithmic bytes.
-TC_GEMM_DRAM_OVER_ALGORITHMIC = 3670.4 / 3799.7
+TC_GEMM_DRAM_OVER_ALGORITHMIC = 3674.3 / 3799.7
 
 
 def tc_gemm_algorithmic_bytes(w, rows_padded):
