@@ -96,7 +96,7 @@ def test_expert_parallel_layer_on_two_ranks_sharing_the_gpu():
     procs = [ctx.Process(target=_rank_main, args=(r, world, port, q)) for r in range(world)]
     for p in procs:
         p.start()
-    res = sorted(q.get(timeout=600) for _ in range(world))
+    res = sorted(q.get(timeout=240) for _ in range(world))
     for p in procs:
         p.join(timeout=120)
     assert [r[1] for r in res] == ["ok", "ok"], res
