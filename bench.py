@@ -272,6 +272,27 @@ def timed_steps(layer, n, barrier):
     return e0.elapsed_time(e1)
 
 
+def graph_ms_per_step(layer, n, barrier):
+    """One step captured in a CUDA graph (the calls enqueue stream work only) and replayed n times."""
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        layer.step()
+    torch.cuda.current_stream().wait_stream(side)
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        layer.step()
+    g.replay()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record()
+    for _ in range(n):
+        g.replay()
+    e1.record()
+    barrier()
+    return e0.elapsed_time(e1) / n
+
+
 def per_kernel_pass(etr, layer, n, barrier):
     """n more steps with an event pair around every launch; [(kernel, ms)]."""
     etr.timing_enable(True)
@@ -335,11 +356,12 @@ def measure_other(etr, name, w, dev, args, barrier, peaks, inp=None, weights=Non
     ms = timed_steps(layer, steps, barrier) / steps
     kernels = kernel_table(w, per_kernel_pass(etr, layer, steps, barrier), st.rows_total, st.unrouted, steps, peaks,
                            peaks["bf16_tflops"], None, dev)
+    ms_graph = graph_ms_per_step(layer, steps, barrier)
     assert layer.buf.read_stats().error_word == 0
     g = gemm_summary(w, kernels, st.rows_total)
     out = {"workload": name, "T": w.T, "mode": mode_name(w), "C": st.C, "capacity": w.capacity,
            "rows": st.rows_total, "unrouted": st.unrouted, "delta_max": st.delta_max, "steps": steps,
-           "ms_per_step": ms, "tokens_per_s": w.T / (ms * 1e-3)}
+           "ms_per_step": ms, "tokens_per_s": w.T / (ms * 1e-3), "ms_per_step_cuda_graph": ms_graph}
     if g:
         out.update(gemm_tflops=g["tflops"], gemm_frac_of_burst_peak=g["tflops"] / peaks["bf16_tflops"],
                    gemm_share_of_step=g["share_of_step"])

@@ -264,3 +264,51 @@ def test_top1_combine_in_the_down_gemm_epilogue(name, cf, impl):
     etr.layer_forward(cfg2, dev.X, dev.R, dev.W1g, dev.W1u, dev.W2, buf2, Y2)
     assert "combine_kernel" in [n for n, _ in etr.timing_collect()]
     etr.timing_enable(False)
+
+
+@pytest.mark.parametrize("name", ["small_s", "sweep_s_ecr"])
+def test_layer_calls_can_be_captured_in_a_cuda_graph(name):
+    """etr_layer_forward + etr_layer_backward enqueue only stream work (kernels and one memset; mode,
+    capacity and row counts stay on the device), so a step can be captured once and replayed: the
+    replays must give the bits of the direct calls, also after the inputs changed in place."""
+    w, inp, o, fw, bw = case(name)
+    cfg = hz.make_cfg(w, delta_max_override=override_of(name) if w.adaptive else -1.0)
+    dev = hz.upload(w, inp)
+    buf = etr.LayerBuffers(cfg)
+    out = dict(Y=torch.empty_like(dev.X), dX=torch.empty_like(dev.X), dR=torch.empty_like(dev.R),
+               dW1g=torch.empty_like(dev.W1g), dW1u=torch.empty_like(dev.W1u), dW2=torch.empty_like(dev.W2))
+
+    def step():
+        etr.layer_forward(cfg, dev.X, dev.R, dev.W1g, dev.W1u, dev.W2, buf, out["Y"])
+        etr.layer_backward(cfg, dev.X, dev.R, dev.W1g, dev.W1u, dev.W2, dev.dY, buf, out["dX"], out["dR"],
+                           out["dW1g"], out["dW1u"], out["dW2"])
+
+    step()                                        # direct calls first (and every kernel's one-time set-up)
+    torch.cuda.synchronize()
+    ref = {k: v.clone() for k, v in out.items()}
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        step()
+    torch.cuda.current_stream().wait_stream(side)
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        step()
+    for v in out.values():
+        v.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert buf.read_stats().error_word == 0
+    for k in ref:
+        assert torch.equal(out[k], ref[k]), k
+    # other tokens in the same buffers: the replay follows the data (routing is decided on the device)
+    X0 = dev.X.clone()
+    dev.X.copy_(X0.flip(0))
+    graph.replay()
+    torch.cuda.synchronize()
+    got = {k: v.clone() for k, v in out.items()}
+    step()
+    torch.cuda.synchronize()
+    for k in got:
+        assert torch.equal(out[k], got[k]), k
+    assert not torch.equal(got["Y"], ref["Y"])
