@@ -174,8 +174,8 @@ class ClockSampler:
 def oracle_sample_run(w, inputs_host, weights_host, Ts, steps, warmup, threads=None, gpu_routing=None):
     """Times the CPU oracle (as it stands) on the first Ts tokens of the workload, all experts.
 
-    The sample's capacity is scaled so that it does the same work per token as the GPU step when the
-    GPU step's routing is known (gpu_routing = (C, rows, T)): C_sample = max(1, round(C * Ts / T)),
+    The sample's capacity is scaled so that it does the same work per token as the full step when the
+    full step's routing is known (gpu_routing = (C, rows, T)): C_sample = max(1, round(C * Ts / T)),
     fixed, not adaptive.  Otherwise the workload's own rule on Ts tokens."""
     from oracle import binding as ob
     cores = ob.set_threads(threads or os.cpu_count() or 1)
@@ -199,7 +199,7 @@ def oracle_sample_run(w, inputs_host, weights_host, Ts, steps, warmup, threads=N
     sec = sum(times) / len(times)
     note = ""
     if gpu_routing is not None:
-        note = f" (the GPU step: {gpu_routing[1] / gpu_routing[2]:.2f} rows per token at C={gpu_routing[0]})"
+        note = f" (the full step: {gpu_routing[1] / gpu_routing[2]:.2f} rows per token at C={gpu_routing[0]})"
     return {"value": Ts / sec, "unit": UNIT, "cores": cores, "kind": "oracle",
             "rows_per_token": rows / Ts,
             "sample": f"first {Ts} tokens of the workload, all {w.E} experts, capacity {capacity}: "
@@ -411,10 +411,27 @@ def main():
             return
         w = w0
         Ts = min(args.cpu_tokens, w.T)
-        inp = gw.make_inputs(replace(w, T=Ts), weights=False)
-        inp["R"] = gw.expert_embeddings(w)
+        routing = None
+        if w.adaptive and Ts < w.T:
+            # The capacity the whole batch gives (its maximum affinity sets the adaptive bound), from the
+            # oracle's own affinity pass over all T tokens, so that the sample does the work per token of
+            # the full step; the timed steps then run on the first Ts tokens.
+            from oracle import binding as ob
+            ob.set_threads(os.cpu_count() or 1)
+            full = gw.make_inputs(w, weights=False)
+            _, _, _, dmax = ob.Oracle("f32").affinity(full["X"], full["R"], w.D)
+            C = ob.capacity_bound(w.d, w.E, w.capacity, 1, True, float(dmax))
+            mode = ob.MODE_TCR if mode_name(w) == "tcr" else ob.MODE_ECR
+            rows = min(C, w.T) * w.E if mode == ob.MODE_ECR else None
+            inp = {"X": full["X"][:Ts].copy(), "dY": full["dY"][:Ts].copy(), "R": full["R"]}
+            del full
+            if rows is not None:
+                routing = (C, rows, w.T)
+        else:
+            inp = gw.make_inputs(replace(w, T=Ts), weights=False)
+            inp["R"] = gw.expert_embeddings(w)
         W = gw.expert_weights(w)
-        base, sec = oracle_sample_run(w, inp, W, Ts, max(1, args.steps), args.warmup)
+        base, sec = oracle_sample_run(w, inp, W, Ts, max(1, args.steps), args.warmup, gpu_routing=routing)
         print(json.dumps({
             "impl": "reference", "metric": METRIC, "value": base["value"], "unit": UNIT,
             "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
