@@ -111,9 +111,16 @@ typedef struct etr_config {
   int32_t gate_mode;          /* etr_gate: what weighs an expert's output in the combine */
   int32_t grad_fp32;          /* != 0: dW1g, dW1u, dW2 are written as fp32 (same shapes) whatever `dtype` is;
                                  0: in `dtype`.  The accumulation is fp32 either way. */
-  int32_t weight_dtype;       /* etr_dtype of W1g, W1u, W2.  Must equal `dtype`: the tensor-core
-                                 instruction takes both operands in one 16-bit type, so a layer with
-                                 bf16 activations and fp32 weights has no kernel (ETR_ERR_UNSUPPORTED) */
+  int32_t weight_dtype;       /* etr_dtype of W1g, W1u, W2: equal to `dtype`, or ETR_F32 under dtype = ETR_BF16
+                                 (fp32 master weights).  The GEMMs take both operands in one 16-bit type,
+                                 so in the mixed case every call that multiplies by the weights
+                                 (etr_expert_ffn, etr_expert_ffn_bwd, etr_layer_forward) first rounds them to
+                                 bf16, nearest even, into the tail of ws (etr_workspace_bytes grows by
+                                 3 E d h 2 bytes), dW1g, dW1u, dW2 are written as fp32 whatever grad_fp32
+                                 says, and etr_layer_backward reads the copies etr_layer_forward left in
+                                 buf->ws (same buffers, weights unchanged in between).  Results equal those of
+                                 a bf16 layer with grad_fp32 on weights rounded beforehand, bit for bit.
+                                 bf16 weights under fp32 activations: ETR_ERR_UNSUPPORTED */
   int32_t threshold_mode;     /* etr_threshold flags: selections also cut by a running sum of affinities */
   float threshold_tau;        /* ETR_THRESHOLD_EXPERT: the sum at which an expert stops taking tokens */
   float threshold_tau_token;  /* ETR_THRESHOLD_TOKEN: the sum at which a token stops taking experts */

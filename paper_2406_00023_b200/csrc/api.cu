@@ -57,6 +57,41 @@ static bool fuse_combine(const etr_config* c) {
   return use_tc(c) && c->fuse_combine != ETR_FUSE_OFF && c->k == 1 && resolve_mode(c) == ETR_MODE_TCR;
 }
 
+// bf16 activations with fp32 expert weights (master weights of mixed-precision training): the GEMMs take
+// both operands in one 16-bit type, so every call that multiplies by the weights first rounds them to bf16
+// (round to nearest even) into the tail of the workspace, and the weight gradients come back in fp32.
+static bool mixed_weights(const etr_config* c) { return c->dtype == ETR_BF16 && c->weight_dtype == ETR_F32; }
+static size_t scratch_bytes(const etr_config* c) {      // the part of ws the stages use from offset 0
+  size_t w = select_workspace_bytes(c);
+  w = w > affinity_bwd_workspace_bytes(c) ? w : affinity_bwd_workspace_bytes(c);
+  if (use_tc(c)) w = w > tc_workspace_bytes(c) ? w : tc_workspace_bytes(c);
+  return align_up(w, 256);
+}
+static size_t weight_elems(const etr_config* c) { return (size_t)c->E * c->d * c->h; }
+struct ExpertWeights { const void *W1g, *W1u, *W2; };
+// The weights the kernels read: the caller's, or their bf16 copies behind the scratch part of ws
+// (written here when `cast`, otherwise taken as an earlier call on the same ws left them).
+static etr_status kernel_weights(const etr_config* c, const void* W1g, const void* W1u, const void* W2, void* ws,
+                                 bool cast, ExpertWeights* out, cudaStream_t st) {
+  *out = ExpertWeights{W1g, W1u, W2};
+  if (!mixed_weights(c)) return ETR_OK;
+  if (ws == nullptr) return ETR_ERR_ARG;
+  const size_t n = weight_elems(c);
+  char* base = (char*)ws + scratch_bytes(c);
+  void* dst[3] = {base, base + 2 * n, base + 4 * n};
+  const void* src[3] = {W1g, W1u, W2};
+  if (cast)
+    for (int i = 0; i < 3; ++i) ETR_TRY(cast_f32_to_bf16(src[i], dst[i], n, st));
+  *out = ExpertWeights{dst[0], dst[1], dst[2]};
+  return ETR_OK;
+}
+// The configuration the GEMM stages see under mixed weights: bf16 weights, fp32 weight gradients.
+static etr_config gemm_config(const etr_config* c) {
+  etr_config g = *c;
+  if (mixed_weights(c)) { g.weight_dtype = ETR_BF16; g.grad_fp32 = 1; }
+  return g;
+}
+
 static etr_status check_ptrs(std::initializer_list<const void*> ps) {
   for (const void* p : ps) {
     if (p == nullptr) return ETR_ERR_ARG;
@@ -161,7 +196,7 @@ etr_status etr_validate(const etr_config* c) {
                                                   c->threshold_tau_token != c->threshold_tau_token))
     return ETR_ERR_ARG;                                   // NaN thresholds
   if (c->wait_limit_cycles < 0) return ETR_ERR_ARG;
-  if (c->weight_dtype != c->dtype) return ETR_ERR_UNSUPPORTED;
+  if (c->weight_dtype != c->dtype && !(c->dtype == ETR_BF16 && c->weight_dtype == ETR_F32)) return ETR_ERR_UNSUPPORTED;
   if (c->d % c->D != 0 || c->d % 8 != 0 || c->h % 8 != 0) return ETR_ERR_SHAPE;
   if (c->k > c->E || c->E > 256 || c->E > c->d / c->D) return ETR_ERR_SHAPE;
   if ((long long)c->T * c->E >= (1ll << 31)) return ETR_ERR_SHAPE;
@@ -178,10 +213,7 @@ int32_t etr_c_stride(const etr_config* c) { return c ? c_stride_of(c) : 0; }
 etr_status etr_workspace_bytes(const etr_config* c, size_t* bytes) {
   if (bytes == nullptr) return ETR_ERR_ARG;
   ETR_TRY(etr_validate(c));
-  size_t w = select_workspace_bytes(c);
-  w = w > affinity_bwd_workspace_bytes(c) ? w : affinity_bwd_workspace_bytes(c);
-  if (use_tc(c)) w = w > tc_workspace_bytes(c) ? w : tc_workspace_bytes(c);
-  *bytes = align_up(w, 256);
+  *bytes = scratch_bytes(c) + (mixed_weights(c) ? align_up(3 * 2 * weight_elems(c), 256) : 0);
   return ETR_OK;
 }
 
@@ -258,11 +290,15 @@ etr_status etr_expert_ffn(const etr_config* c, const etr_route* route, const voi
   ETR_TRY(etr_validate(c));
   ETR_TRY(check_ptrs({Xp, W1g, W1u, W2, G, U, H, O}));
   ETR_TRY(check_route(route));
+  ExpertWeights w;
+  ETR_TRY(kernel_weights(c, W1g, W1u, W2, ws, true, &w, (cudaStream_t)stream));
+  const etr_config g = gemm_config(c);
   if (use_tc(c)) {
     ETR_TRY(check_ptrs({stats, ws}));
-    return tc_ffn_forward(c, route, Xp, nullptr, W1g, W1u, W2, G, U, H, O, stats, ws, nullptr, (cudaStream_t)stream);
+    return tc_ffn_forward(&g, route, Xp, nullptr, w.W1g, w.W1u, w.W2, G, U, H, O, stats, ws, nullptr,
+                          (cudaStream_t)stream);
   }
-  return simt_ffn_forward(c, route, Xp, W1g, W1u, W2, G, U, H, O, (cudaStream_t)stream);
+  return simt_ffn_forward(&g, route, Xp, w.W1g, w.W1u, w.W2, G, U, H, O, (cudaStream_t)stream);
 }
 
 etr_status etr_combine(const etr_config* c, const etr_route* route, const void* O, void* Y,
@@ -281,21 +317,35 @@ etr_status etr_combine_bwd(const etr_config* c, const etr_route* route, const vo
   return combine_backward(c, route, dY, O, dO, dgate, (cudaStream_t)stream);
 }
 
+// cast_weights: under mixed weights, round the fp32 weights to bf16 now (false: an earlier call on the same
+// ws, the layer's forward pass, already left them there).
+static etr_status expert_ffn_bwd(const etr_config* c, const etr_route* route, const void* dO,
+                                 const void* Xp, const void* G, const void* U, const void* H,
+                                 const void* W1g, const void* W1u, const void* W2, void* dG, void* dU,
+                                 void* dXp, void* dW1g, void* dW1u, void* dW2, etr_stats* stats,
+                                 void* ws, bool cast_weights, void* stream) {
+  ETR_TRY(etr_validate(c));
+  ETR_TRY(check_ptrs({dO, Xp, G, U, H, W1g, W1u, W2, dG, dU, dXp, dW1g, dW1u, dW2}));
+  ETR_TRY(check_route(route));
+  ExpertWeights w;
+  ETR_TRY(kernel_weights(c, W1g, W1u, W2, ws, cast_weights, &w, (cudaStream_t)stream));
+  const etr_config g = gemm_config(c);
+  if (use_tc(c)) {
+    ETR_TRY(check_ptrs({stats, ws}));
+    return tc_ffn_backward(&g, route, dO, Xp, nullptr, G, U, H, w.W1g, w.W1u, w.W2, dG, dU, dXp, dW1g, dW1u, dW2,
+                           stats, ws, (cudaStream_t)stream);
+  }
+  return simt_ffn_backward(&g, route, dO, Xp, G, U, H, w.W1g, w.W1u, w.W2, dG, dU, dXp, dW1g, dW1u, dW2,
+                           (cudaStream_t)stream);
+}
+
 etr_status etr_expert_ffn_bwd(const etr_config* c, const etr_route* route, const void* dO,
                               const void* Xp, const void* G, const void* U, const void* H,
                               const void* W1g, const void* W1u, const void* W2, void* dG, void* dU,
                               void* dXp, void* dW1g, void* dW1u, void* dW2, etr_stats* stats,
                               void* ws, void* stream) {
-  ETR_TRY(etr_validate(c));
-  ETR_TRY(check_ptrs({dO, Xp, G, U, H, W1g, W1u, W2, dG, dU, dXp, dW1g, dW1u, dW2}));
-  ETR_TRY(check_route(route));
-  if (use_tc(c)) {
-    ETR_TRY(check_ptrs({stats, ws}));
-    return tc_ffn_backward(c, route, dO, Xp, nullptr, G, U, H, W1g, W1u, W2, dG, dU, dXp, dW1g, dW1u, dW2,
-                           stats, ws, (cudaStream_t)stream);
-  }
-  return simt_ffn_backward(c, route, dO, Xp, G, U, H, W1g, W1u, W2, dG, dU, dXp, dW1g, dW1u, dW2,
-                           (cudaStream_t)stream);
+  return expert_ffn_bwd(c, route, dO, Xp, G, U, H, W1g, W1u, W2, dG, dU, dXp, dW1g, dW1u, dW2, stats, ws, true,
+                        stream);
 }
 
 etr_status etr_dispatch_bwd(const etr_config* c, const etr_route* route, const void* dXp, void* dX,
@@ -379,8 +429,11 @@ etr_status etr_layer_forward(const etr_config* c, const void* X, const float* R,
     const bool fd = fuse_dispatch(c);      // the first GEMM gathers its rows from X: no Xp
     ETR_TRY(check_ptrs({X, W1g, W1u, W2, b->G, b->U, b->H, b->O, b->ws}));
     if (!fd) ETR_TRY(etr_dispatch(c, X, &b->route, b->Xp, stream));
-    ETR_TRY(tc_ffn_forward(c, &b->route, fd ? nullptr : b->Xp, fd ? X : nullptr, W1g, W1u, W2, b->G, b->U, b->H,
-                           b->O, b->stats, b->ws, fc ? Y : nullptr, (cudaStream_t)stream));
+    ExpertWeights w;
+    ETR_TRY(kernel_weights(c, W1g, W1u, W2, b->ws, true, &w, (cudaStream_t)stream));
+    const etr_config g = gemm_config(c);
+    ETR_TRY(tc_ffn_forward(&g, &b->route, fd ? nullptr : b->Xp, fd ? X : nullptr, w.W1g, w.W1u, w.W2, b->G, b->U,
+                           b->H, b->O, b->stats, b->ws, fc ? Y : nullptr, (cudaStream_t)stream));
   } else {
     ETR_TRY(etr_dispatch(c, X, &b->route, b->Xp, stream));
     ETR_TRY(etr_expert_ffn(c, &b->route, b->Xp, W1g, W1u, W2, b->G, b->U, b->H, b->O, b->stats, b->ws,
@@ -398,11 +451,14 @@ etr_status etr_layer_backward(const etr_config* c, const void* X, const float* R
     ETR_TRY(etr_validate(c));
     ETR_TRY(check_ptrs({X, b->dO, b->G, b->U, b->H, W1g, W1u, W2, b->dG, b->dU, b->dXp, dW1g, dW1u, dW2,
                         b->stats, b->ws}));
-    ETR_TRY(tc_ffn_backward(c, &b->route, b->dO, nullptr, X, b->G, b->U, b->H, W1g, W1u, W2, b->dG, b->dU,
+    ExpertWeights w;
+    ETR_TRY(kernel_weights(c, W1g, W1u, W2, b->ws, false, &w, (cudaStream_t)stream));
+    const etr_config g = gemm_config(c);
+    ETR_TRY(tc_ffn_backward(&g, &b->route, b->dO, nullptr, X, b->G, b->U, b->H, w.W1g, w.W1u, w.W2, b->dG, b->dU,
                             b->dXp, dW1g, dW1u, dW2, b->stats, b->ws, (cudaStream_t)stream));
   } else {
-    ETR_TRY(etr_expert_ffn_bwd(c, &b->route, b->dO, b->Xp, b->G, b->U, b->H, W1g, W1u, W2, b->dG, b->dU,
-                               b->dXp, dW1g, dW1u, dW2, b->stats, b->ws, stream));
+    ETR_TRY(expert_ffn_bwd(c, &b->route, b->dO, b->Xp, b->G, b->U, b->H, W1g, W1u, W2, b->dG, b->dU,
+                           b->dXp, dW1g, dW1u, dW2, b->stats, b->ws, false, stream));
   }
   // dispatch backward and the router gradient in one pass over dX
   ETR_TRY(etr_select_bwd(c, &b->route, b->dgate));

@@ -220,6 +220,8 @@ etr_status tc_ffn_forward(const etr_config* cfg, const etr_route* route, const v
 // Y_top1 != nullptr (Top-1 token choice only): the down GEMM's epilogue also writes gate * O of every
 // row in use to the row of its token in Y; rows of tokens without a row are not touched.
 etr_status zero_unrouted_rows(const etr_config* c, const etr_route* rt, void* Y, cudaStream_t st);
+// n fp32 values rounded to bf16 (nearest even); n a multiple of 8, both pointers 16-byte aligned
+etr_status cast_f32_to_bf16(const void* src, void* dst, size_t n, cudaStream_t st);
 etr_status tc_ffn_backward(const etr_config* cfg, const etr_route* route, const void* dO,
                            const void* Xp, const void* X_tokens, const void* G, const void* U, const void* H,
                            const void* W1g, const void* W1u, const void* W2, void* dG, void* dU,

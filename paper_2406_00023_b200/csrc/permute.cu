@@ -210,4 +210,31 @@ etr_status dispatch_backward(const etr_config* c, const etr_route* rt, const voi
   return permute_dispatch(3, c, rt, dXp, nullptr, dX, nullptr, st);
 }
 
+
+// fp32 -> bf16 (round to nearest even), eight values per thread: the expert weights of a layer that keeps
+// fp32 master weights, rounded once per pass for the GEMMs.
+__global__ void __launch_bounds__(256) cast_f32_to_bf16_kernel(const float4* __restrict__ src, uint4* __restrict__ dst,
+                                                               size_t n8) {
+  for (size_t i = (size_t)blockIdx.x * 256 + threadIdx.x; i < n8; i += (size_t)gridDim.x * 256) {
+    const float4 a = src[2 * i], b = src[2 * i + 1];
+    const __nv_bfloat162 p0 = __floats2bfloat162_rn(a.x, a.y), p1 = __floats2bfloat162_rn(a.z, a.w);
+    const __nv_bfloat162 p2 = __floats2bfloat162_rn(b.x, b.y), p3 = __floats2bfloat162_rn(b.z, b.w);
+    dst[i] = make_uint4(*reinterpret_cast<const uint32_t*>(&p0), *reinterpret_cast<const uint32_t*>(&p1),
+                        *reinterpret_cast<const uint32_t*>(&p2), *reinterpret_cast<const uint32_t*>(&p3));
+  }
+}
+
+etr_status cast_f32_to_bf16(const void* src, void* dst, size_t n, cudaStream_t st) {
+  if (src == nullptr || dst == nullptr) return ETR_ERR_ARG;
+  if (n % 8 != 0) return ETR_ERR_SHAPE;
+  if (!aligned16(src) || !aligned16(dst)) return ETR_ERR_ALIGN;
+  const size_t n8 = n / 8;
+  const size_t want = (n8 + 255) / 256, cap = (size_t)current_sm_count() * 16;
+  ETR_TIME_BEGIN("cast_weights_kernel");
+  cast_f32_to_bf16_kernel<<<(unsigned)(want < cap ? (want ? want : 1) : cap), 256, 0, st>>>((const float4*)src,
+                                                                                            (uint4*)dst, n8);
+  ETR_LAUNCH_CHECK();
+  return ETR_OK;
+}
+
 }  // namespace etr

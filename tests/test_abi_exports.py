@@ -43,9 +43,14 @@ def test_host_side_validation_needs_no_gpu():
     assert etr.lib().etr_buffers_bytes(ctypes.byref(good), 1, ctypes.byref(n)) == etr.OK and n.value > 1 << 20
     # struct layouts the binding relies on
     assert ctypes.sizeof(etr.Config) == 112 and ctypes.sizeof(etr.Stats) == 64
-    # the expert weights share the activations' dtype: anything else has no kernel
+    # fp32 master weights under bf16 activations are taken (rounded to bf16 in the tail of the workspace, which
+    # grows by three weight tensors of 2 bytes); bf16 weights under fp32 activations have no kernel
     assert etr.validate(etr.make_config(T=512, d=256, D=4, E=8, k=2, h=512, capacity=160, dtype=etr.F32,
                                         weight_dtype=etr.BF16)) == etr.ERR_UNSUPPORTED
+    b16 = etr.make_config(T=512, d=256, D=4, E=8, k=2, h=512, capacity=160, dtype=etr.BF16)
+    mixed = etr.make_config(T=512, d=256, D=4, E=8, k=2, h=512, capacity=160, dtype=etr.BF16, weight_dtype=etr.F32)
+    assert etr.validate(mixed) == etr.OK
+    assert etr.workspace_bytes(mixed) == etr.workspace_bytes(b16) + 3 * 2 * 8 * 256 * 512
 
 
 def test_layout_gives_the_offsets_bind_uses():

@@ -83,6 +83,65 @@ def test_layer_with_fp32_weight_gradients():
         hz.assert_close_rms(hz.to_np(res[True][k]), getattr(bw, k), 2e-2, k + " fp32", chain=chain)
 
 
+@pytest.mark.parametrize("impl", [etr.GEMM_AUTO, etr.GEMM_TCGEN05, etr.GEMM_SIMT])
+def test_fp32_master_weights_with_bf16_activations(impl):
+    """weight_dtype = fp32 under dtype = bf16: the library rounds the weights to bf16 (nearest even) for the
+    GEMMs and returns fp32 weight gradients.  Every output must equal, bit for bit, the bf16 layer with
+    grad_fp32 run on weights rounded the same way beforehand; the fp32 weights here are not on the bf16 grid."""
+    w, inp, o, fw, bw = case("small_s")
+    dev = hz.upload(w, inp)
+    g = torch.Generator(device="cuda").manual_seed(7)
+    master = {}
+    for k in ("W1g", "W1u", "W2"):
+        wb = getattr(dev, k)
+        # the same values to bf16 precision, plus bits below it that rounding must remove again
+        noise = (torch.rand(wb.shape, device="cuda", generator=g) - 0.5) * 2.0 ** -10
+        m32 = wb.float() * (1.0 + noise)
+        assert torch.equal(m32.to(torch.bfloat16), wb) and not torch.equal(m32, wb.float())
+        master[k] = m32.contiguous()
+    res = {}
+    for mixed in (False, True):
+        cfg = hz.make_cfg(w, gemm_impl=impl, grad_fp32=not mixed,
+                          **(dict(weight_dtype=etr.F32) if mixed else {}))
+        W = [master[k] if mixed else getattr(dev, k) for k in ("W1g", "W1u", "W2")]
+        buf = etr.LayerBuffers(cfg)
+        out = dict(Y=torch.empty_like(dev.X), dX=torch.empty_like(dev.X), dR=torch.empty_like(dev.R),
+                   dW1g=torch.empty(dev.W1g.shape, dtype=torch.float32, device="cuda"),
+                   dW1u=torch.empty(dev.W1u.shape, dtype=torch.float32, device="cuda"),
+                   dW2=torch.empty(dev.W2.shape, dtype=torch.float32, device="cuda"))
+        etr.layer_forward(cfg, dev.X, dev.R, *W, buf, out["Y"])
+        etr.layer_backward(cfg, dev.X, dev.R, *W, dev.dY, buf, out["dX"], out["dR"], out["dW1g"], out["dW1u"],
+                           out["dW2"])
+        torch.cuda.synchronize()
+        assert buf.read_stats().error_word == 0
+        # the stage calls round the weights themselves: same G, U, H, O and gradients as the layer's
+        st = dict(G=torch.empty_like(buf.G), U=torch.empty_like(buf.U), H=torch.empty_like(buf.H),
+                  O=torch.empty_like(buf.O), dG=torch.empty_like(buf.dG), dU=torch.empty_like(buf.dU),
+                  dXp=torch.empty_like(buf.dXp), dW1g=torch.empty_like(out["dW1g"]),
+                  dW1u=torch.empty_like(out["dW1u"]), dW2=torch.empty_like(out["dW2"]))
+        ws = torch.empty(etr.workspace_bytes(cfg), dtype=torch.uint8, device="cuda")
+        etr.expert_ffn(cfg, buf.route, buf.Xp, *W, st["G"], st["U"], st["H"], st["O"], buf.c.stats, ws)
+        etr.expert_ffn_bwd(cfg, buf.route, buf.dO, buf.Xp, buf.G, buf.U, buf.H, *W, st["dG"], st["dU"], st["dXp"],
+                           st["dW1g"], st["dW1u"], st["dW2"], buf.c.stats, ws)
+        torch.cuda.synchronize()
+        live = buf.slot_token >= 0                   # rows beyond an expert's count are not part of the result
+        for k in ("G", "U", "H", "O", "dG", "dU", "dXp"):
+            assert torch.equal(st[k].view(live.numel(), -1)[live], getattr(buf, k).view(live.numel(), -1)[live]), k
+        for k in ("dW1g", "dW1u", "dW2"):
+            assert torch.equal(st[k], out[k]), k
+        res[mixed] = out
+    for k in res[False]:
+        assert torch.equal(res[False][k], res[True][k]), k
+    hz.assert_close_rms(hz.to_np(res[True]["dW2"]), bw.dW2, 2e-2, "dW2 fp32 master", chain=3)
+
+
+def test_mixed_weight_dtype_is_bf16_activations_only():
+    w = gw.WORKLOADS["tiny"]
+    assert w.dtype == "f32"
+    with pytest.raises(etr.EtrError):
+        etr.workspace_bytes(hz.make_cfg(w, weight_dtype=etr.BF16))      # fp32 activations, bf16 weights
+
+
 @pytest.mark.parametrize("name", ["small_s", "sweep_s_ecr"])
 def test_select_may_be_repeated_on_one_stats_block(name):
     """The selection sets every counter it reports: a second selection on the same stats (another
