@@ -79,6 +79,7 @@ def algorithmic_work(w, rows, kernel, unrouted=0):
         "affinity_fwd_warp_kernel": (T * d * b + T * E * 4 + T * m * 4 + T * 4, "bytes"),
         "grap_pool_kernel": (T * d * b + T * m * 4 + T * 4, "bytes"),
         "affinity_score_kernel": (2 * T * m * E, "fp32_flops"),        # the product z R^T: fp32 FMA issue, not HBM
+        "affinity_score_tc_kernel": (T * m * 4 + T * E * 4 + T * 4, "bytes"),   # the same product on the tensor cores
         "select_token_side_kernel": (2 * T * E * 4, "bytes"),
         "select_expert_side_kernel": (T * E * 4 + rows * 8, "bytes"),
         "csr_count_kernel": (T * E * 4, "bytes"),

@@ -8,7 +8,8 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libetr.so")
-SOURCES = ["api.cu", "affinity.cu", "select.cu", "permute.cu", "gate.cu", "gemm_simt.cu", "gemm_tcgen05.cu"]
+SOURCES = ["api.cu", "affinity.cu", "select.cu", "permute.cu", "gate.cu", "gemm_simt.cu", "gemm_tcgen05.cu",
+           "score_tcgen05.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-shared"]
 

@@ -1160,6 +1160,13 @@ static etr_status affinity_forward_split(const etr_config* c, const void* X, con
   if (((size_t)(32 * EPL + 4 * TPG) * ldm + 32 * EPL) * sizeof(float) > 220 * 1024) return ETR_OK;
   if (c->dtype == ETR_BF16) ETR_TRY(launch_pool<__nv_bfloat16>(c, X, Z, xnorm, st));
   else ETR_TRY(launch_pool<float>(c, X, Z, xnorm, st));
+  // The product on the tensor cores wherever its shape rules hold, whatever the token count: a token's
+  // affinities must not depend on how a batch is cut (an expert-parallel rank scores its own tokens).
+  if (affinity_score_tc_takes(c, Z, R, delta)) {
+    ETR_TRY(affinity_score_tc(c, Z, xnorm, R, delta, rnorm, stats, st));
+    *done = true;
+    return ETR_OK;
+  }
   // the tiled form needs a tile of 256 tokens for every SM to pay for its set-up (R and its norms per block)
   if (c->E <= 64 && m % SC_KC == 0 && ceil_div(c->T, SC_TM) >= current_sm_count()) {
     if (c->E <= 16) ETR_TRY(launch_score_tile<2>(c, Z, xnorm, R, delta, rnorm, stats, st, done));

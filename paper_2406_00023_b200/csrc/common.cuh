@@ -182,6 +182,10 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
 etr_status affinity_forward(const etr_config* c, const void* X, const float* R, float* delta,
                             float* Z, float* xnorm, float* rnorm, etr_stats* stats, cudaStream_t st);
 size_t affinity_bwd_workspace_bytes(const etr_config* c);
+// score_tcgen05.cu: the score product on the tensor cores (E <= 64, 32 | d/D, 16-byte aligned Z, R, delta)
+bool affinity_score_tc_takes(const etr_config* c, const float* Z, const float* R, const float* delta);
+etr_status affinity_score_tc(const etr_config* c, const float* Z, const float* xnorm, const float* R, float* delta,
+                             float* rnorm, etr_stats* stats, cudaStream_t st);
 etr_status affinity_backward(const etr_config* c, const void* X, const float* R, const float* delta,
                              const float* Z, const float* xnorm, const float* rnorm,
                              const etr_route* rt, const float* dgate, const float* ddelta,
