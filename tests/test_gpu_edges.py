@@ -121,11 +121,51 @@ def test_fused_dx_at_wide_hidden_sizes(d, D, dtype):
     assert n.min() == 0 and n.max() >= 6 and n.sum() > 3 * w.T
 
 
-@pytest.mark.parametrize("E,dtype", [(16, "bf16"), (32, "f32"), (64, "bf16")])
-def test_affinity_with_a_score_tile_for_every_sm(E, dtype):
-    """38100 tokens: at least one 256-token tile per SM, which is when the score kernel takes its
-    register-tiled form (2, 4 or 8 experts per lane for E <= 16, 32, 64), and a ragged last tile."""
-    w = gw.scaled(W["small"], T=38100, d=512, D=8, E=E, h=64, dtype=dtype)
+def _affinity_on_device(w, inp, rows=None):
+    cfg = hz.make_cfg(w if rows is None else gw.scaled(w, T=rows.stop - rows.start))
+    X = hz.to_dev(inp["X"] if rows is None else inp["X"][rows], w)
+    R = torch.from_numpy(inp["R"]).cuda()
+    T, m = X.shape[0], w.d // w.D
+    delta = torch.empty(T, w.E, dtype=torch.float32, device="cuda")
+    Z = torch.empty(T, m, dtype=torch.float32, device="cuda")
+    xnorm = torch.empty(T, dtype=torch.float32, device="cuda")
+    rnorm = torch.empty(w.E, dtype=torch.float32, device="cuda")
+    stats = torch.zeros(16, dtype=torch.int32, device="cuda")
+    etr.affinity(cfg, X, R, delta, Z, xnorm, rnorm, stats)
+    torch.cuda.synchronize()
+    assert int(stats[6].item()) == 0            # error_word
+    return delta, rnorm, stats
+
+
+@pytest.mark.parametrize("T,d,D,E,dtype", [(1000, 256, 8, 7, "bf16"), (130, 512, 4, 64, "f32"), (4097, 2048, 8, 33, "bf16"),
+                                            (127, 64, 2, 1, "bf16"), (20000, 1024, 4, 12, "bf16")])
+def test_affinity_scores_on_the_tensor_cores(T, d, D, E, dtype):
+    """Shapes the tensor-core score kernel takes (E <= 64, 32 | d/D): expert counts that are not a multiple of 4
+    (scalar stores), a single expert, one K block, a ragged last tile of tokens, more tiles than SMs.  Affinities
+    within the usual 1e-5, the batch maximum equal to the largest affinity stored, and a token's affinities the
+    same bits whether it is scored in the whole batch or in a slice of it."""
+    w = gw.scaled(W["small"], T=T, d=d, D=D, E=E, k=1, h=64, dtype=dtype)
+    assert E <= 64 and (d // D) % 32 == 0
+    inp = gw.make_inputs(w, weights=False)
+    delta_ref, _, rnorm_ref, _ = ob.Oracle("f32").affinity(inp["X"], inp["R"], w.D)
+    delta, rnorm, stats = _affinity_on_device(w, inp)
+    got = hz.to_np(delta)
+    hz.assert_affinity_close(got, delta_ref)
+    assert np.allclose(hz.to_np(rnorm), rnorm_ref, rtol=1e-6, atol=0)
+    u = int(np.float32(got.max()).view(np.uint32))
+    key = (~u & 0xffffffff) if (u & 0x80000000) else (u | 0x80000000)
+    assert int(stats[5].item()) & 0xffffffff == key
+    rows = slice(T // 3, T // 3 + min(300, T - T // 3))
+    part, _, _ = _affinity_on_device(w, inp, rows)
+    assert torch.equal(part, delta[rows])
+
+
+@pytest.mark.parametrize("E,dtype,d", [(16, "bf16", 640), (32, "f32", 640), (64, "bf16", 640), (64, "bf16", 512)])
+def test_affinity_with_a_score_tile_for_every_sm(E, dtype, d):
+    """38100 tokens: at least one 256-token tile per SM and a ragged last tile.  With d/D = 80 (16 divides it, 32
+    does not) the fp32 score kernel takes its register-tiled form (2, 4 or 8 experts per lane for E <= 16, 32,
+    64); with d/D = 64 the tensor-core kernel takes the same batch."""
+    w = gw.scaled(W["small"], T=38100, d=d, D=8, E=E, h=64, dtype=dtype)
     inp = gw.make_inputs(w, weights=False)
     delta_ref, *_ = ob.Oracle("f32").affinity(inp["X"], inp["R"], w.D)
     cfg = hz.make_cfg(w)
