@@ -3,17 +3,17 @@
 //
 // The router decides on these numbers, so they keep fp32 accuracy: every fp32 operand v is split in
 // shared memory into hi = v with its low 13 mantissa bits cleared (exactly a tf32 value) and
-// lo = (v - hi) cut the same way, and the product is accumulated as lo*hi + hi*lo + hi*hi in the fp32
-// accumulator in tensor memory.  The products of two tf32 values are exact in fp32; what is dropped is
+// lo = (v - hi) cut the same way, and the product is accumulated as hi*hi + hi*lo + lo*hi in fp32
+// accumulators in tensor memory.  The products of two tf32 values are exact in fp32; what is dropped is
 // lo*lo (2^-22 of a product) and the second cut of lo (2^-24).  Both operand splits are made by a group
 // of converter warps between the TMA load and the MMA, in place, so the caller's Z and R stay plain
 // fp32 and no scratch memory is needed.
 //
 // Roles in a CTA of 320 threads: warp 0 lane 0 loads (TMA, 128-byte swizzle: a K block is 32 floats of
-// every row), warps 2-5 split, warp 1 lane 0 issues the MMAs, warps 6-9 read the accumulator (two
-// stages of 64 columns), scale by the norms, store delta and track the batch maximum.  All waits are
-// bounded; on expiry the kernel leaves 0x7c09 in etr_stats.error_word, frees its tensor memory and
-// returns.
+// every row), warps 2-5 split, warp 1 lane 0 issues the MMAs, warps 6-9 read the accumulators (two
+// stages of four 64-column partial sums: all 512 columns), add them, scale by the norms, store delta
+// through a staging tile (whole 128-byte rows) and track the batch maximum.  All waits are bounded; on
+// expiry the kernel leaves 0x7c09 in etr_stats.error_word, frees its tensor memory and returns.
 #include <algorithm>
 
 #include "common.cuh"
@@ -29,7 +29,7 @@ constexpr int SCT_THREADS = 320;
 constexpr uint32_t SCT_A_BYTES = SCT_BM * SCT_BK * 4;      // 16 KiB
 constexpr uint32_t SCT_B_BYTES = SCT_N * SCT_BK * 4;       //  8 KiB
 constexpr uint32_t SCT_STAGE_BYTES = 2 * SCT_A_BYTES + 2 * SCT_B_BYTES;      // hi and lo of both
-constexpr int SCT_CHAINS = SCT_BK / 8;              // independent accumulators of a tile (one per 8-float step of a K block)
+constexpr int SCT_CHAINS = 4;                       // 64-column partial sums of a tile: two chains x {hi*hi + lo*hi, hi*lo}
 constexpr uint32_t SCT_TMEM_COLS = 2 * SCT_CHAINS * SCT_N;      // two stages of them: 512 columns
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
@@ -105,6 +105,7 @@ affinity_score_tc_kernel(const __grid_constant__ CUtensorMap mapZ, const __grid_
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = tmem_base_slot;
+  const uint32_t idesc_wide = (idesc & ~(0x3fu << 17)) | ((uint32_t)(2 * SCT_N >> 3) << 17);      // N = 128
   const int ntiles = (Ttok + SCT_BM - 1) / SCT_BM, nkb = m / SCT_BK;
 
   if (warp == 0) {
@@ -139,16 +140,24 @@ affinity_score_tc_kernel(const __grid_constant__ CUtensorMap mapZ, const __grid_
           tc_fence_after();
           const uint32_t a_hi = tiles_base + stage * SCT_STAGE_BYTES, a_lo = a_hi + SCT_A_BYTES;
           const uint32_t b_hi = a_hi + 2 * SCT_A_BYTES, b_lo = b_hi + SCT_B_BYTES;
-          // 8 floats (32 bytes) per MMA.  Step kk of every K block adds into accumulator kk: consecutive
-          // MMAs then never wait for one another's result (these are small MMAs, 128 x 64 x 8, whose latency
-          // is several times their time in the pipe); the epilogue adds the four partial sums.
+          // 8 floats (32 bytes) per MMA, two MMAs per step: the hi and lo tiles of R lie one behind the other in
+          // the stage, so A_hi x [R_hi; R_lo]^T is ONE MMA of 128 expert columns (hi*hi in columns 0-63 of the
+          // chain, hi*lo in 64-127), and A_lo x R_hi^T adds lo*hi to columns 0-63.  These are small MMAs whose
+          // issue costs about 75 cycles each whatever their width, and the issue lane is the longest stage.
+          // Even and odd steps add into different chains (128 columns each), so that consecutive MMAs do not
+          // wait for one another's result; the epilogue adds the four 64-column partial sums.
 #pragma unroll
-          for (int term = 0; term < 3; ++term) {
+          for (int pairk = 0; pairk < SCT_BK / 8; pairk += 2) {
 #pragma unroll
-            for (int kk = 0; kk < SCT_CHAINS; ++kk) {
-              const uint64_t ad = make_smem_desc((term == 0 ? a_lo : a_hi) + 32 * kk, 16u, 1024u);
-              const uint64_t bd = make_smem_desc((term == 1 ? b_lo : b_hi) + 32 * kk, 16u, 1024u);
-              tc_mma_tf32(d_tmem + (uint32_t)(kk * SCT_N), ad, bd, idesc, (kb > 0 || term > 0) ? 1u : 0u);
+            for (int term = 0; term < 2; ++term) {
+#pragma unroll
+              for (int c = 0; c < 2; ++c) {
+                const int kk = pairk + c;
+                const uint64_t ad = make_smem_desc((term == 0 ? a_hi : a_lo) + 32 * kk, 16u, 1024u);
+                const uint64_t bd = make_smem_desc(b_hi + 32 * kk, 16u, 1024u);
+                tc_mma_tf32(d_tmem + (uint32_t)(c * 2 * SCT_N), ad, bd, term == 0 ? idesc_wide : idesc,
+                            (kb > 0 || pairk > 0 || term > 0) ? 1u : 0u);
+              }
             }
           }
           tc_commit(empty_bar + 8 * stage);
@@ -179,6 +188,7 @@ affinity_score_tc_kernel(const __grid_constant__ CUtensorMap mapZ, const __grid_
   } else {
     // ---- epilogue warps: a lane owns a token --------------------------------------------------------------
     const int q = warp & 3;                      // tensor-memory lanes 32 q .. 32 q + 31
+    float* stg = reinterpret_cast<float*>(tiles + (size_t)SCT_STAGES * SCT_STAGE_BYTES) + (warp - 6) * 32 * 33;
     // ||R_i|| while the first tile is on its way: a warp per row, lanes over the columns, the same sums
     // as the other score kernels (eight columns per lane requested together)
     for (int i = q; i < SCT_N; i += 4) {
@@ -226,29 +236,33 @@ affinity_score_tc_kernel(const __grid_constant__ CUtensorMap mapZ, const __grid_
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(tempty_bar + 8 * acc);      // the values are in registers
-      if (t < Ttok) {
-        float* out = delta + (size_t)t * E;
+      // scale: delta = sqrt(D) s / (||x|| ||R_i||), 0 where a norm is 0.  A fast division (reciprocal and product,
+      // 2 ulp) taken unconditionally and selected afterwards: 64 correctly rounded divisions per token, each behind
+      // its own zero test, overlapped with nothing and were the longest stage of the kernel; the result is
+      // compared at 1e-5, not to the last bit.
 #pragma unroll
-        for (int i = 0; i < SCT_N; ++i) {
-          if (i < E) {
-            const float den = xn * rn[i];
-            // a fast division (reciprocal and product, 2 ulp) taken unconditionally: 64 correctly rounded ones per
-            // token, each behind its own branch, were the longest stage of this kernel (no two overlapped), and
-            // the result is compared at 1e-5, not to the last bit
-            const float quot = __fdividef(sqD * __uint_as_float(r[i]), den);      // computed first: a select, no branch
-            const float v = den == 0.f ? 0.f : quot;
-            r[i] = __float_as_uint(v);
-            best = fmaxf(best, v);
-          }
-        }
-        if ((E & 3) == 0) {
+      for (int i = 0; i < SCT_N; ++i) {
+        const float den = xn * rn[i];
+        const float quot = __fdividef(sqD * __uint_as_float(r[i]), den);
+        const float v = den == 0.f ? 0.f : quot;
+        r[i] = __float_as_uint(v);
+        if (i < E && t < Ttok) best = fmaxf(best, v);
+      }
+      // store: a lane holds a token's row, but 32 lanes writing 32 different rows would send 16 bytes per
+      // sector.  The warp turns 32 x 32 blocks through its staging tile (row stride 33 words: no bank
+      // conflicts either way) and writes 128 contiguous bytes of one token per instruction.
+      const int t_warp = tile * SCT_BM + 32 * q;
 #pragma unroll
-          for (int i = 0; i < SCT_N; i += 4)
-            if (i < E) *reinterpret_cast<uint4*>(out + i) = make_uint4(r[i], r[i + 1], r[i + 2], r[i + 3]);
-        } else {
+      for (int half = 0; half < SCT_N / 32; ++half) {
+        if (32 * half < E) {
+          __syncwarp();
 #pragma unroll
-          for (int i = 0; i < SCT_N; ++i)
-            if (i < E) out[i] = __uint_as_float(r[i]);
+          for (int j = 0; j < 32; ++j) stg[lane * 33 + j] = __uint_as_float(r[32 * half + j]);
+          __syncwarp();
+          const int i = 32 * half + lane;
+          const int nrow = min(32, Ttok - t_warp);
+          for (int rr = 0; rr < nrow; ++rr)
+            if (i < E) delta[(size_t)(t_warp + rr) * E + i] = stg[rr * 33 + lane];
         }
       }
       if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
@@ -299,7 +313,7 @@ etr_status affinity_score_tc(const etr_config* c, const float* Z, const float* x
   CUtensorMap mapZ, mapR;
   ETR_TRY(make_map_f32(&mapZ, Z, m, c->T, SCT_BM));
   ETR_TRY(make_map_f32(&mapR, R, m, c->E, SCT_N));
-  constexpr size_t smem = (size_t)SCT_STAGES * SCT_STAGE_BYTES + 1024;
+  constexpr size_t smem = (size_t)SCT_STAGES * SCT_STAGE_BYTES + 1024 + 4 * 32 * 33 * sizeof(float);      // stages, alignment, staging
   static std::atomic<unsigned long long> attr_done{0};      // one bit per device
   if (!ensure_dyn_smem(affinity_score_tc_kernel, smem, attr_done)) return ETR_ERR_CUDA;
   uint32_t idesc = 0;
