@@ -212,7 +212,12 @@ etr_status etr_layout(const etr_config* cfg, int with_host_staging, etr_layout_i
  *   z_t = avgpool_D(x_t);  delta_ti = sqrt(D) <z_t, R_i> / (||x_t|| ||R_i||), 0 if a norm is 0.
  * Writes delta, xnorm, rnorm, optionally Z (NULL to skip), and raises
  * stats->delta_max_key to the batch maximum.  stats must have been zeroed by the caller
- * (etr_layer_forward does it) — the call only ever raises the key. */
+ * (etr_layer_forward does it) — the call only ever raises the key.
+ * Arithmetic: fp32 throughout.  With Z given, E <= 64 and 32 | d/D the products <z_t, R_i> run on the
+ * tensor cores as tf32 MMAs on operands split into two tf32 parts each (hi*hi + hi*lo + lo*hi in an fp32
+ * accumulator: what is dropped is 2^-22 of a product), otherwise as fp32 FMAs; either way within 1e-5 of
+ * the exact quotient relative to max(|delta|, rms(delta)).  A token's affinities depend on that token,
+ * R and the shape (d, D, E) only, not on T or on which other tokens share the batch. */
 etr_status etr_affinity(const etr_config* cfg, const void* X, const float* R, float* delta,
                         float* Z, float* xnorm, float* rnorm, etr_stats* stats, void* stream);
 
